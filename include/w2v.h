@@ -1,0 +1,219 @@
+/*
+ * w2v.h -- C ABI of libw2v: the skip-gram negative-sampling (SGNS) minibatch
+ * step of "Network-Efficient Distributed Word2vec Training System for Large
+ * Vocabularies" (arXiv 1606.08495) on one NVIDIA B200 (sm_100a).
+ *
+ * The paper spreads one minibatch over parameter-server shards: each shard
+ * holds a column slice of every input vector u(w) and output vector v(w),
+ * returns partial dot products (Algorithm 1, "dotprod"), the client sums them
+ * and forms the coefficients G+ = a(1 - s(F+)), G- = -a s(F-) (Algorithm 3),
+ * and the shards apply the linear combinations (Algorithm 2, "adjust").  On
+ * one GPU the shards become the lanes of a warp, each owning a column slice,
+ * and the two remote calls and the client sum become one kernel.
+ *
+ * Conventions
+ *   - Every function returns a w2v_status (0 = success, negative = error); no
+ *     exception crosses this boundary and nothing aborts.  w2v_last_error()
+ *     gives a text for the last failure on a handle.
+ *   - "device" pointers are CUDA device memory owned by the caller; the
+ *     library never frees or reallocates them.  "host" pointers are ordinary
+ *     host memory.  The handle owns only its sampling tables and scratch.
+ *   - All work is enqueued on the stream given to w2v_create.  Calls that
+ *     return values to the host synchronise that stream; the others are
+ *     asynchronous.
+ *   - Tables are row-major fp32: row w of U (input vectors) or V (output
+ *     vectors) is d consecutive floats at offset w*d.  Row index = rank of the
+ *     word by decreasing frequency (Section 5.1, the ordering O).
+ *   - Token streams are int32 word ids in [0, vocab); -1 ends a sentence;
+ *     any other value is skipped as out of vocabulary and reported.  Windows
+ *     are taken over the tokens that survive sub-sampling ("dirty" contexts,
+ *     footnote to Section 3) and never cross a sentence end or the chunk edge.
+ *   - Random choices are a pure function of (seed, step number, token index):
+ *     a Philox4x32-10 counter-based generator stands in for the seeded
+ *     generator of Algorithms 1 and 2, so that any party regenerates the same
+ *     negatives from the same seed, as the paper's shards do.
+ *   - Limits: 2 <= vocab < 2^31, d a multiple of 4 with 4 <= d <= 1024,
+ *     1 <= window <= 127, 1 <= negatives <= 64, n < 2^31 tokens per call.
+ */
+#ifndef W2V_H
+#define W2V_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct w2v_handle w2v_handle;
+
+typedef enum {
+    W2V_OK = 0,
+    W2V_ERR_ARG = -1,          /* NULL pointer or value outside the documented limits */
+    W2V_ERR_STATE = -2,        /* e.g. a step before w2v_build_alias */
+    W2V_ERR_NOMEM = -3,        /* device or host allocation failed */
+    W2V_ERR_CUDA = -4,         /* a CUDA runtime call failed; see w2v_last_error */
+    W2V_ERR_TOKEN_RANGE = -5,  /* the chunk held ids outside [-1, vocab); they were skipped */
+    W2V_ERR_CAPACITY = -6      /* an output array was too small; see the call */
+} w2v_status;
+
+enum { W2V_MODE_SNAPSHOT = 0, W2V_MODE_HOGWILD = 1 };
+enum { W2V_TABLE_U = 0, W2V_TABLE_V = 1 };
+
+/* Counters of one step (or one w2v_sample_pairs call). */
+typedef struct {
+    uint64_t tokens;       /* entries in the chunk */
+    uint64_t kept;         /* word tokens that survived sub-sampling */
+    uint64_t centres;      /* kept tokens with at least one context */
+    uint64_t pairs;        /* positive (centre, context) pairs */
+    uint64_t neg_draws;    /* alias-table draws, re-draws included */
+    uint64_t neg_redraws;  /* draws thrown away because they hit the context word */
+    uint64_t oov;          /* ids outside [-1, vocab) */
+    uint32_t status;       /* bit 0: out-of-vocabulary ids seen */
+    uint32_t reserved;
+} w2v_step_stats;
+
+/*
+ * Create a model: U ~ uniform[-0.5/d, 0.5/d), V = 0 ("initialized ... as in
+ * word2vec", Section 5.1).  U[w][j] = (x - 0.5)/d with x = (r >> 8) 2^-24 and r
+ * word j%4 of Philox(key = seed; counter = (w, j/4, 0, 0)).
+ *   U, V    device, caller-owned, vocab*d floats each, 16-byte aligned; or both
+ *           NULL, in which case the library allocates and owns them.
+ *   stream  a cudaStream_t (NULL = the legacy default stream).
+ *   out     host; receives the handle.
+ * The current CUDA device at the time of the call becomes the handle's device.
+ * Asynchronous.  Errors: W2V_ERR_ARG, W2V_ERR_NOMEM, W2V_ERR_CUDA.
+ */
+int32_t w2v_create(uint64_t vocab, uint32_t d, uint64_t seed, float *U, float *V,
+                   void *stream, w2v_handle **out);
+
+/* Waits for the handle's stream, frees what the handle owns.  NULL is accepted. */
+int32_t w2v_destroy(w2v_handle *h);
+
+/*
+ * Build the sampling tables from the vocabulary histogram (Section 5.1,
+ * "a probability distribution derived from the vocabulary histogram";
+ * Section 3, sub-sampling of frequent words) and upload them.
+ *   counts       host, vocab entries, all >= 1 (else W2V_ERR_ARG).
+ *   subsample_t  keep probability min(1, sqrt(x) + x), x = t * sum(counts) / count;
+ *                t <= 0 keeps every token.
+ * Negatives follow count^(3/4) / sum count^(3/4) through a Vose alias table
+ * with 32-bit thresholds; weight = sqrt(c) * sqrt(sqrt(c)) in fp64.
+ * Synchronises the stream.  May be called again to replace the tables.
+ */
+int32_t w2v_build_alias(w2v_handle *h, const uint64_t *counts, double subsample_t);
+
+/*
+ * Download the tables built by w2v_build_alias (for checking them).
+ *   thr, alias, keep_thr  host, vocab entries each; any may be NULL.
+ */
+int32_t w2v_get_tables(w2v_handle *h, uint32_t *thr, uint32_t *alias, uint32_t *keep_thr);
+
+/*
+ * One minibatch step over a chunk of tokens: Eq. (3)-(5), Algorithms 1-3.
+ * Sub-sample, compact, draw one window radius b in 1..window per centre, and
+ * for every (centre, context) pair draw `negatives` words != context from the
+ * alias table; then for every target t of the pair (the context with label 1,
+ * the negatives with label 0): F = u(centre).v(t), G = lr (label - s(F)),
+ * u(centre) += G v(t), v(t) += G u(centre)  -- summed over the chunk, not averaged.
+ *   tokens  device, n int32 entries.
+ *   mode    W2V_MODE_SNAPSHOT: every dot and every linear combination uses the
+ *           tables as they were at the start of the call and the sums are applied
+ *           at the end (Section 5.1, "not updated until the end of the call").
+ *           W2V_MODE_HOGWILD: one pass, updates land as they are computed and
+ *           later reads may or may not see them (Section 5.1, no locking).
+ *   stats   host, may be NULL.  Non-NULL: the call waits for the step and fills
+ *           it, and returns W2V_ERR_TOKEN_RANGE if bad ids were skipped.  NULL:
+ *           the step is only enqueued (Hogwild mode never waits; snapshot mode
+ *           waits once to size its coefficient array).
+ * Adds one to the step number.  Scratch is grown on the first call with a
+ * larger n and reused afterwards: no allocation in the steady state.
+ * Errors: W2V_ERR_ARG, W2V_ERR_STATE (no tables), W2V_ERR_NOMEM, W2V_ERR_CUDA.
+ */
+int32_t w2v_sgns_step(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window,
+                      uint32_t negatives, float lr, uint32_t mode, w2v_step_stats *stats);
+
+/*
+ * The same step with the chunk in HOST memory (pinned memory makes the copy
+ * asynchronous): copies it to a staging buffer owned by the handle, then
+ * behaves exactly as w2v_sgns_step.
+ */
+int32_t w2v_sgns_step_host(w2v_handle *h, const int32_t *tokens_host, uint64_t n, uint32_t window,
+                           uint32_t negatives, float lr, uint32_t mode, w2v_step_stats *stats);
+
+/*
+ * The index sets the next step would use (same seed, same step number), without
+ * touching the tables or the step number: W_input / W_output of Algorithm 3 and
+ * the negatives NS of Algorithms 1 and 2.  Pairs are ordered by centre position,
+ * then context position.
+ *   centre, context  device, cap int32 each;  negs  device, cap*negatives int32.
+ *   n_pairs          host; receives the number of pairs (also when > cap, in
+ *                    which case only the first cap are written and the call
+ *                    returns W2V_ERR_CAPACITY).
+ *   stats            host, may be NULL.
+ * Synchronises the stream.
+ */
+int32_t w2v_sample_pairs(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window,
+                         uint32_t negatives, int32_t *centre, int32_t *context, int32_t *negs,
+                         uint64_t cap, uint64_t *n_pairs, w2v_step_stats *stats);
+
+/*
+ * Partial dot products of one column slice, the body of Algorithm 1 on shard s:
+ * out[i] = sum_{j = col_lo}^{col_hi - 1} U[pairs[2i]][j] * V[pairs[2i+1]][j].
+ * Summing the results over any partition of [0, d) gives the full dot products
+ * (Algorithm 3, "(F+, F-) <- sum_s").
+ *   pairs  device, m*2 int32 (input row, output row), each in [0, vocab).
+ *   out    device, m floats.
+ * Asynchronous.  Rows out of range leave out[i] = NaN and set status bit 0.
+ * Errors: W2V_ERR_ARG unless 0 <= col_lo < col_hi <= d.
+ */
+int32_t w2v_partial_dots(w2v_handle *h, const int32_t *pairs, uint64_t m, uint32_t col_lo,
+                         uint32_t col_hi, float *out);
+
+/*
+ * Copy rows out of / into a table (the "get" of the vector export, Section 6.1).
+ *   which  W2V_TABLE_U or W2V_TABLE_V.
+ *   ids    device, m int64 row numbers; rows outside [0, vocab) are skipped
+ *          (read: the output row is left untouched).
+ *   out/in device, m*d floats.
+ * Asynchronous.
+ */
+int32_t w2v_read_rows(w2v_handle *h, uint32_t which, const int64_t *ids, uint64_t m, float *out);
+int32_t w2v_write_rows(w2v_handle *h, uint32_t which, const int64_t *ids, uint64_t m, const float *in);
+
+/* Step number used by the next step (resume = write the rows back, set the step). */
+int32_t w2v_set_step(w2v_handle *h, uint64_t step_id);
+int32_t w2v_get_step(w2v_handle *h, uint64_t *step_id);
+
+/* Device pointers of the two tables (caller's or library-owned). */
+int32_t w2v_get_table_ptrs(w2v_handle *h, float **U, float **V);
+
+/* Wait for the handle's stream; returns W2V_ERR_CUDA if a kernel failed. */
+int32_t w2v_sync(w2v_handle *h);
+
+/*
+ * Timing of the update kernels with CUDA events on the handle's stream.
+ * w2v_profile_enable(h, 1) starts recording one event pair around every launch of
+ * the step's update kernel(s); w2v_profile_read waits for the stream and returns
+ * the summed device time in milliseconds and the number of launches since the
+ * last read, then resets both.
+ */
+int32_t w2v_profile_enable(w2v_handle *h, int32_t on);
+int32_t w2v_profile_read(w2v_handle *h, double *kernel_ms, uint64_t *launches);
+
+/* Number of kernels this handle has launched since it was created. */
+int32_t w2v_get_launch_count(w2v_handle *h, uint64_t *launches);
+
+/*
+ * Launch shape of the update kernels: rows in flight per warp (1..8; 0 = default)
+ * and resident thread blocks per SM (0 = as many as fit).  Results do not depend
+ * on it in snapshot mode.
+ */
+int32_t w2v_set_tuning(w2v_handle *h, uint32_t rows_in_flight, uint32_t blocks_per_sm);
+
+/* Text of the last error on this handle (never NULL; h == NULL gives a generic text). */
+const char *w2v_last_error(w2v_handle *h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* W2V_H */

@@ -1,0 +1,521 @@
+// C-ABI layer of libw2v: argument checks, the handle, scratch management and the
+// sequence of kernel launches that makes one step.  See include/w2v.h for the contract.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/w2v.h"
+#include "w2v_internal.h"
+
+using namespace w2v;
+
+struct w2v_handle {
+    uint64_t vocab = 0;
+    uint32_t d = 0;
+    uint64_t seed = 0;
+    uint64_t step_id = 0;
+    int device = 0;
+    int sms = 148;
+    cudaStream_t stream = nullptr;
+    float *U = nullptr, *V = nullptr;
+    bool owns_tables = false;
+    // sampling tables
+    uint32_t *keep_thr = nullptr;
+    uint2 *alias = nullptr;
+    bool have_tables = false;
+    // scratch
+    Scratch sc;
+    DevState *st = nullptr;          // device
+    DevState *st_host = nullptr;     // pinned mirror
+    float *G = nullptr;
+    uint64_t G_cap = 0;
+    float *DU = nullptr;
+    uint64_t DU_cap = 0;             // floats
+    int32_t *tok_stage = nullptr;
+    uint64_t tok_stage_cap = 0;
+    // tuning / accounting
+    uint32_t rows_in_flight = 0, blocks_per_sm = 0;
+    uint64_t launches = 0;
+    bool profiling = false;
+    std::vector<cudaEvent_t> ev;     // pairs (start, stop)
+    size_t ev_used = 0;
+    double prof_ms = 0.0;
+    uint64_t prof_launches = 0;
+    char err[256] = "no error";
+};
+
+namespace {
+
+int32_t fail(w2v_handle *h, int32_t code, const char *what, cudaError_t ce = cudaSuccess)
+{
+    if (h) {
+        if (ce != cudaSuccess)
+            std::snprintf(h->err, sizeof(h->err), "%s: %s", what, cudaGetErrorString(ce));
+        else
+            std::snprintf(h->err, sizeof(h->err), "%s", what);
+    }
+    return code;
+}
+
+#define W2V_CUDA(h, call)                                                     \
+    do {                                                                      \
+        cudaError_t ce_ = (call);                                             \
+        if (ce_ != cudaSuccess)                                               \
+            return fail(h, ce_ == cudaErrorMemoryAllocation ? W2V_ERR_NOMEM : W2V_ERR_CUDA, #call, ce_); \
+    } while (0)
+
+struct DeviceGuard {
+    int prev = -1;
+    explicit DeviceGuard(int dev) { cudaGetDevice(&prev); if (prev != dev) cudaSetDevice(dev); else prev = -1; }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+template <typename T>
+cudaError_t dev_alloc(T **p, uint64_t count)
+{
+    return cudaMalloc(reinterpret_cast<void **>(p), (count ? count : 1) * sizeof(T));
+}
+
+void free_scratch(Scratch &sc)
+{
+    cudaFree(sc.flags); cudaFree(sc.tile_sums); cudaFree(sc.tile_offs); cudaFree(sc.ctok);
+    cudaFree(sc.cidx); cudaFree(sc.csent); cudaFree(sc.win); cudaFree(sc.cnt_tile); cudaFree(sc.pair_off);
+    sc = Scratch();
+}
+
+// Scratch for chunks of up to n tokens; grows only.
+int32_t ensure_scratch(w2v_handle *h, uint64_t n)
+{
+    if (n <= h->sc.n_cap) return W2V_OK;
+    W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+    free_scratch(h->sc);
+    const uint64_t tiles = (n + kScanTile - 1) / kScanTile + 1;
+    Scratch &sc = h->sc;
+    W2V_CUDA(h, dev_alloc(&sc.flags, n));
+    W2V_CUDA(h, dev_alloc(&sc.tile_sums, tiles));
+    W2V_CUDA(h, dev_alloc(&sc.tile_offs, tiles));
+    W2V_CUDA(h, dev_alloc(&sc.ctok, n));
+    W2V_CUDA(h, dev_alloc(&sc.cidx, n));
+    W2V_CUDA(h, dev_alloc(&sc.csent, n));
+    W2V_CUDA(h, dev_alloc(&sc.win, n));
+    W2V_CUDA(h, dev_alloc(&sc.cnt_tile, tiles));
+    W2V_CUDA(h, dev_alloc(&sc.pair_off, n + 1));
+    sc.n_cap = n;
+    return W2V_OK;
+}
+
+int32_t check_step_args(w2v_handle *h, const void *tokens, uint64_t n, uint32_t window, uint32_t negatives)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (!tokens && n) return fail(h, W2V_ERR_ARG, "tokens is NULL");
+    if (n >= (1ull << 31)) return fail(h, W2V_ERR_ARG, "n must be below 2^31");
+    if (window < 1 || window > 127) return fail(h, W2V_ERR_ARG, "window must be in 1..127");
+    if (negatives < 1 || negatives > 64) return fail(h, W2V_ERR_ARG, "negatives must be in 1..64");
+    if (!h->have_tables) return fail(h, W2V_ERR_STATE, "w2v_build_alias has not been called");
+    return W2V_OK;
+}
+
+StepParams make_params(w2v_handle *h, uint32_t window, uint32_t negatives, float lr)
+{
+    StepParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.U = h->U; p.V = h->V;
+    p.tab.keep_thr = h->keep_thr; p.tab.alias = h->alias;
+    p.ctok = h->sc.ctok; p.cidx = h->sc.cidx; p.win = h->sc.win;
+    p.st = h->st;
+    p.vocab = (uint32_t)h->vocab; p.d4 = h->d / 4;
+    p.window = window; p.negatives = negatives;
+    p.k0 = (uint32_t)h->seed;
+    p.k1 = (uint32_t)(h->seed >> 32) ^ (uint32_t)(h->step_id >> 32);
+    p.step_lo = (uint32_t)h->step_id;
+    p.lr = lr;
+    p.pair_off = h->sc.pair_off; p.G = h->G; p.DU = h->DU;
+    return p;
+}
+
+// sub-sampling, compaction and windows for the chunk; counters zeroed first
+int32_t enqueue_sampling(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window)
+{
+    int32_t rc = ensure_scratch(h, n);
+    if (rc != W2V_OK) return rc;
+    W2V_CUDA(h, cudaMemsetAsync(h->st, 0, sizeof(DevState), h->stream));
+    const uint32_t k0 = (uint32_t)h->seed;
+    const uint32_t k1 = (uint32_t)(h->seed >> 32) ^ (uint32_t)(h->step_id >> 32);
+    const uint32_t step_lo = (uint32_t)h->step_id;
+    SampleTables tab{h->keep_thr, h->alias};
+    int k = launch_compact(tokens, n, tab, (uint32_t)h->vocab, k0, k1, step_lo, h->sc, h->st, h->stream);
+    if (k < 0) return fail(h, W2V_ERR_CUDA, "compaction launch", cudaGetLastError());
+    h->launches += (uint64_t)k;
+    k = launch_windows(n, window, k0, k1, step_lo, h->sc, h->st, h->stream);
+    if (k < 0) return fail(h, W2V_ERR_CUDA, "window launch", cudaGetLastError());
+    h->launches += (uint64_t)k;
+    return W2V_OK;
+}
+
+int32_t read_state(w2v_handle *h, uint64_t n, w2v_step_stats *stats)
+{
+    W2V_CUDA(h, cudaMemcpyAsync(h->st_host, h->st, sizeof(DevState), cudaMemcpyDeviceToHost, h->stream));
+    W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+    if (stats) {
+        const DevState &s = *h->st_host;
+        stats->tokens = n; stats->kept = s.n_kept; stats->centres = s.centres; stats->pairs = s.pairs;
+        stats->neg_draws = s.neg_draws; stats->neg_redraws = s.neg_redraws; stats->oov = s.oov;
+        stats->status = s.status; stats->reserved = 0;
+    }
+    return W2V_OK;
+}
+
+void profile_collect(w2v_handle *h)
+{
+    for (size_t i = 0; i + 1 < h->ev_used; i += 2) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, h->ev[i], h->ev[i + 1]) == cudaSuccess) h->prof_ms += ms;
+    }
+    h->ev_used = 0;
+}
+
+// records an event on the stream; every second call closes a (start, stop) pair
+int32_t profile_mark(w2v_handle *h)
+{
+    if (!h->profiling) return W2V_OK;
+    if (h->ev_used == h->ev.size()) {
+        if (h->ev.size() >= 512) {           // recycle: wait, fold into the sum, start over
+            W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+            profile_collect(h);
+        } else {
+            cudaEvent_t e;
+            W2V_CUDA(h, cudaEventCreate(&e));
+            h->ev.push_back(e);
+        }
+    }
+    W2V_CUDA(h, cudaEventRecord(h->ev[h->ev_used++], h->stream));
+    return W2V_OK;
+}
+
+int32_t step_impl(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window, uint32_t negatives,
+                  float lr, uint32_t mode, w2v_step_stats *stats)
+{
+    if (mode > 1) return fail(h, W2V_ERR_ARG, "mode must be 0 (snapshot) or 1 (hogwild)");
+    int32_t rc = enqueue_sampling(h, tokens, n, window);
+    if (rc != W2V_OK) return rc;
+    if (mode == W2V_MODE_HOGWILD) {
+        StepParams p = make_params(h, window, negatives, lr);
+        if ((rc = profile_mark(h)) != W2V_OK) return rc;
+        int k = launch_hogwild(p, h->rows_in_flight, h->blocks_per_sm, h->sms, h->stream);
+        if (k < 0) return fail(h, W2V_ERR_CUDA, "update kernel launch", cudaGetLastError());
+        h->launches += (uint64_t)k;
+        if (h->profiling) h->prof_launches += (uint64_t)k;
+        if ((rc = profile_mark(h)) != W2V_OK) return rc;
+    } else {
+        int k = launch_pair_offsets(n, h->sc, h->st, h->stream);
+        if (k < 0) return fail(h, W2V_ERR_CUDA, "pair offset launch", cudaGetLastError());
+        h->launches += (uint64_t)k;
+        // the coefficient array is sized by the pair count, which only the device knows
+        if ((rc = read_state(h, n, nullptr)) != W2V_OK) return rc;
+        const uint64_t need_g = h->st_host->pairs * (uint64_t)(negatives + 1);
+        if (need_g > h->G_cap) {
+            cudaFree(h->G); h->G = nullptr; h->G_cap = 0;
+            const uint64_t cap = need_g + need_g / 4 + 1024;
+            W2V_CUDA(h, dev_alloc(&h->G, cap));
+            h->G_cap = cap;
+        }
+        const uint64_t need_du = h->sc.n_cap * (uint64_t)h->d;
+        if (need_du > h->DU_cap) {
+            cudaFree(h->DU); h->DU = nullptr; h->DU_cap = 0;
+            W2V_CUDA(h, dev_alloc(&h->DU, need_du));
+            h->DU_cap = need_du;
+        }
+        if (h->st_host->pairs > 0) {
+            StepParams p = make_params(h, window, negatives, lr);
+            if ((rc = profile_mark(h)) != W2V_OK) return rc;
+            k = launch_snapshot(p, h->rows_in_flight, h->blocks_per_sm, h->sms, h->stream);
+            if (k < 0) return fail(h, W2V_ERR_CUDA, "update kernel launch", cudaGetLastError());
+            h->launches += (uint64_t)k;
+            if (h->profiling) h->prof_launches += (uint64_t)k;
+            if ((rc = profile_mark(h)) != W2V_OK) return rc;
+        }
+    }
+    h->step_id += 1;
+    if (stats) {
+        if ((rc = read_state(h, n, stats)) != W2V_OK) return rc;
+        if (stats->status & 1u) return fail(h, W2V_ERR_TOKEN_RANGE, "token ids outside [-1, vocab) were skipped");
+    }
+    return W2V_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t w2v_create(uint64_t vocab, uint32_t d, uint64_t seed, float *U, float *V, void *stream,
+                   w2v_handle **out)
+{
+    if (!out) return W2V_ERR_ARG;
+    *out = nullptr;
+    if (vocab < 2 || vocab >= (1ull << 31)) return W2V_ERR_ARG;
+    if (d < 4 || d > 1024 || (d % 4) != 0) return W2V_ERR_ARG;
+    if ((U == nullptr) != (V == nullptr)) return W2V_ERR_ARG;
+    if (U && ((reinterpret_cast<uintptr_t>(U) | reinterpret_cast<uintptr_t>(V)) & 15u)) return W2V_ERR_ARG;
+    w2v_handle *h = new (std::nothrow) w2v_handle();
+    if (!h) return W2V_ERR_NOMEM;
+    h->vocab = vocab; h->d = d; h->seed = seed;
+    h->stream = static_cast<cudaStream_t>(stream);
+    auto bail = [&](int32_t code) { w2v_destroy(h); return code; };
+    if (cudaGetDevice(&h->device) != cudaSuccess) return bail(W2V_ERR_CUDA);
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device) == cudaSuccess && sms > 0)
+        h->sms = sms;
+    const uint64_t elems = vocab * (uint64_t)d;
+    if (!U) {
+        if (dev_alloc(&h->U, elems) != cudaSuccess) { cudaGetLastError(); return bail(W2V_ERR_NOMEM); }
+        h->owns_tables = true;
+        if (dev_alloc(&h->V, elems) != cudaSuccess) { cudaGetLastError(); return bail(W2V_ERR_NOMEM); }
+    } else {
+        h->U = U; h->V = V;
+    }
+    if (dev_alloc(&h->st, 1) != cudaSuccess) return bail(W2V_ERR_NOMEM);
+    if (cudaMallocHost(reinterpret_cast<void **>(&h->st_host), sizeof(DevState)) != cudaSuccess)
+        return bail(W2V_ERR_NOMEM);
+    if (cudaMemsetAsync(h->st, 0, sizeof(DevState), h->stream) != cudaSuccess) return bail(W2V_ERR_CUDA);
+    if (launch_init_tables(h->U, h->V, vocab, d, seed, h->stream) < 0) return bail(W2V_ERR_CUDA);
+    h->launches += 1;
+    *out = h;
+    return W2V_OK;
+}
+
+int32_t w2v_destroy(w2v_handle *h)
+{
+    if (!h) return W2V_OK;
+    DeviceGuard g(h->device);
+    cudaStreamSynchronize(h->stream);
+    if (h->owns_tables) { cudaFree(h->U); cudaFree(h->V); }
+    cudaFree(h->keep_thr); cudaFree(h->alias);
+    free_scratch(h->sc);
+    cudaFree(h->st);
+    if (h->st_host) cudaFreeHost(h->st_host);
+    cudaFree(h->G); cudaFree(h->DU); cudaFree(h->tok_stage);
+    for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
+    cudaGetLastError();
+    delete h;
+    return W2V_OK;
+}
+
+int32_t w2v_build_alias(w2v_handle *h, const uint64_t *counts, double subsample_t)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (!counts) return fail(h, W2V_ERR_ARG, "counts is NULL");
+    DeviceGuard g(h->device);
+    std::vector<uint2> ta;
+    std::vector<uint32_t> keep;
+    try {
+        ta.resize(h->vocab);
+        keep.resize(h->vocab);
+    } catch (const std::bad_alloc &) {
+        return fail(h, W2V_ERR_NOMEM, "host memory for the sampling tables");
+    }
+    int rc;
+    try {
+        rc = build_tables_host(counts, h->vocab, subsample_t, ta.data(), keep.data());
+    } catch (const std::bad_alloc &) {
+        return fail(h, W2V_ERR_NOMEM, "host memory for the sampling tables");
+    }
+    if (rc != 0) return fail(h, W2V_ERR_ARG, "every count must be at least 1");
+    if (!h->alias) W2V_CUDA(h, dev_alloc(&h->alias, h->vocab));
+    if (!h->keep_thr) W2V_CUDA(h, dev_alloc(&h->keep_thr, h->vocab));
+    W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+    W2V_CUDA(h, cudaMemcpyAsync(h->alias, ta.data(), h->vocab * sizeof(uint2), cudaMemcpyHostToDevice, h->stream));
+    W2V_CUDA(h, cudaMemcpyAsync(h->keep_thr, keep.data(), h->vocab * sizeof(uint32_t), cudaMemcpyHostToDevice, h->stream));
+    W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+    h->have_tables = true;
+    return W2V_OK;
+}
+
+int32_t w2v_get_tables(w2v_handle *h, uint32_t *thr, uint32_t *alias, uint32_t *keep_thr)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (!h->have_tables) return fail(h, W2V_ERR_STATE, "w2v_build_alias has not been called");
+    DeviceGuard g(h->device);
+    W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+    if (thr || alias) {
+        std::vector<uint2> ta(h->vocab);
+        W2V_CUDA(h, cudaMemcpy(ta.data(), h->alias, h->vocab * sizeof(uint2), cudaMemcpyDeviceToHost));
+        for (uint64_t w = 0; w < h->vocab; ++w) {
+            if (thr) thr[w] = ta[w].x;
+            if (alias) alias[w] = ta[w].y;
+        }
+    }
+    if (keep_thr)
+        W2V_CUDA(h, cudaMemcpy(keep_thr, h->keep_thr, h->vocab * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    return W2V_OK;
+}
+
+int32_t w2v_sgns_step(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window, uint32_t negatives,
+                      float lr, uint32_t mode, w2v_step_stats *stats)
+{
+    int32_t rc = check_step_args(h, tokens, n, window, negatives);
+    if (rc != W2V_OK) return rc;
+    DeviceGuard g(h->device);
+    return step_impl(h, tokens, n, window, negatives, lr, mode, stats);
+}
+
+int32_t w2v_sgns_step_host(w2v_handle *h, const int32_t *tokens_host, uint64_t n, uint32_t window,
+                           uint32_t negatives, float lr, uint32_t mode, w2v_step_stats *stats)
+{
+    int32_t rc = check_step_args(h, tokens_host, n, window, negatives);
+    if (rc != W2V_OK) return rc;
+    DeviceGuard g(h->device);
+    if (n > h->tok_stage_cap) {
+        W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+        cudaFree(h->tok_stage); h->tok_stage = nullptr; h->tok_stage_cap = 0;
+        W2V_CUDA(h, dev_alloc(&h->tok_stage, n));
+        h->tok_stage_cap = n;
+    }
+    if (n)
+        W2V_CUDA(h, cudaMemcpyAsync(h->tok_stage, tokens_host, n * sizeof(int32_t), cudaMemcpyHostToDevice, h->stream));
+    return step_impl(h, h->tok_stage, n, window, negatives, lr, mode, stats);
+}
+
+int32_t w2v_sample_pairs(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window, uint32_t negatives,
+                         int32_t *centre, int32_t *context, int32_t *negs, uint64_t cap, uint64_t *n_pairs,
+                         w2v_step_stats *stats)
+{
+    int32_t rc = check_step_args(h, tokens, n, window, negatives);
+    if (rc != W2V_OK) return rc;
+    if (!n_pairs) return fail(h, W2V_ERR_ARG, "n_pairs is NULL");
+    if (cap && (!centre || !context || !negs)) return fail(h, W2V_ERR_ARG, "output array is NULL");
+    DeviceGuard g(h->device);
+    if ((rc = enqueue_sampling(h, tokens, n, window)) != W2V_OK) return rc;
+    int k = launch_pair_offsets(n, h->sc, h->st, h->stream);
+    if (k < 0) return fail(h, W2V_ERR_CUDA, "pair offset launch", cudaGetLastError());
+    h->launches += (uint64_t)k;
+    if (n) {
+        StepParams p = make_params(h, window, negatives, 0.f);
+        k = launch_emit_pairs(p, centre, context, negs, cap, h->sms * 8, h->stream);
+        if (k < 0) return fail(h, W2V_ERR_CUDA, "pair list launch", cudaGetLastError());
+        h->launches += (uint64_t)k;
+    }
+    w2v_step_stats local;
+    if ((rc = read_state(h, n, &local)) != W2V_OK) return rc;
+    if (stats) *stats = local;
+    *n_pairs = local.pairs;
+    if (local.pairs > cap) return fail(h, W2V_ERR_CAPACITY, "more pairs than the output arrays hold");
+    if (local.status & 1u) return fail(h, W2V_ERR_TOKEN_RANGE, "token ids outside [-1, vocab) were skipped");
+    return W2V_OK;
+}
+
+int32_t w2v_partial_dots(w2v_handle *h, const int32_t *pairs, uint64_t m, uint32_t col_lo, uint32_t col_hi,
+                         float *out)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (m && (!pairs || !out)) return fail(h, W2V_ERR_ARG, "pairs or out is NULL");
+    if (!(col_lo < col_hi && col_hi <= h->d)) return fail(h, W2V_ERR_ARG, "need 0 <= col_lo < col_hi <= d");
+    DeviceGuard g(h->device);
+    int k = launch_partial_dots(h->U, h->V, (uint32_t)h->vocab, h->d, pairs, m, col_lo, col_hi, out, h->st,
+                                h->sms, h->stream);
+    if (k < 0) return fail(h, W2V_ERR_CUDA, "partial dots launch", cudaGetLastError());
+    h->launches += (uint64_t)k;
+    return W2V_OK;
+}
+
+static int32_t copy_rows(w2v_handle *h, uint32_t which, const int64_t *ids, uint64_t m, float *buf, bool to_table)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (which > 1) return fail(h, W2V_ERR_ARG, "which must be 0 (U) or 1 (V)");
+    if (m && (!ids || !buf)) return fail(h, W2V_ERR_ARG, "ids or buffer is NULL");
+    if (reinterpret_cast<uintptr_t>(buf) & 15u) return fail(h, W2V_ERR_ARG, "row buffer must be 16-byte aligned");
+    DeviceGuard g(h->device);
+    int k = launch_copy_rows(which ? h->V : h->U, (uint32_t)h->vocab, h->d, ids, m, buf, to_table, h->sms, h->stream);
+    if (k < 0) return fail(h, W2V_ERR_CUDA, "row copy launch", cudaGetLastError());
+    h->launches += (uint64_t)k;
+    return W2V_OK;
+}
+
+int32_t w2v_read_rows(w2v_handle *h, uint32_t which, const int64_t *ids, uint64_t m, float *out)
+{
+    return copy_rows(h, which, ids, m, out, false);
+}
+
+int32_t w2v_write_rows(w2v_handle *h, uint32_t which, const int64_t *ids, uint64_t m, const float *in)
+{
+    return copy_rows(h, which, ids, m, const_cast<float *>(in), true);
+}
+
+int32_t w2v_set_step(w2v_handle *h, uint64_t step_id)
+{
+    if (!h) return W2V_ERR_ARG;
+    h->step_id = step_id;
+    return W2V_OK;
+}
+
+int32_t w2v_get_step(w2v_handle *h, uint64_t *step_id)
+{
+    if (!h || !step_id) return W2V_ERR_ARG;
+    *step_id = h->step_id;
+    return W2V_OK;
+}
+
+int32_t w2v_get_table_ptrs(w2v_handle *h, float **U, float **V)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (U) *U = h->U;
+    if (V) *V = h->V;
+    return W2V_OK;
+}
+
+int32_t w2v_sync(w2v_handle *h)
+{
+    if (!h) return W2V_ERR_ARG;
+    DeviceGuard g(h->device);
+    W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+    return W2V_OK;
+}
+
+int32_t w2v_profile_enable(w2v_handle *h, int32_t on)
+{
+    if (!h) return W2V_ERR_ARG;
+    DeviceGuard g(h->device);
+    W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+    profile_collect(h);
+    h->profiling = on != 0;
+    h->prof_ms = 0.0;
+    h->prof_launches = 0;
+    return W2V_OK;
+}
+
+int32_t w2v_profile_read(w2v_handle *h, double *kernel_ms, uint64_t *launches)
+{
+    if (!h) return W2V_ERR_ARG;
+    DeviceGuard g(h->device);
+    W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+    profile_collect(h);
+    if (kernel_ms) *kernel_ms = h->prof_ms;
+    if (launches) *launches = h->prof_launches;
+    h->prof_ms = 0.0;
+    h->prof_launches = 0;
+    return W2V_OK;
+}
+
+int32_t w2v_get_launch_count(w2v_handle *h, uint64_t *launches)
+{
+    if (!h || !launches) return W2V_ERR_ARG;
+    *launches = h->launches;
+    return W2V_OK;
+}
+
+int32_t w2v_set_tuning(w2v_handle *h, uint32_t rows_in_flight, uint32_t blocks_per_sm)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (rows_in_flight > 8) return fail(h, W2V_ERR_ARG, "rows_in_flight must be in 0..8");
+    h->rows_in_flight = rows_in_flight;
+    h->blocks_per_sm = blocks_per_sm;
+    return W2V_OK;
+}
+
+const char *w2v_last_error(w2v_handle *h)
+{
+    return h ? h->err : "invalid handle";
+}
+
+}  // extern "C"

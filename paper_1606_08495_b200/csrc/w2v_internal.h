@@ -1,0 +1,104 @@
+// Internal declarations of libw2v: device-side state, kernel parameter blocks and
+// the host launchers each .cu file exports to the C-ABI layer.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace w2v {
+
+// Counter layout of every random choice (key = seed, with the high word of the step
+// number xor-ed into the high key word):
+//   c0 = token index in the chunk (row number for initialisation)
+//   c1 = low word of the step number (column/4 for initialisation)
+//   c2 = purpose | slot << 8, slot = context position - centre position + window
+//   c3 = k | attempt << 16 (k-th negative of the pair, attempt-th re-draw)
+
+constexpr int kBlock = 256;            // threads per block of the update kernels
+constexpr int kScanBlock = 256;        // threads per block of the compaction kernels
+constexpr int kScanItems = 8;          // tokens per thread
+constexpr int kScanTile = kScanBlock * kScanItems;
+constexpr int kMaxRedraw = 16;
+
+// Counters and results that live on the device during a step.
+struct DevState {
+    unsigned long long n_kept;
+    unsigned long long n_sent;
+    unsigned long long centres;
+    unsigned long long pairs;
+    unsigned long long neg_draws;
+    unsigned long long neg_redraws;
+    unsigned long long oov;
+    unsigned int status;
+    unsigned int pad;
+};
+
+struct SampleTables {
+    const uint32_t *keep_thr;   // [vocab] keep iff thr == 2^32-1 or random word < thr
+    const uint2 *alias;         // [vocab] .x = acceptance threshold, .y = alias
+};
+
+// Everything the kernels of one step need.
+struct StepParams {
+    float *U;
+    float *V;
+    SampleTables tab;
+    // compacted chunk
+    const int32_t *ctok;        // word id of kept token q
+    const uint32_t *cidx;       // its index in the chunk (random counter c0)
+    const uint16_t *win;        // contexts to the left (low byte) and right (high byte)
+    DevState *st;
+    uint32_t vocab;
+    uint32_t d4;                // d / 4
+    uint32_t window;
+    uint32_t negatives;
+    uint32_t k0, k1;            // Philox key
+    uint32_t step_lo;
+    float lr;
+    // snapshot mode / pair list
+    const unsigned long long *pair_off;   // first pair index of centre q
+    float *G;                   // [pairs * (1 + negatives)] coefficients
+    float *DU;                  // [kept * d] per-centre sums of G v(target)
+};
+
+struct Scratch {
+    uint64_t n_cap = 0;
+    uint8_t *flags = nullptr;
+    uint2 *tile_sums = nullptr;
+    uint2 *tile_offs = nullptr;
+    int32_t *ctok = nullptr;
+    uint32_t *cidx = nullptr;
+    uint32_t *csent = nullptr;
+    uint16_t *win = nullptr;
+    unsigned long long *cnt_tile = nullptr;
+    unsigned long long *pair_off = nullptr;
+};
+
+// ---- launchers (each returns the number of kernels it launched, or -1 on a launch error) ----
+int launch_init_tables(float *U, float *V, uint64_t vocab, uint32_t d, uint64_t seed, cudaStream_t s);
+
+int launch_compact(const int32_t *tokens, uint64_t n, const SampleTables &tab, uint32_t vocab,
+                   uint32_t k0, uint32_t k1, uint32_t step_lo, const Scratch &sc, DevState *st,
+                   cudaStream_t s);
+int launch_windows(uint64_t n, uint32_t window, uint32_t k0, uint32_t k1, uint32_t step_lo,
+                   const Scratch &sc, DevState *st, cudaStream_t s);
+int launch_pair_offsets(uint64_t n, const Scratch &sc, DevState *st, cudaStream_t s);
+int launch_emit_pairs(const StepParams &p, int32_t *centre, int32_t *context, int32_t *negs,
+                      uint64_t cap, int grid, cudaStream_t s);
+
+int launch_hogwild(const StepParams &p, uint32_t rows_in_flight, uint32_t blocks_per_sm, int sms,
+                   cudaStream_t s);
+int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t blocks_per_sm, int sms,
+                    cudaStream_t s);
+
+int launch_partial_dots(const float *U, const float *V, uint32_t vocab, uint32_t d,
+                        const int32_t *pairs, uint64_t m, uint32_t col_lo, uint32_t col_hi,
+                        float *out, DevState *st, int sms, cudaStream_t s);
+int launch_copy_rows(float *table, uint32_t vocab, uint32_t d, const int64_t *ids, uint64_t m,
+                     float *buf, bool to_table, int sms, cudaStream_t s);
+
+// ---- host-side table construction (w2v_tables.cpp) ----
+// Returns 0, or -1 if a count is zero.  thr_alias is [vocab] pairs, keep_thr [vocab].
+int build_tables_host(const uint64_t *counts, uint64_t vocab, double subsample_t, uint2 *thr_alias,
+                      uint32_t *keep_thr);
+
+}  // namespace w2v

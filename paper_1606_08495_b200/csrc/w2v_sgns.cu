@@ -1,0 +1,307 @@
+// The floating-point half of the step: gather rows, column-sliced partial dots reduced
+// over the warp, sigmoid coefficients and scatter-add updates (Algorithms 1-3).
+//
+// One warp owns one centre token at a time.  Lane l holds float4 number l, l+32, ... of
+// every row it touches -- a fixed column slice, the role a parameter-server shard has in
+// the paper -- so "sum the shards' partial dot products" (Algorithm 3) is a butterfly of
+// warp shuffles, and "apply the coefficients to the shard's columns" (Algorithm 2) is a
+// 16-byte reduction into global memory per lane.  The centre row u(c) is read once and
+// kept in registers for all its contexts and their 1+N targets.
+#include "w2v_sample.cuh"
+
+namespace w2v {
+
+// Walks the targets of one (centre, context) pair in batches of TB rows so that TB row
+// gathers are in flight before the first dot is reduced.
+//   onTarget(t, target_row, v, f) is called once per target in order t = 0..N with the
+//   gathered row and the full dot product.
+template <int VPL, int TB, typename F>
+__device__ __forceinline__ void for_each_target(const StepParams &p, const Row<VPL> &u, uint32_t w_out,
+                                                uint32_t n0, uint32_t n1, uint32_t lane, F &&onTarget)
+{
+    const float4 *V4 = reinterpret_cast<const float4 *>(p.V);
+    const bool wide = p.negatives > 32u;
+    for (uint32_t t0 = 0; t0 <= p.negatives; t0 += TB) {
+        uint32_t tgt[TB];
+        Row<VPL> v[TB];
+        float f[TB];
+#pragma unroll
+        for (int b = 0; b < TB; ++b) {
+            const uint32_t t = t0 + b;
+            tgt[b] = pair_target(t, w_out, n0, n1, wide);
+            if (t <= p.negatives) row_load(v[b], V4 + (size_t)tgt[b] * p.d4, p.d4, lane);
+            else row_zero(v[b]);
+        }
+#pragma unroll
+        for (int b = 0; b < TB; ++b) f[b] = row_dot_partial(u, v[b]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+            for (int b = 0; b < TB; ++b) f[b] += __shfl_xor_sync(kFullMask, f[b], o);
+        }
+#pragma unroll
+        for (int b = 0; b < TB; ++b) {
+            const uint32_t t = t0 + b;
+            if (t <= p.negatives) onTarget(t, tgt[b], v[b], f[b]);
+        }
+    }
+}
+
+// ---- Hogwild mode: one pass, updates land as they are computed ---------------------------
+template <int VPL, int TB>
+__global__ void __launch_bounds__(kBlock)
+sgns_hogwild_kernel(StepParams p)
+{
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    const uint32_t nk = (uint32_t)p.st->n_kept;
+    float4 *U4 = reinterpret_cast<float4 *>(p.U);
+    float4 *V4 = reinterpret_cast<float4 *>(p.V);
+    uint32_t draws = 0, redraws = 0;
+    for (uint32_t q = warp; q < nk; q += nwarps) {
+        const uint32_t w = p.win[q];
+        const uint32_t left = w & 0xFFu, right = w >> 8;
+        if (left + right == 0) continue;
+        const uint32_t c = (uint32_t)p.ctok[q];
+        const uint32_t i = p.cidx[q];
+        Row<VPL> u, etot;
+        row_load(u, U4 + (size_t)c * p.d4, p.d4, lane);
+        row_zero(etot);
+        for (uint32_t pp = q - left; pp <= q + right; ++pp) {
+            if (pp == q) continue;
+            const uint32_t w_out = (uint32_t)p.ctok[pp];
+            uint32_t n0, n1;
+            draw_pair_negatives(p, i, pp + p.window - q, w_out, lane, n0, n1, draws, redraws);
+            Row<VPL> e;
+            row_zero(e);
+            for_each_target<VPL, TB>(p, u, w_out, n0, n1, lane,
+                [&](uint32_t t, uint32_t tgt, const Row<VPL> &v, float f) {
+                    const float g = p.lr * ((t == 0 ? 1.0f : 0.0f) - sigmoidf_exact(f));
+                    row_axpy(e, g, v);                                         // e += g v(t)
+                    row_red_scaled(V4 + (size_t)tgt * p.d4, g, u, p.d4, lane);  // v(t) += g u(c)
+                });
+            row_add(u, e);       // later pairs of this centre see the moved vector
+            row_add(etot, e);
+        }
+        row_red_scaled(U4 + (size_t)c * p.d4, 1.0f, etot, p.d4, lane);          // u(c) += sum e
+    }
+    flush_draw_counts(p.st, draws, redraws);
+}
+
+// ---- snapshot mode, pass 1 (Algorithm 1 + the client's aggregation): dots and coefficients ----
+// Reads only start-of-step tables.  Writes G for every target and the per-centre sum
+// DU[q] = sum G v(target) (the scratch area of Algorithm 2 for the centre's own row).
+template <int VPL, int TB>
+__global__ void __launch_bounds__(kBlock)
+sgns_snap_dots_kernel(StepParams p)
+{
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    const uint32_t nk = (uint32_t)p.st->n_kept;
+    const float4 *U4 = reinterpret_cast<const float4 *>(p.U);
+    float4 *DU4 = reinterpret_cast<float4 *>(p.DU);
+    const uint32_t n1p = p.negatives + 1u;
+    uint32_t draws = 0, redraws = 0;
+    for (uint32_t q = warp; q < nk; q += nwarps) {
+        const uint32_t w = p.win[q];
+        const uint32_t left = w & 0xFFu, right = w >> 8;
+        if (left + right == 0) continue;
+        const uint32_t c = (uint32_t)p.ctok[q];
+        const uint32_t i = p.cidx[q];
+        Row<VPL> u, du;
+        row_load(u, U4 + (size_t)c * p.d4, p.d4, lane);
+        row_zero(du);
+        unsigned long long gi = p.pair_off[q] * n1p;
+        for (uint32_t pp = q - left; pp <= q + right; ++pp) {
+            if (pp == q) continue;
+            const uint32_t w_out = (uint32_t)p.ctok[pp];
+            uint32_t n0, n1;
+            draw_pair_negatives(p, i, pp + p.window - q, w_out, lane, n0, n1, draws, redraws);
+            for_each_target<VPL, TB>(p, u, w_out, n0, n1, lane,
+                [&](uint32_t t, uint32_t, const Row<VPL> &v, float f) {
+                    const float s = sigmoidf_exact(f);
+                    const float g = t == 0 ? p.lr * (1.0f - s) : -p.lr * s;
+                    if (lane == 0) p.G[gi + t] = g;
+                    row_axpy(du, g, v);
+                });
+            gi += n1p;
+        }
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+            const uint32_t idx = lane + 32u * v;
+            if (idx < p.d4) DU4[(size_t)q * p.d4 + idx] = du.x[v];
+        }
+    }
+    flush_draw_counts(p.st, draws, redraws);
+}
+
+// ---- snapshot mode, pass 2 (Algorithm 2, output rows): v(target) += G u(c) ------------------
+// U is still untouched, so u(c) is the start-of-step vector; V is only added to, never read.
+template <int VPL>
+__global__ void __launch_bounds__(kBlock)
+sgns_snap_adjust_v_kernel(StepParams p)
+{
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    const uint32_t nk = (uint32_t)p.st->n_kept;
+    const float4 *U4 = reinterpret_cast<const float4 *>(p.U);
+    float4 *V4 = reinterpret_cast<float4 *>(p.V);
+    const uint32_t n1p = p.negatives + 1u;
+    const bool wide = p.negatives > 32u;
+    uint32_t draws = 0, redraws = 0;   // regenerated draws are not counted twice
+    for (uint32_t q = warp; q < nk; q += nwarps) {
+        const uint32_t w = p.win[q];
+        const uint32_t left = w & 0xFFu, right = w >> 8;
+        if (left + right == 0) continue;
+        const uint32_t c = (uint32_t)p.ctok[q];
+        const uint32_t i = p.cidx[q];
+        Row<VPL> u;
+        row_load(u, U4 + (size_t)c * p.d4, p.d4, lane);
+        unsigned long long gi = p.pair_off[q] * n1p;
+        for (uint32_t pp = q - left; pp <= q + right; ++pp) {
+            if (pp == q) continue;
+            const uint32_t w_out = (uint32_t)p.ctok[pp];
+            uint32_t n0, n1;
+            draw_pair_negatives(p, i, pp + p.window - q, w_out, lane, n0, n1, draws, redraws);
+            for (uint32_t t = 0; t <= p.negatives; ++t) {
+                const uint32_t tgt = pair_target(t, w_out, n0, n1, wide);
+                const float g = __ldcg(p.G + gi + t);
+                row_red_scaled(V4 + (size_t)tgt * p.d4, g, u, p.d4, lane);
+            }
+            gi += n1p;
+        }
+    }
+}
+
+// ---- snapshot mode, pass 3 (Algorithm 2, input rows): u(c) += DU[q] -------------------------
+__global__ void __launch_bounds__(kBlock)
+sgns_snap_apply_u_kernel(StepParams p)
+{
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    const uint32_t nk = (uint32_t)p.st->n_kept;
+    float4 *U4 = reinterpret_cast<float4 *>(p.U);
+    const float4 *DU4 = reinterpret_cast<const float4 *>(p.DU);
+    for (uint32_t q = warp; q < nk; q += nwarps) {
+        if (p.win[q] == 0) continue;
+        const uint32_t c = (uint32_t)p.ctok[q];
+        for (uint32_t idx = lane; idx < p.d4; idx += 32) {
+            const float4 x = __ldcg(DU4 + (size_t)q * p.d4 + idx);
+            red_add_f32x4(U4 + (size_t)c * p.d4 + idx, x.x, x.y, x.z, x.w);
+        }
+    }
+}
+
+// ---- launch shapes --------------------------------------------------------------------------
+template <typename K>
+static int grid_for(K kernel, uint32_t blocks_per_sm, int sms)
+{
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kBlock, 0) != cudaSuccess || occ < 1)
+        occ = 1;
+    if (blocks_per_sm && (int)blocks_per_sm < occ) occ = (int)blocks_per_sm;
+    return occ * sms;   // whole waves: a multiple of the SM count
+}
+
+// Only shapes whose gathered rows fit the register file are instantiated
+// (VPL * TB float4 per lane).
+constexpr int kMaxRowRegs = 16;
+
+template <int VPL, int TB>
+struct Shape {
+    static void hogwild(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s)
+    {
+        if constexpr (VPL * TB <= kMaxRowRegs) {
+            const int grid = grid_for(sgns_hogwild_kernel<VPL, TB>, blocks_per_sm, sms);
+            sgns_hogwild_kernel<VPL, TB><<<grid, kBlock, 0, s>>>(p);
+        }
+    }
+    static void snap_dots(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s)
+    {
+        if constexpr (VPL * TB <= kMaxRowRegs) {
+            const int grid = grid_for(sgns_snap_dots_kernel<VPL, TB>, blocks_per_sm, sms);
+            sgns_snap_dots_kernel<VPL, TB><<<grid, kBlock, 0, s>>>(p);
+        }
+    }
+};
+
+template <int VPL>
+static void snap_adjust_v(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s)
+{
+    const int grid = grid_for(sgns_snap_adjust_v_kernel<VPL>, blocks_per_sm, sms);
+    sgns_snap_adjust_v_kernel<VPL><<<grid, kBlock, 0, s>>>(p);
+}
+
+#define W2V_FOR_TB(VPL, CALL)                                        \
+    switch (tb) {                                                    \
+        case 1: Shape<VPL, 1>::CALL; break;                          \
+        case 2: Shape<VPL, 2>::CALL; break;                          \
+        case 3: Shape<VPL, 3>::CALL; break;                          \
+        case 4: Shape<VPL, 4>::CALL; break;                          \
+        case 6: Shape<VPL, 6>::CALL; break;                          \
+        default: Shape<VPL, 8>::CALL; break;                         \
+    }
+
+#define W2V_FOR_VPL(CALL)                                            \
+    switch (vpl) {                                                   \
+        case 1: W2V_FOR_TB(1, CALL) break;                           \
+        case 2: W2V_FOR_TB(2, CALL) break;                           \
+        case 3: W2V_FOR_TB(3, CALL) break;                           \
+        case 4: W2V_FOR_TB(4, CALL) break;                           \
+        case 5: W2V_FOR_TB(5, CALL) break;                           \
+        case 6: W2V_FOR_TB(6, CALL) break;                           \
+        case 7: W2V_FOR_TB(7, CALL) break;                           \
+        default: W2V_FOR_TB(8, CALL) break;                          \
+    }
+
+// rows in flight per warp: the requested value rounded down to an instantiated shape
+static int pick_tb(uint32_t req, int vpl, uint32_t negatives)
+{
+    int tb = req ? (int)req : (vpl <= 2 ? 6 : (vpl <= 4 ? 4 : 2));
+    if (tb > (int)negatives + 1) tb = (int)negatives + 1;
+    if (tb > 8) tb = 8;
+    while (tb > 1 && tb * vpl > kMaxRowRegs) --tb;
+    if (tb == 5) tb = 4;
+    if (tb == 7) tb = 6;
+    return tb;
+}
+
+int launch_hogwild(const StepParams &p, uint32_t rows_in_flight, uint32_t blocks_per_sm, int sms,
+                   cudaStream_t s)
+{
+    const int vpl = (int)((p.d4 + 31) / 32);
+    const int tb = pick_tb(rows_in_flight, vpl, p.negatives);
+    W2V_FOR_VPL(hogwild(p, blocks_per_sm, sms, s))
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    return 1;
+}
+
+int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t blocks_per_sm, int sms,
+                    cudaStream_t s)
+{
+    const int vpl = (int)((p.d4 + 31) / 32);
+    const int tb = pick_tb(rows_in_flight, vpl, p.negatives);
+    W2V_FOR_VPL(snap_dots(p, blocks_per_sm, sms, s))
+    switch (vpl) {
+        case 1: snap_adjust_v<1>(p, blocks_per_sm, sms, s); break;
+        case 2: snap_adjust_v<2>(p, blocks_per_sm, sms, s); break;
+        case 3: snap_adjust_v<3>(p, blocks_per_sm, sms, s); break;
+        case 4: snap_adjust_v<4>(p, blocks_per_sm, sms, s); break;
+        case 5: snap_adjust_v<5>(p, blocks_per_sm, sms, s); break;
+        case 6: snap_adjust_v<6>(p, blocks_per_sm, sms, s); break;
+        case 7: snap_adjust_v<7>(p, blocks_per_sm, sms, s); break;
+        default: snap_adjust_v<8>(p, blocks_per_sm, sms, s); break;
+    }
+    {
+        const int grid = grid_for(sgns_snap_apply_u_kernel, blocks_per_sm, sms);
+        sgns_snap_apply_u_kernel<<<grid, kBlock, 0, s>>>(p);
+    }
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    return 3;
+}
+
+}  // namespace w2v
