@@ -1,0 +1,334 @@
+#!/usr/bin/env python
+"""Benchmark of the SGNS minibatch step (positive word-context pairs per second).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload large|sponsored|medium|small|tiny]
+    python bench.py --impl reference ...      # the CPU checker timed on the host cores
+
+One step = the whole hot path (sub-sampling, compaction, windows, negatives, gather, dots,
+coefficients, scatter-add) over one chunk of a seeded synthetic Zipfian token stream, in
+Hogwild mode.  Prints ONE JSON line.  With N > 1 (under torchrun) every rank trains its own
+replica on its own chunks: there is no data-path collective, only the timing reduction.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1606_08495_b200 import corpus  # noqa: E402
+
+METRIC = "sgns_positive_pairs_per_sec"
+UNIT = "pairs/s"
+FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes moved per algorithmic byte by the Hogwild update kernel, from the ncu capture
+# summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over the model bytes of
+# the captured launch).  None until a capture exists.
+TRAFFIC_PER_ALGORITHMIC_BYTE = None
+
+
+def algorithmic_bytes(d, centres, pairs, negatives):
+    """Rows touched by a Hogwild step, 4d bytes each, read once and written once:
+    the centre rows plus one output row per target (no credit for cache hits)."""
+    return 4 * d * (2 * centres + 2 * pairs * (1 + negatives))
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def physical_gpu_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        parts = [p for p in vis.split(",") if p]
+        if local_rank < len(parts) and parts[local_rank].isdigit():
+            return int(parts[local_rank])
+    return local_rank
+
+
+def pick_workload(name, free_bytes):
+    """The named configuration, else the largest one whose tables fit the GPU."""
+    order = ["large", "sponsored", "medium", "small", "tiny"]
+    if name:
+        return name
+    for cand in order:
+        c = corpus.CONFIGS[cand]
+        need = 2 * c["vocab"] * c["d"] * 4 + 12 * c["vocab"] + 3 * (1 << 30)
+        if need < free_bytes:
+            return cand
+    return "tiny"
+
+
+# --------------------------------------------------------------------------------------------
+# the CPU checker timed on the host (cpu_baseline leg and --impl reference)
+# --------------------------------------------------------------------------------------------
+def time_oracle(cfg, cp, sample_words, steps, warmup, first_chunk=500_000):
+    from oracle import Oracle
+
+    dense_bytes = 2 * cfg["vocab"] * cfg["d"] * 4
+    sparse = dense_bytes > 8 * (1 << 30)
+    o = Oracle(cfg["vocab"], cfg["d"], 1, sparse=sparse)
+    o.build_tables(cp.counts, cfg["subsample_t"])
+    W, N, lr = cfg["window"], cfg["negatives"], cfg["lr"]
+    for i in range(warmup):
+        o.step(cp.chunk(first_chunk + i, sample_words), W, N, lr, 1)
+    pairs, secs = 0, 0.0
+    for i in range(steps):
+        toks = cp.chunk(first_chunk + warmup + i, sample_words)
+        t0 = time.perf_counter()
+        st = o.step(toks, W, N, lr, 1)
+        secs += time.perf_counter() - t0
+        pairs += st["pairs"]
+    o.close()
+    store = "sparse lazily initialised row store" if sparse else "dense tables"
+    return pairs, secs, store
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    name = args.workload or "large"
+    cfg = corpus.CONFIGS[name]
+    cp = corpus.Corpus(cfg)
+    words = args.ref_words
+    pairs, secs, store = time_oracle(cfg, cp, words, args.steps, args.warmup)
+    value = pairs / secs if secs > 0 else 0.0
+    sample = f"{args.steps} steps of a {words}-word prefix of a chunk of the {name} workload, sequential mode, {store}"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / max(1, args.steps),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": name, "vocab": cfg["vocab"], "d": cfg["d"], "window": cfg["window"],
+                   "negatives": cfg["negatives"], "tokens_per_step": words},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------
+# the CUDA library
+# --------------------------------------------------------------------------------------------
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_1606_08495_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    name = pick_workload(args.workload, free_b)
+    cfg = corpus.CONFIGS[name]
+    cp = corpus.Corpus(cfg)
+    W, N, lr, d = cfg["window"], cfg["negatives"], cfg["lr"], cfg["d"]
+    K, Wu = args.steps, args.warmup
+
+    model = binding.W2V(cfg["vocab"], d, seed=1, device=dev)
+    model.build_alias(cp.counts, cfg["subsample_t"])
+    model.set_tuning(args.rows_in_flight, args.blocks_per_sm)
+
+    # every rank reads its own part of the stream: chunk index = rank * stride + i
+    stride = 10_000
+    n_chunks = Wu + 2 * K
+    host_chunks = [torch.from_numpy(cp.chunk(rank * stride + i)).pin_memory() for i in range(n_chunks)]
+    dev_chunks = [c.to(dev) for c in host_chunks[: Wu + K]]
+    torch.cuda.synchronize(dev)
+
+    # exact counts of the timed steps (same seed and step number as the steps themselves)
+    centres, pairs = [], []
+    for i in range(Wu, Wu + K):
+        model.set_step(i)
+        t = dev_chunks[i]
+        st = binding.StepStats()
+        binding.w2v_sample_pairs(model.h, t, t.numel(), W, N, None, None, None, 0, st,
+                                 allow=(binding.W2V_ERR_CAPACITY,))
+        centres.append(st.centres); pairs.append(st.pairs)
+    model.set_step(0)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    # ---- device-timed run: inputs already resident in HBM ----
+    for i in range(Wu):
+        binding.w2v_sgns_step(model.h, dev_chunks[i], dev_chunks[i].numel(), W, N, lr, binding.MODE_HOGWILD, None)
+    model.sync()
+    binding.w2v_profile_enable(model.h, True)
+    launches0 = model.launch_count()
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(); torch.cuda.synchronize(dev)
+    sampler.start()
+    ev0.record()
+    for i in range(Wu, Wu + K):
+        binding.w2v_sgns_step(model.h, dev_chunks[i], dev_chunks[i].numel(), W, N, lr, binding.MODE_HOGWILD, None)
+    ev1.record()
+    torch.cuda.synchronize(dev); barrier()
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1)
+    launches = model.launch_count() - launches0
+    kernel_ms, kernel_launches = binding.w2v_profile_read(model.h)
+    binding.w2v_profile_enable(model.h, False)
+
+    # ---- end-to-end run: host chunks in pinned memory, counters read back every step ----
+    e2e_pairs = 0
+    h2d = d2h = 0
+    st = binding.StepStats()
+    barrier(); torch.cuda.synchronize(dev)
+    ev2, ev3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev2.record()
+    for i in range(Wu + K, Wu + 2 * K):
+        t = host_chunks[i]
+        binding.w2v_sgns_step_host(model.h, t, t.numel(), W, N, lr, binding.MODE_HOGWILD, st)
+        e2e_pairs += st.pairs
+        h2d += 4 * t.numel(); d2h += 64
+    ev3.record()
+    torch.cuda.synchronize(dev); barrier()
+    e2e_ms = ev2.elapsed_time(ev3)
+
+    tot_pairs = float(sum(pairs))
+    tot_bytes = float(sum(algorithmic_bytes(d, c, p, N) for c, p in zip(centres, pairs)))
+    vals = torch.tensor([ms, e2e_ms, tot_pairs, float(e2e_pairs), float(launches)], dtype=torch.float64, device=dev)
+    if world > 1:
+        mx = vals.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+        sm = vals.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+        ms, e2e_ms = float(mx[0]), float(mx[1])
+        all_pairs, all_e2e_pairs, all_launches = float(sm[2]), float(sm[3]), int(sm[4])
+    else:
+        all_pairs, all_e2e_pairs, all_launches = tot_pairs, float(e2e_pairs), launches
+
+    if rank == 0:
+        peak, peak_kind = measured_peak()
+        achieved = tot_bytes / (kernel_ms * 1e-3) / 1e9 if kernel_ms > 0 else 0.0
+        per_launch_bytes = tot_bytes / max(1, kernel_launches)
+        line = {
+            "metric": METRIC, "value": all_pairs / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": Wu, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": name, "vocab": cfg["vocab"], "d": d, "window": W, "negatives": N,
+                       "subsample_t": cfg["subsample_t"], "tokens_per_step": int(dev_chunks[0].numel()),
+                       "mode": "hogwild", "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
+                       "l2": "tables and gathers far larger than L2 (random rows of %.1f GB)" % (2 * cfg["vocab"] * d * 4 / 1e9)
+                             if 2 * cfg["vocab"] * d * 4 > 4 * 126e6 else "tables fit in L2; no flush between steps",
+                       "pairs_per_step": tot_pairs / K, "centres_per_step": sum(centres) / K,
+                       "trained_pairs_incl_negatives_per_sec": all_pairs * (1 + N) / (ms * 1e-3),
+                       "centres_per_sec": world * sum(centres) / (ms * 1e-3)},
+            "clocks": clocks,
+            "e2e": {"value": all_e2e_pairs / (e2e_ms * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": h2d // K, "d2h_bytes_per_step": d2h // K},
+            "gpu_launches": all_launches,
+            "roofline": {"bound": "hbm", "kernel": "sgns_hogwild_kernel", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                         "frac_of_8TBps": achieved / 8000.0,
+                         "algorithmic_bytes_per_launch": per_launch_bytes,
+                         "kernel_ms_per_launch": kernel_ms / max(1, kernel_launches),
+                         "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE * per_launch_bytes
+                                     if TRAFFIC_PER_ALGORITHMIC_BYTE is not None else None)},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            words = args.cpu_words
+            p, s, store = time_oracle(cfg, cp, words, 1, 0)
+            line["cpu_baseline"] = {
+                "value": p / s if s > 0 else 0.0, "unit": UNIT, "cores": 1, "kind": "oracle",
+                "sample": f"one step over a {words}-word prefix of a chunk of the {name} workload "
+                          f"({p} pairs, {s:.1f} s), sequential mode, {store}"}
+        print(json.dumps(line), flush=True)
+    model.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=list(corpus.CONFIGS), default=None)
+    ap.add_argument("--rows-in-flight", type=int, default=0)
+    ap.add_argument("--blocks-per-sm", type=int, default=0)
+    ap.add_argument("--cpu-words", type=int, default=150_000, help="word tokens in the cpu_baseline sample")
+    ap.add_argument("--ref-words", type=int, default=20_000, help="word tokens per step of --impl reference")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        print("note: fewer than 3 warm-up steps; not a valid timing", file=sys.stderr)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()
