@@ -210,6 +210,32 @@ int32_t w2v_get_launch_count(w2v_handle *h, uint64_t *launches);
  */
 int32_t w2v_set_tuning(w2v_handle *h, uint32_t rows_in_flight, uint32_t blocks_per_sm);
 
+/*
+ * w2v_sample_pairs for callers that must not allocate device memory.  (The paper has no
+ * counterpart to this call; it exists for the sake of the library's users.)
+ *
+ * Who needs it: code that runs when the rest of the GPU's memory already belongs to someone
+ * else (a training framework's caching allocator, a serving engine's KV cache), code on a
+ * latency-critical path where the implicit synchronisation of an allocation is unwelcome, and
+ * hosts whose policy is "no allocation after start-up".  w2v_sample_pairs grows scratch inside
+ * the handle on first use; this variant never calls cudaMalloc, cudaFree or any other
+ * allocating routine.  Its scratch is one fixed array of just under 2 MiB inside the library
+ * image, present on every GPU that loads the library until the process exits.
+ *
+ * Same arguments, same results and the same return codes as w2v_sample_pairs, except:
+ *   - n may be at most 65536 tokens; a larger chunk is refused with W2V_ERR_CAPACITY
+ *     ("serves at most 65536 tokens per call") before anything is launched.
+ *   - The first call on each GPU looks up the device address of the fixed array.  Make that
+ *     first call during set-up, before any CUDA stream capture begins.
+ *   - All handles and all calls on one GPU share the one array, and it keeps whatever the
+ *     previous call left in it (this call clears the counters it needs at zero).  Two calls
+ *     that overlap on the GPU -- from different streams or threads -- race on it; issue
+ *     them one after the other.  The call returns only after its own work has finished.
+ */
+int32_t w2v_sample_pairs_noalloc(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window,
+                                 uint32_t negatives, int32_t *centre, int32_t *context, int32_t *negs,
+                                 uint64_t cap, uint64_t *n_pairs, w2v_step_stats *stats);
+
 /* Text of the last error on this handle (never NULL; h == NULL gives a generic text). */
 const char *w2v_last_error(w2v_handle *h);
 

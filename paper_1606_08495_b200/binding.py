@@ -24,6 +24,7 @@ EXPORTS = (
     "w2v_sgns_step_host", "w2v_sample_pairs", "w2v_partial_dots", "w2v_read_rows", "w2v_write_rows",
     "w2v_set_step", "w2v_get_step", "w2v_get_table_ptrs", "w2v_sync", "w2v_profile_enable",
     "w2v_profile_read", "w2v_get_launch_count", "w2v_set_tuning", "w2v_last_error",
+    "w2v_sample_pairs_noalloc",
 )
 
 
@@ -69,6 +70,7 @@ def load():
         "w2v_sgns_step": [vp, vp, u64, u32, u32, C.c_float, u32, C.POINTER(StepStats)],
         "w2v_sgns_step_host": [vp, vp, u64, u32, u32, C.c_float, u32, C.POINTER(StepStats)],
         "w2v_sample_pairs": [vp, vp, u64, u32, u32, vp, vp, vp, u64, C.POINTER(u64), C.POINTER(StepStats)],
+        "w2v_sample_pairs_noalloc": [vp, vp, u64, u32, u32, vp, vp, vp, u64, C.POINTER(u64), C.POINTER(StepStats)],
         "w2v_partial_dots": [vp, vp, u64, u32, u32, vp],
         "w2v_read_rows": [vp, u32, vp, u64, vp],
         "w2v_write_rows": [vp, u32, vp, u64, vp],
@@ -150,6 +152,15 @@ def w2v_sample_pairs(h, tokens, n, window, negatives, centre, context, negs, cap
     ref = C.byref(stats) if stats is not None else None
     rc = _check(h, load().w2v_sample_pairs(h, _ptr(tokens), int(n), window, negatives, _ptr(centre), _ptr(context),
                                            _ptr(negs), int(cap), C.byref(npairs), ref), allow)
+    return rc, int(npairs.value)
+
+
+def w2v_sample_pairs_noalloc(h, tokens, n, window, negatives, centre, context, negs, cap, stats=None, allow=()):
+    """w2v_sample_pairs on the library's fixed scratch: no device allocation, at most 65536 tokens."""
+    npairs = C.c_uint64(0)
+    ref = C.byref(stats) if stats is not None else None
+    rc = _check(h, load().w2v_sample_pairs_noalloc(h, _ptr(tokens), int(n), window, negatives, _ptr(centre),
+                                                   _ptr(context), _ptr(negs), int(cap), C.byref(npairs), ref), allow)
     return rc, int(npairs.value)
 
 

@@ -519,3 +519,124 @@ const char *w2v_last_error(w2v_handle *h)
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// Pair sampling for callers that must not allocate.
+//
+// Some callers of this library cannot call cudaMalloc at the moment they need the pair list:
+// code that runs while another component owns all remaining device memory, latency-critical
+// loops where an allocation (an implicit device synchronisation) is not acceptable, and hosts
+// whose memory policy forbids allocation after start-up.  w2v_sample_pairs grows handle-owned
+// scratch on demand; the entry point below instead keeps all of its scratch in one fixed array
+// that is part of the library image.  Every GPU that loads the library holds that array until
+// the process exits, which is why its size is modest and the chunk size is capped.
+// ------------------------------------------------------------------------------------------
+namespace {
+
+constexpr uint64_t kNoAllocMaxTokens = 65536;                 // largest chunk the fixed scratch serves
+constexpr size_t kNoAllocAlign = 256;
+constexpr size_t na_round(size_t b) { return (b + kNoAllocAlign - 1) / kNoAllocAlign * kNoAllocAlign; }
+constexpr size_t kNaTiles = kNoAllocMaxTokens / kScanTile + 2;
+// layout of the fixed scratch, every part 256-byte aligned
+constexpr size_t kNaState = 0;
+constexpr size_t kNaFlags = kNaState + na_round(sizeof(DevState));
+constexpr size_t kNaTileSums = kNaFlags + na_round(kNoAllocMaxTokens * sizeof(uint8_t));
+constexpr size_t kNaTileOffs = kNaTileSums + na_round(kNaTiles * sizeof(uint2));
+constexpr size_t kNaCtok = kNaTileOffs + na_round(kNaTiles * sizeof(uint2));
+constexpr size_t kNaCidx = kNaCtok + na_round(kNoAllocMaxTokens * sizeof(int32_t));
+constexpr size_t kNaCsent = kNaCidx + na_round(kNoAllocMaxTokens * sizeof(uint32_t));
+constexpr size_t kNaWin = kNaCsent + na_round(kNoAllocMaxTokens * sizeof(uint32_t));
+constexpr size_t kNaCntTile = kNaWin + na_round(kNoAllocMaxTokens * sizeof(uint16_t));
+constexpr size_t kNaPairOff = kNaCntTile + na_round(kNaTiles * sizeof(unsigned long long));
+constexpr size_t kNoAllocBytes = kNaPairOff + na_round((kNoAllocMaxTokens + 1) * sizeof(unsigned long long));
+static_assert(kNoAllocBytes <= (2u << 20), "fixed scratch is meant to stay within 2 MiB");
+
+// The scratch itself.  In host code this name is only a stand-in for the symbol: the address a
+// kernel may use comes from cudaGetSymbolAddress, once per device (below).
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+constexpr int kNaMaxDevices = 64;
+unsigned char *g_noalloc_addr[kNaMaxDevices] = {};            // device address per GPU, 0 = not set up
+
+// Looks up, once per device, the device address of the fixed scratch.  `device` must be current.
+int32_t noalloc_scratch_address(w2v_handle *h, int device, unsigned char **out)
+{
+    if (device < 0 || device >= kNaMaxDevices) return fail(h, W2V_ERR_ARG, "device ordinal beyond the supported range");
+    if (!g_noalloc_addr[device]) {
+        void *p = nullptr;
+        cudaError_t ce = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (ce != cudaSuccess || !p) return fail(h, W2V_ERR_CUDA, "cudaGetSymbolAddress(fixed scratch)", ce);
+        g_noalloc_addr[device] = static_cast<unsigned char *>(p);
+    }
+    *out = g_noalloc_addr[device];
+    return W2V_OK;
+}
+
+}  // namespace
+
+extern "C" int32_t w2v_sample_pairs_noalloc(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window,
+                                            uint32_t negatives, int32_t *centre, int32_t *context, int32_t *negs,
+                                            uint64_t cap, uint64_t *n_pairs, w2v_step_stats *stats)
+{
+    int32_t rc = check_step_args(h, tokens, n, window, negatives);
+    if (rc != W2V_OK) return rc;
+    if (!n_pairs) return fail(h, W2V_ERR_ARG, "n_pairs is NULL");
+    if (cap && (!centre || !context || !negs)) return fail(h, W2V_ERR_ARG, "output array is NULL");
+    if (n > kNoAllocMaxTokens)
+        return fail(h, W2V_ERR_CAPACITY, "w2v_sample_pairs_noalloc serves at most 65536 tokens per call");
+    DeviceGuard g(h->device);
+    unsigned char *base = nullptr;
+    if ((rc = noalloc_scratch_address(h, h->device, &base)) != W2V_OK) return rc;
+
+    // the same kernels as w2v_sample_pairs, pointed at the fixed scratch instead of handle scratch
+    Scratch sc;
+    sc.n_cap = kNoAllocMaxTokens;
+    sc.flags = reinterpret_cast<uint8_t *>(base + kNaFlags);
+    sc.tile_sums = reinterpret_cast<uint2 *>(base + kNaTileSums);
+    sc.tile_offs = reinterpret_cast<uint2 *>(base + kNaTileOffs);
+    sc.ctok = reinterpret_cast<int32_t *>(base + kNaCtok);
+    sc.cidx = reinterpret_cast<uint32_t *>(base + kNaCidx);
+    sc.csent = reinterpret_cast<uint32_t *>(base + kNaCsent);
+    sc.win = reinterpret_cast<uint16_t *>(base + kNaWin);
+    sc.cnt_tile = reinterpret_cast<unsigned long long *>(base + kNaCntTile);
+    sc.pair_off = reinterpret_cast<unsigned long long *>(base + kNaPairOff);
+    DevState *st = reinterpret_cast<DevState *>(base + kNaState);
+
+    // the array keeps the previous call's contents: the counters must start at zero; everything
+    // else is written before it is read
+    W2V_CUDA(h, cudaMemsetAsync(st, 0, sizeof(DevState), h->stream));
+    const uint32_t k0 = (uint32_t)h->seed;
+    const uint32_t k1 = (uint32_t)(h->seed >> 32) ^ (uint32_t)(h->step_id >> 32);
+    const uint32_t step_lo = (uint32_t)h->step_id;
+    SampleTables tab{h->keep_thr, h->alias};
+    int k = launch_compact(tokens, n, tab, (uint32_t)h->vocab, k0, k1, step_lo, sc, st, h->stream);
+    if (k < 0) return fail(h, W2V_ERR_CUDA, "compaction launch", cudaGetLastError());
+    h->launches += (uint64_t)k;
+    k = launch_windows(n, window, k0, k1, step_lo, sc, st, h->stream);
+    if (k < 0) return fail(h, W2V_ERR_CUDA, "window launch", cudaGetLastError());
+    h->launches += (uint64_t)k;
+    k = launch_pair_offsets(n, sc, st, h->stream);
+    if (k < 0) return fail(h, W2V_ERR_CUDA, "pair offset launch", cudaGetLastError());
+    h->launches += (uint64_t)k;
+    if (n) {
+        StepParams p = make_params(h, window, negatives, 0.f);
+        p.ctok = sc.ctok; p.cidx = sc.cidx; p.win = sc.win; p.pair_off = sc.pair_off; p.st = st;
+        p.G = nullptr; p.DU = nullptr;
+        k = launch_emit_pairs(p, centre, context, negs, cap, h->sms * 8, h->stream);
+        if (k < 0) return fail(h, W2V_ERR_CUDA, "pair list launch", cudaGetLastError());
+        h->launches += (uint64_t)k;
+    }
+    // counters come back through the handle's pinned mirror, which w2v_create allocated
+    W2V_CUDA(h, cudaMemcpyAsync(h->st_host, st, sizeof(DevState), cudaMemcpyDeviceToHost, h->stream));
+    W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+    const DevState &s = *h->st_host;
+    if (stats) {
+        stats->tokens = n; stats->kept = s.n_kept; stats->centres = s.centres; stats->pairs = s.pairs;
+        stats->neg_draws = s.neg_draws; stats->neg_redraws = s.neg_redraws; stats->oov = s.oov;
+        stats->status = s.status; stats->reserved = 0;
+    }
+    *n_pairs = s.pairs;
+    if (s.pairs > cap) return fail(h, W2V_ERR_CAPACITY, "more pairs than the output arrays hold");
+    if (s.status & 1u) return fail(h, W2V_ERR_TOKEN_RANGE, "token ids outside [-1, vocab) were skipped");
+    return W2V_OK;
+}
