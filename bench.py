@@ -30,16 +30,25 @@ from paper_1606_08495_b200 import corpus  # noqa: E402
 METRIC = "sgns_positive_pairs_per_sec"
 UNIT = "pairs/s"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes moved per algorithmic byte by the Hogwild update kernel, from the ncu capture
-# summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over the model bytes of
-# the captured launch).  None until a capture exists.
-TRAFFIC_PER_ALGORITHMIC_BYTE = None
+# DRAM bytes moved per algorithmic byte by the Hogwild update kernel on the large workload, from
+# the one-pass ncu capture summarised in profiles/sgns_update_kernels_large.md
+# ((dram__bytes_read.sum + dram__bytes_write.sum) / model bytes of the captured launch: 127.8 / 121.9 GB).
+# Applies to the large workload in Hogwild mode only; other workloads report null.
+TRAFFIC_PER_ALGORITHMIC_BYTE = 1.049
 
 
 def algorithmic_bytes(d, centres, pairs, negatives):
     """Rows touched by a Hogwild step, 4d bytes each, read once and written once:
     the centre rows plus one output row per target (no credit for cache hits)."""
     return 4 * d * (2 * centres + 2 * pairs * (1 + negatives))
+
+
+def algorithmic_bytes_snapshot(d, centres, pairs, negatives):
+    """Three-pass snapshot plan: pass 1 reads C + T rows, writes C scratch rows and T coefficients;
+    pass 2 reads C rows and T coefficients and read-modify-writes T rows; pass 3 reads C scratch rows
+    and read-modify-writes C rows (T = pairs * (1 + negatives))."""
+    T = pairs * (1 + negatives)
+    return 4 * d * (3 * T + 6 * centres) + 8 * T
 
 
 def measured_peak():
@@ -193,6 +202,7 @@ def run_gpu(args):
     cp = corpus.Corpus(cfg)
     W, N, lr, d = cfg["window"], cfg["negatives"], cfg["lr"], cfg["d"]
     K, Wu = args.steps, args.warmup
+    mode = binding.MODE_HOGWILD if args.mode == "hogwild" else binding.MODE_SNAPSHOT
 
     model = binding.W2V(cfg["vocab"], d, seed=1, device=dev)
     model.build_alias(cp.counts, cfg["subsample_t"])
@@ -222,7 +232,7 @@ def run_gpu(args):
 
     # ---- device-timed run: inputs already resident in HBM ----
     for i in range(Wu):
-        binding.w2v_sgns_step(model.h, dev_chunks[i], dev_chunks[i].numel(), W, N, lr, binding.MODE_HOGWILD, None)
+        binding.w2v_sgns_step(model.h, dev_chunks[i], dev_chunks[i].numel(), W, N, lr, mode, None)
     model.sync()
     binding.w2v_profile_enable(model.h, True)
     launches0 = model.launch_count()
@@ -232,7 +242,7 @@ def run_gpu(args):
     sampler.start()
     ev0.record()
     for i in range(Wu, Wu + K):
-        binding.w2v_sgns_step(model.h, dev_chunks[i], dev_chunks[i].numel(), W, N, lr, binding.MODE_HOGWILD, None)
+        binding.w2v_sgns_step(model.h, dev_chunks[i], dev_chunks[i].numel(), W, N, lr, mode, None)
     ev1.record()
     torch.cuda.synchronize(dev); barrier()
     clocks = sampler.stop()
@@ -250,7 +260,7 @@ def run_gpu(args):
     ev2.record()
     for i in range(Wu + K, Wu + 2 * K):
         t = host_chunks[i]
-        binding.w2v_sgns_step_host(model.h, t, t.numel(), W, N, lr, binding.MODE_HOGWILD, st)
+        binding.w2v_sgns_step_host(model.h, t, t.numel(), W, N, lr, mode, st)
         e2e_pairs += st.pairs
         h2d += 4 * t.numel(); d2h += 64
     ev3.record()
@@ -258,7 +268,8 @@ def run_gpu(args):
     e2e_ms = ev2.elapsed_time(ev3)
 
     tot_pairs = float(sum(pairs))
-    tot_bytes = float(sum(algorithmic_bytes(d, c, p, N) for c, p in zip(centres, pairs)))
+    model_bytes = algorithmic_bytes if args.mode == "hogwild" else algorithmic_bytes_snapshot
+    tot_bytes = float(sum(model_bytes(d, c, p, N) for c, p in zip(centres, pairs)))
     vals = torch.tensor([ms, e2e_ms, tot_pairs, float(e2e_pairs), float(launches)], dtype=torch.float64, device=dev)
     if world > 1:
         mx = vals.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
@@ -271,14 +282,15 @@ def run_gpu(args):
     if rank == 0:
         peak, peak_kind = measured_peak()
         achieved = tot_bytes / (kernel_ms * 1e-3) / 1e9 if kernel_ms > 0 else 0.0
-        per_launch_bytes = tot_bytes / max(1, kernel_launches)
+        groups = kernel_launches if args.mode == "hogwild" else kernel_launches // 3
+        per_launch_bytes = tot_bytes / max(1, groups)
         line = {
             "metric": METRIC, "value": all_pairs / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": Wu, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": name, "vocab": cfg["vocab"], "d": d, "window": W, "negatives": N,
                        "subsample_t": cfg["subsample_t"], "tokens_per_step": int(dev_chunks[0].numel()),
-                       "mode": "hogwild", "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
+                       "mode": args.mode, "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
                        "l2": "tables and gathers far larger than L2 (random rows of %.1f GB)" % (2 * cfg["vocab"] * d * 4 / 1e9)
                              if 2 * cfg["vocab"] * d * 4 > 4 * 126e6 else "tables fit in L2; no flush between steps",
                        "pairs_per_step": tot_pairs / K, "centres_per_step": sum(centres) / K,
@@ -288,13 +300,15 @@ def run_gpu(args):
             "e2e": {"value": all_e2e_pairs / (e2e_ms * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": h2d // K, "d2h_bytes_per_step": d2h // K},
             "gpu_launches": all_launches,
-            "roofline": {"bound": "hbm", "kernel": "sgns_hogwild_kernel", "achieved": achieved, "peak": peak,
+            "roofline": {"bound": "hbm",
+                         "kernel": "sgns_hogwild_kernel" if args.mode == "hogwild" else "sgns_snap_* (3 passes)",
+                         "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "frac_of_8TBps": achieved / 8000.0,
                          "algorithmic_bytes_per_launch": per_launch_bytes,
-                         "kernel_ms_per_launch": kernel_ms / max(1, kernel_launches),
+                         "kernel_ms_per_launch": kernel_ms / max(1, groups),
                          "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE * per_launch_bytes
-                                     if TRAFFIC_PER_ALGORITHMIC_BYTE is not None else None)},
+                                     if name == "large" and args.mode == "hogwild" else None)},
         }
         if world == 1 and not args.no_cpu_baseline:
             words = args.cpu_words
@@ -312,7 +326,7 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=list(corpus.CONFIGS), default=None)
@@ -321,6 +335,8 @@ def main():
     ap.add_argument("--cpu-words", type=int, default=150_000, help="word tokens in the cpu_baseline sample")
     ap.add_argument("--ref-words", type=int, default=20_000, help="word tokens per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mode", choices=["hogwild", "snapshot"], default="hogwild",
+                    help="update mode of the timed steps (the headline number is hogwild)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         print("note: fewer than 3 warm-up steps; not a valid timing", file=sys.stderr)
