@@ -114,14 +114,19 @@ def physical_gpu_index(local_rank):
     return local_rank
 
 
-def pick_workload(name, free_bytes):
+def row_stride_for(d, requested=0):
+    """Floats between table rows: the requested value, else rows padded to 128-byte boundaries."""
+    return requested if requested else (d + 31) // 32 * 32
+
+
+def pick_workload(name, free_bytes, requested_stride=0):
     """The named configuration, else the largest one whose tables fit the GPU."""
     order = ["large", "sponsored", "medium", "small", "tiny"]
     if name:
         return name
     for cand in order:
         c = corpus.CONFIGS[cand]
-        need = 2 * c["vocab"] * c["d"] * 4 + 12 * c["vocab"] + 3 * (1 << 30)
+        need = 2 * c["vocab"] * row_stride_for(c["d"], requested_stride) * 4 + 12 * c["vocab"] + 3 * (1 << 30)
         if need < free_bytes:
             return cand
     return "tiny"
@@ -197,14 +202,15 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=dev)
 
     free_b, _ = torch.cuda.mem_get_info(dev)
-    name = pick_workload(args.workload, free_b)
+    name = pick_workload(args.workload, free_b, args.row_stride)
     cfg = corpus.CONFIGS[name]
     cp = corpus.Corpus(cfg)
     W, N, lr, d = cfg["window"], cfg["negatives"], cfg["lr"], cfg["d"]
     K, Wu = args.steps, args.warmup
     mode = binding.MODE_HOGWILD if args.mode == "hogwild" else binding.MODE_SNAPSHOT
 
-    model = binding.W2V(cfg["vocab"], d, seed=1, device=dev)
+    row_stride = row_stride_for(d, args.row_stride)
+    model = binding.W2V(cfg["vocab"], d, seed=1, device=dev, row_stride=row_stride)
     model.build_alias(cp.counts, cfg["subsample_t"])
     model.set_tuning(args.rows_in_flight, args.blocks_per_sm)
 
@@ -282,7 +288,7 @@ def run_gpu(args):
     if rank == 0:
         peak, peak_kind = measured_peak()
         achieved = tot_bytes / (kernel_ms * 1e-3) / 1e9 if kernel_ms > 0 else 0.0
-        groups = kernel_launches if args.mode == "hogwild" else kernel_launches // 3
+        groups = K          # one group of update kernels per step (1 launch in hogwild mode, 3-4 in snapshot mode)
         per_launch_bytes = tot_bytes / max(1, groups)
         line = {
             "metric": METRIC, "value": all_pairs / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
@@ -290,7 +296,7 @@ def run_gpu(args):
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": name, "vocab": cfg["vocab"], "d": d, "window": W, "negatives": N,
                        "subsample_t": cfg["subsample_t"], "tokens_per_step": int(dev_chunks[0].numel()),
-                       "mode": args.mode, "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
+                       "mode": args.mode, "row_stride_floats": row_stride, "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
                        "l2": "tables and gathers far larger than L2 (random rows of %.1f GB)" % (2 * cfg["vocab"] * d * 4 / 1e9)
                              if 2 * cfg["vocab"] * d * 4 > 4 * 126e6 else "tables fit in L2; no flush between steps",
                        "pairs_per_step": tot_pairs / K, "centres_per_step": sum(centres) / K,
@@ -332,6 +338,9 @@ def main():
     ap.add_argument("--workload", choices=list(corpus.CONFIGS), default=None)
     ap.add_argument("--rows-in-flight", type=int, default=0)
     ap.add_argument("--blocks-per-sm", type=int, default=0)
+    ap.add_argument("--row-stride", type=int, default=0,
+                    help="floats between table rows (0 = d rounded up to a multiple of 32, i.e. rows on 128-byte "
+                         "boundaries; pass d itself for dense rows)")
     ap.add_argument("--cpu-words", type=int, default=150_000, help="word tokens in the cpu_baseline sample")
     ap.add_argument("--ref-words", type=int, default=20_000, help="word tokens per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -22,8 +22,9 @@
  *     return values to the host synchronise that stream; the others are
  *     asynchronous.
  *   - Tables are row-major fp32: row w of U (input vectors) or V (output
- *     vectors) is d consecutive floats at offset w*d.  Row index = rank of the
- *     word by decreasing frequency (Section 5.1, the ordering O).
+ *     vectors) is d consecutive floats at offset w*d (w*row_stride for a model
+ *     made by w2v_create_strided).  Row index = rank of the word by decreasing
+ *     frequency (Section 5.1, the ordering O).
  *   - Token streams are int32 word ids in [0, vocab); -1 ends a sentence;
  *     any other value is skipped as out of vocabulary and reported.  Windows
  *     are taken over the tokens that survive sub-sampling ("dirty" contexts,
@@ -85,6 +86,25 @@ typedef struct {
  */
 int32_t w2v_create(uint64_t vocab, uint32_t d, uint64_t seed, float *U, float *V,
                    void *stream, w2v_handle **out);
+
+/*
+ * w2v_create with padded rows: row w of U or V starts at float offset w*row_stride and its
+ * first d floats are the vector (the paper fixes only that a vector is an array of d single
+ * precision numbers, Section 1; where the rows sit in memory is this library's choice).
+ *   row_stride  floats between consecutive rows; a multiple of 4 with d <= row_stride <= 2048.
+ *               A stride whose byte size is a multiple of 64 (304 floats for d = 300) makes
+ *               every row start on a DRAM burst boundary, so a gathered row moves no
+ *               neighbouring bytes.  The padding floats are zeroed here and never read or
+ *               written afterwards.
+ *   U, V        device, caller-owned, vocab*row_stride floats each, 16-byte aligned (64-byte
+ *               aligned to get the benefit above); or both NULL (library-owned).
+ * Everything else as w2v_create, which is this call with row_stride = d.
+ */
+int32_t w2v_create_strided(uint64_t vocab, uint32_t d, uint32_t row_stride, uint64_t seed, float *U,
+                           float *V, void *stream, w2v_handle **out);
+
+/* Floats between consecutive rows of U and V. */
+int32_t w2v_get_row_stride(w2v_handle *h, uint32_t *row_stride);
 
 /* Waits for the handle's stream, frees what the handle owns.  NULL is accepted. */
 int32_t w2v_destroy(w2v_handle *h);

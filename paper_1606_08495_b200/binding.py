@@ -20,7 +20,7 @@ MODE_SNAPSHOT, MODE_HOGWILD = 0, 1
 TABLE_U, TABLE_V = 0, 1
 
 EXPORTS = (
-    "w2v_create", "w2v_destroy", "w2v_build_alias", "w2v_get_tables", "w2v_sgns_step",
+    "w2v_create", "w2v_create_strided", "w2v_get_row_stride", "w2v_destroy", "w2v_build_alias", "w2v_get_tables", "w2v_sgns_step",
     "w2v_sgns_step_host", "w2v_sample_pairs", "w2v_partial_dots", "w2v_read_rows", "w2v_write_rows",
     "w2v_set_step", "w2v_get_step", "w2v_get_table_ptrs", "w2v_sync", "w2v_profile_enable",
     "w2v_profile_read", "w2v_get_launch_count", "w2v_set_tuning", "w2v_last_error",
@@ -64,6 +64,8 @@ def load():
     vp, u32, u64, i32 = C.c_void_p, C.c_uint32, C.c_uint64, C.c_int32
     sig = {
         "w2v_create": [u64, u32, u64, vp, vp, vp, C.POINTER(vp)],
+        "w2v_create_strided": [u64, u32, u32, u64, vp, vp, vp, C.POINTER(vp)],
+        "w2v_get_row_stride": [vp, C.POINTER(u32)],
         "w2v_destroy": [vp],
         "w2v_build_alias": [vp, vp, C.c_double],
         "w2v_get_tables": [vp, vp, vp, vp],
@@ -118,6 +120,21 @@ def w2v_create(vocab, d, seed, U, V, stream):
     if rc != W2V_OK:
         raise W2VError(rc, "w2v_create rejected its arguments or could not allocate")
     return h
+
+
+def w2v_create_strided(vocab, d, row_stride, seed, U, V, stream):
+    h = C.c_void_p()
+    rc = load().w2v_create_strided(int(vocab), int(d), int(row_stride), int(seed), _ptr(U), _ptr(V), stream,
+                                   C.byref(h))
+    if rc != W2V_OK:
+        raise W2VError(rc, "w2v_create_strided rejected its arguments or could not allocate")
+    return h
+
+
+def w2v_get_row_stride(h):
+    s = C.c_uint32(0)
+    _check(h, load().w2v_get_row_stride(h, C.byref(s)))
+    return int(s.value)
 
 
 def w2v_destroy(h):
@@ -210,21 +227,30 @@ def w2v_set_tuning(h, rows_in_flight, blocks_per_sm):
     return _check(h, load().w2v_set_tuning(h, int(rows_in_flight), int(blocks_per_sm)))
 
 
+def aligned_row_stride(d):
+    """Smallest row stride (in floats) >= d that puts every row on a 128-byte boundary, the
+    granularity at which the GPU's L2 cache fetches and writes back: a gathered row then moves
+    no bytes of its neighbours."""
+    return (int(d) + 31) // 32 * 32
+
+
 # ---- convenience wrapper: owns the torch tensors the handle points at ----------------------
 class W2V:
     """Tables U and V as torch tensors on one GPU plus the library handle."""
 
-    def __init__(self, vocab, d, seed, device="cuda:0"):
+    def __init__(self, vocab, d, seed, device="cuda:0", row_stride=None):
         load()
         if not torch.cuda.is_available():
             raise RuntimeError("libw2v needs a CUDA device; there is no CPU path")
         self.device = torch.device(device)
         self.vocab, self.d, self.seed = int(vocab), int(d), int(seed)
+        self.row_stride = self.d if row_stride is None else int(row_stride)
         with torch.cuda.device(self.device):
-            self.U = torch.empty(self.vocab * self.d, dtype=torch.float32, device=self.device)
-            self.V = torch.empty(self.vocab * self.d, dtype=torch.float32, device=self.device)
+            self.U = torch.empty(self.vocab * self.row_stride, dtype=torch.float32, device=self.device)
+            self.V = torch.empty(self.vocab * self.row_stride, dtype=torch.float32, device=self.device)
             self.stream = torch.cuda.current_stream(self.device)
-            self.h = w2v_create(self.vocab, self.d, self.seed, self.U, self.V, self.stream.cuda_stream)
+            self.h = w2v_create_strided(self.vocab, self.d, self.row_stride, self.seed, self.U, self.V,
+                                        self.stream.cuda_stream)
 
     def close(self):
         if getattr(self, "h", None):

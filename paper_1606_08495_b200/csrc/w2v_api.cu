@@ -14,6 +14,7 @@ using namespace w2v;
 struct w2v_handle {
     uint64_t vocab = 0;
     uint32_t d = 0;
+    uint32_t ld = 0;                 // row stride of U and V in floats (>= d, a multiple of 4)
     uint64_t seed = 0;
     uint64_t step_id = 0;
     int device = 0;
@@ -33,6 +34,9 @@ struct w2v_handle {
     uint64_t G_cap = 0;
     float *DU = nullptr;
     uint64_t DU_cap = 0;             // floats
+    double *DV = nullptr;            // fp64 sums for the most-hit output rows (snapshot mode), kept zero between steps
+    uint64_t DV_cap = 0;             // doubles
+    uint32_t hot_rows = 0;
     int32_t *tok_stage = nullptr;
     uint64_t tok_stage_cap = 0;
     // tuning / accounting
@@ -125,13 +129,14 @@ StepParams make_params(w2v_handle *h, uint32_t window, uint32_t negatives, float
     p.tab.keep_thr = h->keep_thr; p.tab.alias = h->alias;
     p.ctok = h->sc.ctok; p.cidx = h->sc.cidx; p.win = h->sc.win;
     p.st = h->st;
-    p.vocab = (uint32_t)h->vocab; p.d4 = h->d / 4;
+    p.vocab = (uint32_t)h->vocab; p.d4 = h->d / 4; p.ld4 = h->ld / 4;
     p.window = window; p.negatives = negatives;
     p.k0 = (uint32_t)h->seed;
     p.k1 = (uint32_t)(h->seed >> 32) ^ (uint32_t)(h->step_id >> 32);
     p.step_lo = (uint32_t)h->step_id;
     p.lr = lr;
     p.pair_off = h->sc.pair_off; p.G = h->G; p.DU = h->DU;
+    p.DV = h->DV; p.hot_rows = h->DV ? h->hot_rows : 0;
     return p;
 }
 
@@ -227,6 +232,13 @@ int32_t step_impl(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t win
             W2V_CUDA(h, dev_alloc(&h->DU, need_du));
             h->DU_cap = need_du;
         }
+        const uint64_t need_dv = (uint64_t)h->hot_rows * h->d;
+        if (need_dv > h->DV_cap) {
+            cudaFree(h->DV); h->DV = nullptr; h->DV_cap = 0;
+            W2V_CUDA(h, dev_alloc(&h->DV, need_dv));
+            W2V_CUDA(h, cudaMemsetAsync(h->DV, 0, need_dv * sizeof(double), h->stream));
+            h->DV_cap = need_dv;
+        }
         if (h->st_host->pairs > 0) {
             StepParams p = make_params(h, window, negatives, lr);
             if ((rc = profile_mark(h)) != W2V_OK) return rc;
@@ -252,22 +264,29 @@ extern "C" {
 int32_t w2v_create(uint64_t vocab, uint32_t d, uint64_t seed, float *U, float *V, void *stream,
                    w2v_handle **out)
 {
+    return w2v_create_strided(vocab, d, d, seed, U, V, stream, out);
+}
+
+int32_t w2v_create_strided(uint64_t vocab, uint32_t d, uint32_t row_stride, uint64_t seed, float *U, float *V,
+                           void *stream, w2v_handle **out)
+{
     if (!out) return W2V_ERR_ARG;
     *out = nullptr;
     if (vocab < 2 || vocab >= (1ull << 31)) return W2V_ERR_ARG;
     if (d < 4 || d > 1024 || (d % 4) != 0) return W2V_ERR_ARG;
+    if (row_stride < d || row_stride > 2048 || (row_stride % 4) != 0) return W2V_ERR_ARG;
     if ((U == nullptr) != (V == nullptr)) return W2V_ERR_ARG;
     if (U && ((reinterpret_cast<uintptr_t>(U) | reinterpret_cast<uintptr_t>(V)) & 15u)) return W2V_ERR_ARG;
     w2v_handle *h = new (std::nothrow) w2v_handle();
     if (!h) return W2V_ERR_NOMEM;
-    h->vocab = vocab; h->d = d; h->seed = seed;
+    h->vocab = vocab; h->d = d; h->ld = row_stride; h->seed = seed;
     h->stream = static_cast<cudaStream_t>(stream);
     auto bail = [&](int32_t code) { w2v_destroy(h); return code; };
     if (cudaGetDevice(&h->device) != cudaSuccess) return bail(W2V_ERR_CUDA);
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device) == cudaSuccess && sms > 0)
         h->sms = sms;
-    const uint64_t elems = vocab * (uint64_t)d;
+    const uint64_t elems = vocab * (uint64_t)row_stride;
     if (!U) {
         if (dev_alloc(&h->U, elems) != cudaSuccess) { cudaGetLastError(); return bail(W2V_ERR_NOMEM); }
         h->owns_tables = true;
@@ -279,7 +298,7 @@ int32_t w2v_create(uint64_t vocab, uint32_t d, uint64_t seed, float *U, float *V
     if (cudaMallocHost(reinterpret_cast<void **>(&h->st_host), sizeof(DevState)) != cudaSuccess)
         return bail(W2V_ERR_NOMEM);
     if (cudaMemsetAsync(h->st, 0, sizeof(DevState), h->stream) != cudaSuccess) return bail(W2V_ERR_CUDA);
-    if (launch_init_tables(h->U, h->V, vocab, d, seed, h->stream) < 0) return bail(W2V_ERR_CUDA);
+    if (launch_init_tables(h->U, h->V, vocab, d, row_stride, seed, h->stream) < 0) return bail(W2V_ERR_CUDA);
     h->launches += 1;
     *out = h;
     return W2V_OK;
@@ -295,7 +314,7 @@ int32_t w2v_destroy(w2v_handle *h)
     free_scratch(h->sc);
     cudaFree(h->st);
     if (h->st_host) cudaFreeHost(h->st_host);
-    cudaFree(h->G); cudaFree(h->DU); cudaFree(h->tok_stage);
+    cudaFree(h->G); cudaFree(h->DU); cudaFree(h->DV); cudaFree(h->tok_stage);
     for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
     cudaGetLastError();
     delete h;
@@ -317,7 +336,7 @@ int32_t w2v_build_alias(w2v_handle *h, const uint64_t *counts, double subsample_
     }
     int rc;
     try {
-        rc = build_tables_host(counts, h->vocab, subsample_t, ta.data(), keep.data());
+        rc = build_tables_host(counts, h->vocab, subsample_t, ta.data(), keep.data(), &h->hot_rows);
     } catch (const std::bad_alloc &) {
         return fail(h, W2V_ERR_NOMEM, "host memory for the sampling tables");
     }
@@ -412,7 +431,7 @@ int32_t w2v_partial_dots(w2v_handle *h, const int32_t *pairs, uint64_t m, uint32
     if (m && (!pairs || !out)) return fail(h, W2V_ERR_ARG, "pairs or out is NULL");
     if (!(col_lo < col_hi && col_hi <= h->d)) return fail(h, W2V_ERR_ARG, "need 0 <= col_lo < col_hi <= d");
     DeviceGuard g(h->device);
-    int k = launch_partial_dots(h->U, h->V, (uint32_t)h->vocab, h->d, pairs, m, col_lo, col_hi, out, h->st,
+    int k = launch_partial_dots(h->U, h->V, (uint32_t)h->vocab, h->ld, pairs, m, col_lo, col_hi, out, h->st,
                                 h->sms, h->stream);
     if (k < 0) return fail(h, W2V_ERR_CUDA, "partial dots launch", cudaGetLastError());
     h->launches += (uint64_t)k;
@@ -426,7 +445,8 @@ static int32_t copy_rows(w2v_handle *h, uint32_t which, const int64_t *ids, uint
     if (m && (!ids || !buf)) return fail(h, W2V_ERR_ARG, "ids or buffer is NULL");
     if (reinterpret_cast<uintptr_t>(buf) & 15u) return fail(h, W2V_ERR_ARG, "row buffer must be 16-byte aligned");
     DeviceGuard g(h->device);
-    int k = launch_copy_rows(which ? h->V : h->U, (uint32_t)h->vocab, h->d, ids, m, buf, to_table, h->sms, h->stream);
+    int k = launch_copy_rows(which ? h->V : h->U, (uint32_t)h->vocab, h->d, h->ld, ids, m, buf, to_table, h->sms,
+                             h->stream);
     if (k < 0) return fail(h, W2V_ERR_CUDA, "row copy launch", cudaGetLastError());
     h->launches += (uint64_t)k;
     return W2V_OK;
@@ -461,6 +481,13 @@ int32_t w2v_get_table_ptrs(w2v_handle *h, float **U, float **V)
     if (!h) return W2V_ERR_ARG;
     if (U) *U = h->U;
     if (V) *V = h->V;
+    return W2V_OK;
+}
+
+int32_t w2v_get_row_stride(w2v_handle *h, uint32_t *row_stride)
+{
+    if (!h || !row_stride) return W2V_ERR_ARG;
+    *row_stride = h->ld;
     return W2V_OK;
 }
 

@@ -158,6 +158,24 @@ __device__ __forceinline__ void row_red_scaled(float4 *dst, float g, const Row<V
     }
 }
 
+// dst_row (double precision sums, d consecutive doubles) += g * r
+template <int VPL>
+__device__ __forceinline__ void row_add_scaled_f64(double *dst, float g, const Row<VPL> &r, uint32_t d4, uint32_t lane)
+{
+    const double gd = (double)g;
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+        const uint32_t idx = lane + 32u * v;
+        if (idx < d4) {
+            double *a = dst + 4u * idx;
+            atomicAdd(a + 0, gd * (double)r.x[v].x);
+            atomicAdd(a + 1, gd * (double)r.x[v].y);
+            atomicAdd(a + 2, gd * (double)r.x[v].z);
+            atomicAdd(a + 3, gd * (double)r.x[v].w);
+        }
+    }
+}
+
 __device__ __forceinline__ float sigmoidf_exact(float x)
 {
     return 1.0f / (1.0f + expf(-x));

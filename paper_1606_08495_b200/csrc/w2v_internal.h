@@ -49,6 +49,7 @@ struct StepParams {
     DevState *st;
     uint32_t vocab;
     uint32_t d4;                // d / 4
+    uint32_t ld4;               // row stride of U and V in float4 units (>= d4)
     uint32_t window;
     uint32_t negatives;
     uint32_t k0, k1;            // Philox key
@@ -58,6 +59,8 @@ struct StepParams {
     const unsigned long long *pair_off;   // first pair index of centre q
     float *G;                   // [pairs * (1 + negatives)] coefficients
     float *DU;                  // [kept * d] per-centre sums of G v(target)
+    double *DV;                 // [hot_rows * d] fp64 sums of G u(c) for the most-hit output rows
+    uint32_t hot_rows;          // output rows [0, hot_rows) accumulate in DV (snapshot mode)
 };
 
 struct Scratch {
@@ -74,7 +77,7 @@ struct Scratch {
 };
 
 // ---- launchers (each returns the number of kernels it launched, or -1 on a launch error) ----
-int launch_init_tables(float *U, float *V, uint64_t vocab, uint32_t d, uint64_t seed, cudaStream_t s);
+int launch_init_tables(float *U, float *V, uint64_t vocab, uint32_t d, uint32_t ld, uint64_t seed, cudaStream_t s);
 
 int launch_compact(const int32_t *tokens, uint64_t n, const SampleTables &tab, uint32_t vocab,
                    uint32_t k0, uint32_t k1, uint32_t step_lo, const Scratch &sc, DevState *st,
@@ -90,15 +93,17 @@ int launch_hogwild(const StepParams &p, uint32_t rows_in_flight, uint32_t blocks
 int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t blocks_per_sm, int sms,
                     cudaStream_t s);
 
-int launch_partial_dots(const float *U, const float *V, uint32_t vocab, uint32_t d,
+int launch_partial_dots(const float *U, const float *V, uint32_t vocab, uint32_t ld,
                         const int32_t *pairs, uint64_t m, uint32_t col_lo, uint32_t col_hi,
                         float *out, DevState *st, int sms, cudaStream_t s);
-int launch_copy_rows(float *table, uint32_t vocab, uint32_t d, const int64_t *ids, uint64_t m,
+int launch_copy_rows(float *table, uint32_t vocab, uint32_t d, uint32_t ld, const int64_t *ids, uint64_t m,
                      float *buf, bool to_table, int sms, cudaStream_t s);
 
 // ---- host-side table construction (w2v_tables.cpp) ----
-// Returns 0, or -1 if a count is zero.  thr_alias is [vocab] pairs, keep_thr [vocab].
+// Returns 0, or -1 if a count is zero.  thr_alias is [vocab] pairs, keep_thr [vocab];
+// hot_prefix receives the number of leading rows that are drawn as negatives often enough to
+// be summed in double precision by the snapshot update.
 int build_tables_host(const uint64_t *counts, uint64_t vocab, double subsample_t, uint2 *thr_alias,
-                      uint32_t *keep_thr);
+                      uint32_t *keep_thr, uint32_t *hot_prefix);
 
 }  // namespace w2v

@@ -9,40 +9,44 @@
 namespace w2v {
 
 // U[w][4 j4 .. 4 j4 + 3] = ((r >> 8) 2^-24 - 0.5) / d, r the four words of
-// Philox(seed; w, j4, 0, 0).
+// Philox(seed; w, j4, 0, 0).  Padding columns between d and the row stride are zeroed.
 __global__ void __launch_bounds__(256)
-init_u_kernel(float4 *__restrict__ U4, uint64_t total4, uint32_t d4, float d, uint32_t k0, uint32_t k1)
+init_u_kernel(float4 *__restrict__ U4, uint64_t total4, uint32_t d4, uint32_t ld4, float d, uint32_t k0,
+              uint32_t k1)
 {
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
     for (uint64_t idx = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total4; idx += stride) {
-        const uint32_t row = (uint32_t)(idx / d4), j4 = (uint32_t)(idx % d4);
-        const uint4 r = philox4x32_10(k0, k1, row, j4, kPurInit, 0);
-        const float s = 1.0f / 16777216.0f;
-        float4 o;
-        o.x = ((float)(r.x >> 8) * s - 0.5f) / d;
-        o.y = ((float)(r.y >> 8) * s - 0.5f) / d;
-        o.z = ((float)(r.z >> 8) * s - 0.5f) / d;
-        o.w = ((float)(r.w >> 8) * s - 0.5f) / d;
+        const uint32_t row = (uint32_t)(idx / ld4), j4 = (uint32_t)(idx % ld4);
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (j4 < d4) {
+            const uint4 r = philox4x32_10(k0, k1, row, j4, kPurInit, 0);
+            const float s = 1.0f / 16777216.0f;
+            o.x = ((float)(r.x >> 8) * s - 0.5f) / d;
+            o.y = ((float)(r.y >> 8) * s - 0.5f) / d;
+            o.z = ((float)(r.z >> 8) * s - 0.5f) / d;
+            o.w = ((float)(r.w >> 8) * s - 0.5f) / d;
+        }
         U4[idx] = o;
     }
 }
 
-int launch_init_tables(float *U, float *V, uint64_t vocab, uint32_t d, uint64_t seed, cudaStream_t s)
+int launch_init_tables(float *U, float *V, uint64_t vocab, uint32_t d, uint32_t ld, uint64_t seed,
+                       cudaStream_t s)
 {
-    const uint64_t total4 = vocab * (d / 4);
+    const uint64_t total4 = vocab * (ld / 4);
     const uint64_t want = (total4 + 255) / 256;
     const int grid = (int)(want < 148ull * 32 ? (want ? want : 1) : 148ull * 32);
-    init_u_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<float4 *>(U), total4, d / 4, (float)d,
+    init_u_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<float4 *>(U), total4, d / 4, ld / 4, (float)d,
                                        (uint32_t)seed, (uint32_t)(seed >> 32));
     if (cudaGetLastError() != cudaSuccess) return -1;
-    if (cudaMemsetAsync(V, 0, vocab * (uint64_t)d * sizeof(float), s) != cudaSuccess) return -1;
+    if (cudaMemsetAsync(V, 0, vocab * (uint64_t)ld * sizeof(float), s) != cudaSuccess) return -1;
     return 1;
 }
 
 // One warp per pair; lanes stride over the columns of the slice.  The 16-byte aligned
 // middle of the slice is read as float4, the ragged ends as scalars.
 __global__ void __launch_bounds__(kBlock)
-partial_dots_kernel(const float *__restrict__ U, const float *__restrict__ V, uint32_t vocab, uint32_t d,
+partial_dots_kernel(const float *__restrict__ U, const float *__restrict__ V, uint32_t vocab, uint32_t ld,
                     const int32_t *__restrict__ pairs, uint64_t m, uint32_t col_lo, uint32_t col_hi,
                     float *__restrict__ out, DevState *st)
 {
@@ -57,7 +61,7 @@ partial_dots_kernel(const float *__restrict__ U, const float *__restrict__ V, ui
             if (lane == 0) { out[i] = CUDART_NAN_F; atomicOr(&st->status, 1u); }
             continue;
         }
-        const float *u = U + (size_t)wi * d, *v = V + (size_t)wo * d;
+        const float *u = U + (size_t)wi * ld, *v = V + (size_t)wo * ld;
         float s = 0.f;
         if (a0 < a1) {
             for (uint32_t j = col_lo + lane; j < a0; j += 32) s = fmaf(__ldcg(u + j), __ldcg(v + j), s);
@@ -75,7 +79,7 @@ partial_dots_kernel(const float *__restrict__ U, const float *__restrict__ V, ui
     }
 }
 
-int launch_partial_dots(const float *U, const float *V, uint32_t vocab, uint32_t d, const int32_t *pairs,
+int launch_partial_dots(const float *U, const float *V, uint32_t vocab, uint32_t ld, const int32_t *pairs,
                         uint64_t m, uint32_t col_lo, uint32_t col_hi, float *out, DevState *st, int sms,
                         cudaStream_t s)
 {
@@ -83,14 +87,15 @@ int launch_partial_dots(const float *U, const float *V, uint32_t vocab, uint32_t
     const uint64_t want = (m + (kBlock / 32) - 1) / (kBlock / 32);
     const uint64_t cap = (uint64_t)sms * 8;
     const int grid = (int)(want < cap ? want : cap);
-    partial_dots_kernel<<<grid, kBlock, 0, s>>>(U, V, vocab, d, pairs, m, col_lo, col_hi, out, st);
+    partial_dots_kernel<<<grid, kBlock, 0, s>>>(U, V, vocab, ld, pairs, m, col_lo, col_hi, out, st);
     if (cudaGetLastError() != cudaSuccess) return -1;
     return 1;
 }
 
 // One warp per row, 16 bytes per lane per trip.
 __global__ void __launch_bounds__(kBlock)
-copy_rows_kernel(float4 *__restrict__ table, uint32_t vocab, uint32_t d4, const int64_t *__restrict__ ids,
+copy_rows_kernel(float4 *__restrict__ table, uint32_t vocab, uint32_t d4, uint32_t ld4,
+                 const int64_t *__restrict__ ids,
                  uint64_t m, float4 *__restrict__ buf, bool to_table)
 {
     const uint32_t lane = threadIdx.x & 31;
@@ -99,7 +104,7 @@ copy_rows_kernel(float4 *__restrict__ table, uint32_t vocab, uint32_t d4, const 
     for (uint64_t i = warp; i < m; i += nwarps) {
         const int64_t w = ids[i];
         if (w < 0 || (uint64_t)w >= vocab) continue;
-        float4 *row = table + (size_t)w * d4, *b = buf + (size_t)i * d4;
+        float4 *row = table + (size_t)w * ld4, *b = buf + (size_t)i * d4;
         for (uint32_t j = lane; j < d4; j += 32) {
             if (to_table) row[j] = b[j];
             else b[j] = __ldcg(row + j);
@@ -107,14 +112,14 @@ copy_rows_kernel(float4 *__restrict__ table, uint32_t vocab, uint32_t d4, const 
     }
 }
 
-int launch_copy_rows(float *table, uint32_t vocab, uint32_t d, const int64_t *ids, uint64_t m, float *buf,
-                     bool to_table, int sms, cudaStream_t s)
+int launch_copy_rows(float *table, uint32_t vocab, uint32_t d, uint32_t ld, const int64_t *ids, uint64_t m,
+                     float *buf, bool to_table, int sms, cudaStream_t s)
 {
     if (m == 0) return 0;
     const uint64_t want = (m + (kBlock / 32) - 1) / (kBlock / 32);
     const uint64_t cap = (uint64_t)sms * 8;
     const int grid = (int)(want < cap ? want : cap);
-    copy_rows_kernel<<<grid, kBlock, 0, s>>>(reinterpret_cast<float4 *>(table), vocab, d / 4, ids, m,
+    copy_rows_kernel<<<grid, kBlock, 0, s>>>(reinterpret_cast<float4 *>(table), vocab, d / 4, ld / 4, ids, m,
                                              reinterpret_cast<float4 *>(buf), to_table);
     if (cudaGetLastError() != cudaSuccess) return -1;
     return 1;

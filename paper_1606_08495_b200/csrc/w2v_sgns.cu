@@ -29,7 +29,7 @@ __device__ __forceinline__ void for_each_target(const StepParams &p, const Row<V
         for (int b = 0; b < TB; ++b) {
             const uint32_t t = t0 + b;
             tgt[b] = pair_target(t, w_out, n0, n1, wide);
-            if (t <= p.negatives) row_load(v[b], V4 + (size_t)tgt[b] * p.d4, p.d4, lane);
+            if (t <= p.negatives) row_load(v[b], V4 + (size_t)tgt[b] * p.ld4, p.d4, lane);
             else row_zero(v[b]);
         }
 #pragma unroll
@@ -66,7 +66,7 @@ sgns_hogwild_kernel(StepParams p)
         const uint32_t c = (uint32_t)p.ctok[q];
         const uint32_t i = p.cidx[q];
         Row<VPL> u, etot;
-        row_load(u, U4 + (size_t)c * p.d4, p.d4, lane);
+        row_load(u, U4 + (size_t)c * p.ld4, p.d4, lane);
         row_zero(etot);
         for (uint32_t pp = q - left; pp <= q + right; ++pp) {
             if (pp == q) continue;
@@ -79,12 +79,12 @@ sgns_hogwild_kernel(StepParams p)
                 [&](uint32_t t, uint32_t tgt, const Row<VPL> &v, float f) {
                     const float g = p.lr * ((t == 0 ? 1.0f : 0.0f) - sigmoidf_exact(f));
                     row_axpy(e, g, v);                                         // e += g v(t)
-                    row_red_scaled(V4 + (size_t)tgt * p.d4, g, u, p.d4, lane);  // v(t) += g u(c)
+                    row_red_scaled(V4 + (size_t)tgt * p.ld4, g, u, p.d4, lane);  // v(t) += g u(c)
                 });
             row_add(u, e);       // later pairs of this centre see the moved vector
             row_add(etot, e);
         }
-        row_red_scaled(U4 + (size_t)c * p.d4, 1.0f, etot, p.d4, lane);          // u(c) += sum e
+        row_red_scaled(U4 + (size_t)c * p.ld4, 1.0f, etot, p.d4, lane);          // u(c) += sum e
     }
     flush_draw_counts(p.st, draws, redraws);
 }
@@ -111,7 +111,7 @@ sgns_snap_dots_kernel(StepParams p)
         const uint32_t c = (uint32_t)p.ctok[q];
         const uint32_t i = p.cidx[q];
         Row<VPL> u, du;
-        row_load(u, U4 + (size_t)c * p.d4, p.d4, lane);
+        row_load(u, U4 + (size_t)c * p.ld4, p.d4, lane);
         row_zero(du);
         unsigned long long gi = p.pair_off[q] * n1p;
         for (uint32_t pp = q - left; pp <= q + right; ++pp) {
@@ -159,7 +159,7 @@ sgns_snap_adjust_v_kernel(StepParams p)
         const uint32_t c = (uint32_t)p.ctok[q];
         const uint32_t i = p.cidx[q];
         Row<VPL> u;
-        row_load(u, U4 + (size_t)c * p.d4, p.d4, lane);
+        row_load(u, U4 + (size_t)c * p.ld4, p.d4, lane);
         unsigned long long gi = p.pair_off[q] * n1p;
         for (uint32_t pp = q - left; pp <= q + right; ++pp) {
             if (pp == q) continue;
@@ -169,9 +169,31 @@ sgns_snap_adjust_v_kernel(StepParams p)
             for (uint32_t t = 0; t <= p.negatives; ++t) {
                 const uint32_t tgt = pair_target(t, w_out, n0, n1, wide);
                 const float g = __ldcg(p.G + gi + t);
-                row_red_scaled(V4 + (size_t)tgt * p.d4, g, u, p.d4, lane);
+                if (tgt < p.hot_rows) row_add_scaled_f64(p.DV + (size_t)tgt * (4u * p.d4), g, u, p.d4, lane);
+                else row_red_scaled(V4 + (size_t)tgt * p.ld4, g, u, p.d4, lane);
             }
             gi += n1p;
+        }
+    }
+}
+
+// ---- snapshot mode, pass 2b: the most-hit output rows --------------------------------------
+// A row that is drawn as a negative tens of thousands of times in one step would collect one
+// fp32 rounding error per addition; its sum is kept in double precision instead and added
+// here with a single rounding.  The sums are left at zero for the next step.
+__global__ void __launch_bounds__(kBlock)
+sgns_snap_apply_hot_kernel(StepParams p)
+{
+    const uint32_t d = 4u * p.d4, ld = 4u * p.ld4;
+    const uint64_t total = (uint64_t)p.hot_rows * d;
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const double x = p.DV[i];
+        if (x != 0.0) {
+            const uint64_t row = i / d, col = i % d;
+            float *v = p.V + row * ld + col;
+            *v = (float)((double)*v + x);
+            p.DV[i] = 0.0;
         }
     }
 }
@@ -191,7 +213,7 @@ sgns_snap_apply_u_kernel(StepParams p)
         const uint32_t c = (uint32_t)p.ctok[q];
         for (uint32_t idx = lane; idx < p.d4; idx += 32) {
             const float4 x = __ldcg(DU4 + (size_t)q * p.d4 + idx);
-            red_add_f32x4(U4 + (size_t)c * p.d4 + idx, x.x, x.y, x.z, x.w);
+            red_add_f32x4(U4 + (size_t)c * p.ld4 + idx, x.x, x.y, x.z, x.w);
         }
     }
 }
@@ -296,12 +318,19 @@ int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t block
         case 7: snap_adjust_v<7>(p, blocks_per_sm, sms, s); break;
         default: snap_adjust_v<8>(p, blocks_per_sm, sms, s); break;
     }
+    int launched = 3;
+    if (p.hot_rows) {
+        const uint64_t want = ((uint64_t)p.hot_rows * 4u * p.d4 + kBlock - 1) / kBlock;
+        const int grid = (int)(want < (uint64_t)sms * 8 ? want : (uint64_t)sms * 8);
+        sgns_snap_apply_hot_kernel<<<grid, kBlock, 0, s>>>(p);
+        ++launched;
+    }
     {
         const int grid = grid_for(sgns_snap_apply_u_kernel, blocks_per_sm, sms);
         sgns_snap_apply_u_kernel<<<grid, kBlock, 0, s>>>(p);
     }
     if (cudaGetLastError() != cudaSuccess) return -1;
-    return 3;
+    return launched;
 }
 
 }  // namespace w2v

@@ -10,6 +10,9 @@
 
 namespace w2v {
 
+constexpr double kHotChance = 2e-5;     // per draw
+constexpr uint64_t kHotRowsMax = 8192;
+
 static inline uint2 entry(uint32_t thr, uint32_t alias)
 {
     uint2 e;
@@ -19,7 +22,7 @@ static inline uint2 entry(uint32_t thr, uint32_t alias)
 }
 
 int build_tables_host(const uint64_t *counts, uint64_t vocab, double subsample_t, uint2 *thr_alias,
-                      uint32_t *keep_thr)
+                      uint32_t *keep_thr, uint32_t *hot_prefix)
 {
     const double two32 = 4294967296.0;
     std::vector<double> q(vocab);
@@ -40,8 +43,14 @@ int build_tables_host(const uint64_t *counts, uint64_t vocab, double subsample_t
     under.reserve(vocab);
     over.reserve(vocab);
     const double scale = static_cast<double>(vocab);
+    // Leading rows whose chance of being drawn as a negative is at least kHotChance: with word ids
+    // in frequency order these are the rows that receive thousands of additions per step.
+    const double hot_q = kHotChance * scale;
+    uint64_t hot = 0;
+    bool in_prefix = true;
     for (uint64_t w = 0; w < vocab; ++w) {
         q[w] = (q[w] * scale) / wsum;
+        if (in_prefix && q[w] >= hot_q && hot < kHotRowsMax) ++hot; else in_prefix = false;
         (q[w] < 1.0 ? under : over).push_back(static_cast<uint32_t>(w));
         thr_alias[w] = entry(0xFFFFFFFFu, static_cast<uint32_t>(w));
     }
@@ -68,6 +77,7 @@ int build_tables_host(const uint64_t *counts, uint64_t vocab, double subsample_t
         }
         keep_thr[w] = thr;
     }
+    if (hot_prefix) *hot_prefix = static_cast<uint32_t>(hot);
     return 0;
 }
 

@@ -5,11 +5,11 @@ from oracle import Oracle
 from paper_1606_08495_b200 import binding, corpus
 
 
-def make_pair(cfg, seed=11, sparse=False, counts=None, t=None):
+def make_pair(cfg, seed=11, sparse=False, counts=None, t=None, row_stride=None):
     cp = corpus.Corpus(cfg) if counts is None else None
     counts = cp.counts if counts is None else np.asarray(counts, dtype=np.uint64)
     t = cfg["subsample_t"] if t is None else t
-    gpu = binding.W2V(cfg["vocab"], cfg["d"], seed)
+    gpu = binding.W2V(cfg["vocab"], cfg["d"], seed, row_stride=row_stride)
     cpu = Oracle(cfg["vocab"], cfg["d"], seed, sparse=sparse)
     gpu.build_alias(counts, t)
     cpu.build_tables(counts, t)

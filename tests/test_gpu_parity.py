@@ -178,8 +178,8 @@ def test_read_write_rows_roundtrip():
 
 
 # ---------------------------------------------------------------- snapshot mode
-def check_snapshot_steps(cfg, steps, words=None, seed=11):
-    gpu, cpu, cp = make_pair(cfg, seed=seed)
+def check_snapshot_steps(cfg, steps, words=None, seed=11, row_stride=None):
+    gpu, cpu, cp = make_pair(cfg, seed=seed, row_stride=row_stride)
     W, N, lr = cfg["window"], cfg["negatives"], cfg["lr"]
     worst = 0.0
     for i in range(steps):
@@ -220,6 +220,45 @@ def test_snapshot_steps_medium_shape():
 def test_snapshot_other_dimensions(d):
     cfg = corpus.scaled(TINY, vocab=3000, d=d, minibatch=1500, corpus_tokens=100_000)
     check_snapshot_steps(cfg, steps=2)
+
+
+@pytest.mark.parametrize("d,row_stride", [(300, 320), (300, 304), (100, 128), (8, 16), (132, 2048)])
+def test_snapshot_padded_rows(d, row_stride):
+    # rows on 64-byte boundaries: same vectors, same step, only the addresses differ
+    cfg = corpus.scaled(TINY, vocab=3000, d=d, minibatch=1500, corpus_tokens=100_000)
+    check_snapshot_steps(cfg, steps=2, row_stride=row_stride)
+
+
+def test_padded_rows_init_dots_and_padding_untouched():
+    V, d, ld = 2000, 300, 304
+    gpu = binding.W2V(V, d, seed=5, row_stride=ld)
+    cpu = Oracle(V, d, seed=5)
+    assert binding.w2v_get_row_stride(gpu.h) == ld
+    ids = np.arange(V)
+    assert np.array_equal(gpu.read_rows(0, ids).view(np.uint32), cpu.read_rows(0, ids).view(np.uint32))
+    rng = np.random.default_rng(3)
+    Vt = rng.normal(scale=0.3, size=(V, d)).astype(np.float32)
+    gpu.write_rows(1, ids, Vt); cpu.write_rows(1, ids, Vt)
+    pairs = rng.integers(0, V, size=(3000, 2)).astype(np.int32)
+    for lo, hi in [(0, d), (3, 9), (297, 300), (90, 120)]:
+        want = cpu.partial_dots(pairs, lo, hi)
+        assert np.allclose(gpu.partial_dots(pairs, lo, hi), want, rtol=0, atol=1e-6)
+    counts = np.full(V, 50, dtype=np.uint64)
+    gpu.build_alias(counts, 0.0)
+    toks = np.append(rng.integers(0, V, size=4000).astype(np.int32), -1)
+    gpu.sgns_step(toks, 5, 5, 0.025, binding.MODE_HOGWILD)
+    gpu.sgns_step(toks, 5, 5, 0.025, binding.MODE_SNAPSHOT)
+    pad_u = gpu.U.view(V, ld)[:, d:]
+    pad_v = gpu.V.view(V, ld)[:, d:]
+    assert not pad_u.any().item() and not pad_v.any().item()
+    gpu.close()
+
+
+def test_create_strided_rejects_bad_strides():
+    for d, ld in [(300, 296), (300, 302), (8, 2052)]:
+        with pytest.raises(binding.W2VError) as e:
+            binding.W2V(10, d, seed=1, row_stride=ld)
+        assert e.value.code == binding.W2V_ERR_ARG
 
 
 def test_snapshot_result_does_not_depend_on_launch_shape():
