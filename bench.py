@@ -32,9 +32,10 @@ UNIT = "pairs/s"
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes moved per algorithmic byte by the Hogwild update kernel on the large workload, from
 # the one-pass ncu capture summarised in profiles/sgns_update_kernels_large.md
-# ((dram__bytes_read.sum + dram__bytes_write.sum) / model bytes of the captured launch: 127.8 / 121.9 GB).
-# Applies to the large workload in Hogwild mode only; other workloads report null.
-TRAFFIC_PER_ALGORITHMIC_BYTE = 1.049
+# ((dram__bytes_read.sum + dram__bytes_write.sum) / model bytes of the captured launch: 126.42 / 121.9 GB,
+# rows on 128-byte boundaries).  Applies to the large workload in Hogwild mode with the default row
+# stride and launch shape only; anything else reports null.
+TRAFFIC_PER_ALGORITHMIC_BYTE = 1.037
 
 
 def algorithmic_bytes(d, centres, pairs, negatives):
@@ -314,7 +315,8 @@ def run_gpu(args):
                          "algorithmic_bytes_per_launch": per_launch_bytes,
                          "kernel_ms_per_launch": kernel_ms / max(1, groups),
                          "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE * per_launch_bytes
-                                     if name == "large" and args.mode == "hogwild" else None)},
+                                     if name == "large" and args.mode == "hogwild" and not args.row_stride
+                                     and not args.rows_in_flight and not args.blocks_per_sm else None)},
         }
         if world == 1 and not args.no_cpu_baseline:
             words = args.cpu_words
