@@ -185,6 +185,19 @@ def run_reference(args):
 # --------------------------------------------------------------------------------------------
 # the CUDA library
 # --------------------------------------------------------------------------------------------
+def reduce_over_ranks(ms, e2e_ms, pairs, e2e_pairs, launches, world, device):
+    """Whole-job figures from one rank's: the slowest rank's times, work and launches summed."""
+    if world <= 1:
+        return ms, e2e_ms, pairs, e2e_pairs, launches
+    import torch
+    import torch.distributed as dist
+
+    vals = torch.tensor([ms, e2e_ms, pairs, e2e_pairs, float(launches)], dtype=torch.float64, device=device)
+    mx = vals.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+    sm = vals.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+    return float(mx[0]), float(mx[1]), float(sm[2]), float(sm[3]), int(sm[4])
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -277,14 +290,8 @@ def run_gpu(args):
     tot_pairs = float(sum(pairs))
     model_bytes = algorithmic_bytes if args.mode == "hogwild" else algorithmic_bytes_snapshot
     tot_bytes = float(sum(model_bytes(d, c, p, N) for c, p in zip(centres, pairs)))
-    vals = torch.tensor([ms, e2e_ms, tot_pairs, float(e2e_pairs), float(launches)], dtype=torch.float64, device=dev)
-    if world > 1:
-        mx = vals.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
-        sm = vals.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
-        ms, e2e_ms = float(mx[0]), float(mx[1])
-        all_pairs, all_e2e_pairs, all_launches = float(sm[2]), float(sm[3]), int(sm[4])
-    else:
-        all_pairs, all_e2e_pairs, all_launches = tot_pairs, float(e2e_pairs), launches
+    ms, e2e_ms, all_pairs, all_e2e_pairs, all_launches = reduce_over_ranks(
+        ms, e2e_ms, tot_pairs, float(e2e_pairs), launches, world, dev)
 
     if rank == 0:
         peak, peak_kind = measured_peak()

@@ -177,6 +177,59 @@ int32_t w2v_sample_pairs(w2v_handle *h, const int32_t *tokens, uint64_t n, uint3
                          uint64_t cap, uint64_t *n_pairs, w2v_step_stats *stats);
 
 /*
+ * ---- Column shards: the paper's own partition (Section 5.1, Eq. (6)-(7)) ----------------------
+ * Shard s of S holds columns [col_lo, col_hi) of every row of U and V.  One minibatch is
+ *   1. every shard: w2v_shard_dots    -- Algorithm 1 ("dotprod") on its slice, for the index
+ *                                        sets that every shard regenerates from the same seed;
+ *   2. the partial dots are summed over the shards (Algorithm 3, "(F+, F-) <- sum_s");
+ *   3. every shard: w2v_shard_adjust  -- G+ = lr (1 - s(F+)), G- = -lr s(F-) (Algorithm 3) and
+ *                                        Algorithm 2 ("adjust") on its own columns.
+ * Step 2 is either a collective of the caller (w2v_shard_dots adding into one local array, then
+ * an all-reduce), or it is done by w2v_shard_dots itself: given the F arrays of all shards
+ * (peer-to-peer device pointers), the kernel that computes the partial dots adds them into every
+ * one of them, and after a barrier each shard holds the full sums.
+ *
+ * w2v_create_shard: as w2v_create_strided, for a model that stores only columns
+ * [col_lo, col_hi) of vectors that have d_full columns; col_lo and col_hi multiples of 4.
+ * Initial values are those the whole model would have in these columns.  U, V: vocab*row_stride
+ * floats with row_stride >= col_hi - col_lo.  On the handle of a shard, d means the slice width
+ * in every other call (w2v_read_rows returns col_hi - col_lo floats per row; w2v_partial_dots
+ * takes columns relative to col_lo), and w2v_sgns_step is refused with W2V_ERR_STATE.
+ * All shards must be given the same vocab, d_full, seed, tables, chunks and step numbers.
+ */
+int32_t w2v_create_shard(uint64_t vocab, uint32_t d_full, uint32_t col_lo, uint32_t col_hi,
+                         uint32_t row_stride, uint64_t seed, float *U, float *V, void *stream,
+                         w2v_handle **out);
+
+/*
+ * Algorithm 1 on this handle's columns for the chunk's index sets (sampled exactly as
+ * w2v_sgns_step would).  Target number j = pair*(1+negatives) + t (t = 0 the context word,
+ * t >= 1 negative t-1; pairs in the order of w2v_sample_pairs) gets its partial dot product
+ * ADDED to F_peers[r][j] for every r < n_peers.
+ *   tokens   device, n int32.
+ *   F_peers  host array of n_peers (1..16) device pointers, each to cap floats that the caller
+ *            zeroed before the first shard of this step adds to them; pointers into other
+ *            GPUs' memory are allowed when peer access is enabled.
+ *   stats    host, may be NULL.
+ * Waits once for the pair count.  Returns W2V_ERR_CAPACITY (nothing added) if the chunk has more
+ * than cap targets.  Leaves the sampled chunk in the handle for w2v_shard_adjust; any other
+ * sampling call or w2v_set_step in between cancels the pending step.
+ */
+int32_t w2v_shard_dots(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window,
+                       uint32_t negatives, float *const *F_peers, uint32_t n_peers, uint64_t cap,
+                       w2v_step_stats *stats);
+
+/*
+ * Algorithms 3 and 2 for the step begun by w2v_shard_dots: coefficients from the summed dot
+ * products, then u(centre) += sum G v(target) and v(target) += G u(centre) on this handle's
+ * columns, every vector read as it was at the start of the call.  Adds one to the step number.
+ *   F  device, the dot products summed over all shards, indexed as in w2v_shard_dots; every
+ *      shard's additions must have completed (the caller's barrier or collective).
+ * Asynchronous.  Errors: W2V_ERR_STATE without a pending w2v_shard_dots.
+ */
+int32_t w2v_shard_adjust(w2v_handle *h, const float *F, float lr);
+
+/*
  * Partial dot products of one column slice, the body of Algorithm 1 on shard s:
  * out[i] = sum_{j = col_lo}^{col_hi - 1} U[pairs[2i]][j] * V[pairs[2i+1]][j].
  * Summing the results over any partition of [0, d) gives the full dot products

@@ -20,7 +20,8 @@ MODE_SNAPSHOT, MODE_HOGWILD = 0, 1
 TABLE_U, TABLE_V = 0, 1
 
 EXPORTS = (
-    "w2v_create", "w2v_create_strided", "w2v_get_row_stride", "w2v_destroy", "w2v_build_alias", "w2v_get_tables", "w2v_sgns_step",
+    "w2v_create", "w2v_create_strided", "w2v_create_shard", "w2v_shard_dots", "w2v_shard_adjust",
+    "w2v_get_row_stride", "w2v_destroy", "w2v_build_alias", "w2v_get_tables", "w2v_sgns_step",
     "w2v_sgns_step_host", "w2v_sample_pairs", "w2v_partial_dots", "w2v_read_rows", "w2v_write_rows",
     "w2v_set_step", "w2v_get_step", "w2v_get_table_ptrs", "w2v_sync", "w2v_profile_enable",
     "w2v_profile_read", "w2v_get_launch_count", "w2v_set_tuning", "w2v_last_error",
@@ -66,6 +67,9 @@ def load():
         "w2v_create": [u64, u32, u64, vp, vp, vp, C.POINTER(vp)],
         "w2v_create_strided": [u64, u32, u32, u64, vp, vp, vp, C.POINTER(vp)],
         "w2v_get_row_stride": [vp, C.POINTER(u32)],
+        "w2v_create_shard": [u64, u32, u32, u32, u32, u64, vp, vp, vp, C.POINTER(vp)],
+        "w2v_shard_dots": [vp, vp, u64, u32, u32, C.POINTER(vp), u32, u64, C.POINTER(StepStats)],
+        "w2v_shard_adjust": [vp, vp, C.c_float],
         "w2v_destroy": [vp],
         "w2v_build_alias": [vp, vp, C.c_double],
         "w2v_get_tables": [vp, vp, vp, vp],
@@ -129,6 +133,27 @@ def w2v_create_strided(vocab, d, row_stride, seed, U, V, stream):
     if rc != W2V_OK:
         raise W2VError(rc, "w2v_create_strided rejected its arguments or could not allocate")
     return h
+
+
+def w2v_create_shard(vocab, d_full, col_lo, col_hi, row_stride, seed, U, V, stream):
+    h = C.c_void_p()
+    rc = load().w2v_create_shard(int(vocab), int(d_full), int(col_lo), int(col_hi), int(row_stride), int(seed),
+                                 _ptr(U), _ptr(V), stream, C.byref(h))
+    if rc != W2V_OK:
+        raise W2VError(rc, "w2v_create_shard rejected its arguments or could not allocate")
+    return h
+
+
+def w2v_shard_dots(h, tokens, n, window, negatives, F_peers, cap, stats=None, allow=()):
+    """F_peers: device pointers (ints or tensors), one array of `cap` floats per shard."""
+    ptrs = (C.c_void_p * len(F_peers))(*[_ptr(f) for f in F_peers])
+    ref = C.byref(stats) if stats is not None else None
+    return _check(h, load().w2v_shard_dots(h, _ptr(tokens), int(n), window, negatives, ptrs, len(F_peers),
+                                           int(cap), ref), allow)
+
+
+def w2v_shard_adjust(h, F, lr):
+    return _check(h, load().w2v_shard_adjust(h, _ptr(F), float(lr)))
 
 
 def w2v_get_row_stride(h):
@@ -238,19 +263,24 @@ def aligned_row_stride(d):
 class W2V:
     """Tables U and V as torch tensors on one GPU plus the library handle."""
 
-    def __init__(self, vocab, d, seed, device="cuda:0", row_stride=None):
+    def __init__(self, vocab, d, seed, device="cuda:0", row_stride=None, columns=None):
+        """columns=(col_lo, col_hi) makes this model one column shard of vectors with d columns;
+        its own d is then the slice width."""
         load()
         if not torch.cuda.is_available():
             raise RuntimeError("libw2v needs a CUDA device; there is no CPU path")
         self.device = torch.device(device)
-        self.vocab, self.d, self.seed = int(vocab), int(d), int(seed)
+        self.vocab, self.seed = int(vocab), int(seed)
+        self.d_full = int(d)
+        self.col_lo, self.col_hi = (0, self.d_full) if columns is None else (int(columns[0]), int(columns[1]))
+        self.d = self.col_hi - self.col_lo
         self.row_stride = self.d if row_stride is None else int(row_stride)
         with torch.cuda.device(self.device):
             self.U = torch.empty(self.vocab * self.row_stride, dtype=torch.float32, device=self.device)
             self.V = torch.empty(self.vocab * self.row_stride, dtype=torch.float32, device=self.device)
             self.stream = torch.cuda.current_stream(self.device)
-            self.h = w2v_create_strided(self.vocab, self.d, self.row_stride, self.seed, self.U, self.V,
-                                        self.stream.cuda_stream)
+            self.h = w2v_create_shard(self.vocab, self.d_full, self.col_lo, self.col_hi, self.row_stride,
+                                      self.seed, self.U, self.V, self.stream.cuda_stream)
 
     def close(self):
         if getattr(self, "h", None):

@@ -15,6 +15,13 @@ struct w2v_handle {
     uint64_t vocab = 0;
     uint32_t d = 0;
     uint32_t ld = 0;                 // row stride of U and V in floats (>= d, a multiple of 4)
+    uint32_t d_full = 0;             // columns of the whole vectors (== d unless this is a column shard)
+    uint32_t col_lo = 0;             // first column held (0 unless this is a column shard)
+    bool is_shard = false;
+    // state between w2v_shard_dots and w2v_shard_adjust
+    bool shard_pending = false;
+    uint32_t pend_window = 0, pend_negatives = 0;
+    uint64_t pend_n = 0, pend_pairs = 0;
     uint64_t seed = 0;
     uint64_t step_id = 0;
     int device = 0;
@@ -145,6 +152,7 @@ int32_t enqueue_sampling(w2v_handle *h, const int32_t *tokens, uint64_t n, uint3
 {
     int32_t rc = ensure_scratch(h, n);
     if (rc != W2V_OK) return rc;
+    h->shard_pending = false;            // the scratch a pending w2v_shard_adjust would need is overwritten
     W2V_CUDA(h, cudaMemsetAsync(h->st, 0, sizeof(DevState), h->stream));
     const uint32_t k0 = (uint32_t)h->seed;
     const uint32_t k1 = (uint32_t)(h->seed >> 32) ^ (uint32_t)(h->step_id >> 32);
@@ -203,6 +211,8 @@ int32_t step_impl(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t win
                   float lr, uint32_t mode, w2v_step_stats *stats)
 {
     if (mode > 1) return fail(h, W2V_ERR_ARG, "mode must be 0 (snapshot) or 1 (hogwild)");
+    if (h->is_shard)
+        return fail(h, W2V_ERR_STATE, "a column shard steps through w2v_shard_dots and w2v_shard_adjust");
     int32_t rc = enqueue_sampling(h, tokens, n, window);
     if (rc != W2V_OK) return rc;
     if (mode == W2V_MODE_HOGWILD) {
@@ -270,16 +280,25 @@ int32_t w2v_create(uint64_t vocab, uint32_t d, uint64_t seed, float *U, float *V
 int32_t w2v_create_strided(uint64_t vocab, uint32_t d, uint32_t row_stride, uint64_t seed, float *U, float *V,
                            void *stream, w2v_handle **out)
 {
+    return w2v_create_shard(vocab, d, 0, d, row_stride, seed, U, V, stream, out);
+}
+
+int32_t w2v_create_shard(uint64_t vocab, uint32_t d_full, uint32_t col_lo, uint32_t col_hi, uint32_t row_stride,
+                         uint64_t seed, float *U, float *V, void *stream, w2v_handle **out)
+{
     if (!out) return W2V_ERR_ARG;
     *out = nullptr;
     if (vocab < 2 || vocab >= (1ull << 31)) return W2V_ERR_ARG;
-    if (d < 4 || d > 1024 || (d % 4) != 0) return W2V_ERR_ARG;
+    if (d_full < 4 || d_full > 1024 || (d_full % 4) != 0) return W2V_ERR_ARG;
+    if (!(col_lo < col_hi && col_hi <= d_full) || (col_lo % 4) != 0 || (col_hi % 4) != 0) return W2V_ERR_ARG;
+    const uint32_t d = col_hi - col_lo;
     if (row_stride < d || row_stride > 2048 || (row_stride % 4) != 0) return W2V_ERR_ARG;
     if ((U == nullptr) != (V == nullptr)) return W2V_ERR_ARG;
     if (U && ((reinterpret_cast<uintptr_t>(U) | reinterpret_cast<uintptr_t>(V)) & 15u)) return W2V_ERR_ARG;
     w2v_handle *h = new (std::nothrow) w2v_handle();
     if (!h) return W2V_ERR_NOMEM;
     h->vocab = vocab; h->d = d; h->ld = row_stride; h->seed = seed;
+    h->d_full = d_full; h->col_lo = col_lo; h->is_shard = d != d_full;
     h->stream = static_cast<cudaStream_t>(stream);
     auto bail = [&](int32_t code) { w2v_destroy(h); return code; };
     if (cudaGetDevice(&h->device) != cudaSuccess) return bail(W2V_ERR_CUDA);
@@ -298,7 +317,7 @@ int32_t w2v_create_strided(uint64_t vocab, uint32_t d, uint32_t row_stride, uint
     if (cudaMallocHost(reinterpret_cast<void **>(&h->st_host), sizeof(DevState)) != cudaSuccess)
         return bail(W2V_ERR_NOMEM);
     if (cudaMemsetAsync(h->st, 0, sizeof(DevState), h->stream) != cudaSuccess) return bail(W2V_ERR_CUDA);
-    if (launch_init_tables(h->U, h->V, vocab, d, row_stride, seed, h->stream) < 0) return bail(W2V_ERR_CUDA);
+    if (launch_init_tables(h->U, h->V, vocab, d, row_stride, d_full, col_lo, seed, h->stream) < 0) return bail(W2V_ERR_CUDA);
     h->launches += 1;
     *out = h;
     return W2V_OK;
@@ -424,6 +443,93 @@ int32_t w2v_sample_pairs(w2v_handle *h, const int32_t *tokens, uint64_t n, uint3
     return W2V_OK;
 }
 
+int32_t w2v_shard_dots(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window, uint32_t negatives,
+                       float *const *F_peers, uint32_t n_peers, uint64_t cap, w2v_step_stats *stats)
+{
+    int32_t rc = check_step_args(h, tokens, n, window, negatives);
+    if (rc != W2V_OK) return rc;
+    if (!F_peers || n_peers < 1 || n_peers > (uint32_t)kMaxShards)
+        return fail(h, W2V_ERR_ARG, "need between 1 and 16 arrays for the partial dot products");
+    ShardPeers peers;
+    std::memset(&peers, 0, sizeof(peers));
+    for (uint32_t r = 0; r < n_peers; ++r) {
+        if (!F_peers[r]) return fail(h, W2V_ERR_ARG, "an array for the partial dot products is NULL");
+        peers.F[r] = F_peers[r];
+    }
+    peers.n = n_peers;
+    DeviceGuard g(h->device);
+    if ((rc = enqueue_sampling(h, tokens, n, window)) != W2V_OK) return rc;
+    int k = launch_pair_offsets(n, h->sc, h->st, h->stream);
+    if (k < 0) return fail(h, W2V_ERR_CUDA, "pair offset launch", cudaGetLastError());
+    h->launches += (uint64_t)k;
+    if ((rc = read_state(h, n, nullptr)) != W2V_OK) return rc;      // the pair count sizes everything below
+    const uint64_t pairs = h->st_host->pairs;
+    if (pairs * (uint64_t)(negatives + 1) > cap)
+        return fail(h, W2V_ERR_CAPACITY, "more targets than the arrays for the partial dot products hold");
+    if (pairs > 0) {
+        StepParams p = make_params(h, window, negatives, 0.f);
+        if ((rc = profile_mark(h)) != W2V_OK) return rc;
+        k = launch_shard_dots(p, peers, h->sms, h->stream);
+        if (k < 0) return fail(h, W2V_ERR_CUDA, "partial dots launch", cudaGetLastError());
+        h->launches += (uint64_t)k;
+        if (h->profiling) h->prof_launches += (uint64_t)k;
+        if ((rc = profile_mark(h)) != W2V_OK) return rc;
+    }
+    h->shard_pending = true;
+    h->pend_window = window; h->pend_negatives = negatives; h->pend_n = n; h->pend_pairs = pairs;
+    if (stats) {
+        if ((rc = read_state(h, n, stats)) != W2V_OK) return rc;
+        if (stats->status & 1u) return fail(h, W2V_ERR_TOKEN_RANGE, "token ids outside [-1, vocab) were skipped");
+    }
+    return W2V_OK;
+}
+
+int32_t w2v_shard_adjust(w2v_handle *h, const float *F, float lr)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (!h->shard_pending) return fail(h, W2V_ERR_STATE, "w2v_shard_adjust needs the w2v_shard_dots call of the same step before it");
+    const uint64_t targets = h->pend_pairs * (uint64_t)(h->pend_negatives + 1);
+    if (targets && !F) return fail(h, W2V_ERR_ARG, "F is NULL");
+    DeviceGuard g(h->device);
+    int32_t rc;
+    if (targets > h->G_cap) {
+        W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+        cudaFree(h->G); h->G = nullptr; h->G_cap = 0;
+        const uint64_t cap = targets + targets / 4 + 1024;
+        W2V_CUDA(h, dev_alloc(&h->G, cap));
+        h->G_cap = cap;
+    }
+    const uint64_t need_du = h->sc.n_cap * (uint64_t)h->d;
+    if (need_du > h->DU_cap) {
+        W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+        cudaFree(h->DU); h->DU = nullptr; h->DU_cap = 0;
+        W2V_CUDA(h, dev_alloc(&h->DU, need_du));
+        h->DU_cap = need_du;
+    }
+    const uint64_t need_dv = (uint64_t)h->hot_rows * h->d;
+    if (need_dv > h->DV_cap) {
+        W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+        cudaFree(h->DV); h->DV = nullptr; h->DV_cap = 0;
+        W2V_CUDA(h, dev_alloc(&h->DV, need_dv));
+        W2V_CUDA(h, cudaMemsetAsync(h->DV, 0, need_dv * sizeof(double), h->stream));
+        h->DV_cap = need_dv;
+    }
+    if (targets) {
+        StepParams p = make_params(h, h->pend_window, h->pend_negatives, lr);
+        if ((rc = profile_mark(h)) != W2V_OK) return rc;
+        int k = launch_shard_coefficients(F, h->G, targets, h->pend_negatives + 1, lr, h->sms, h->stream);
+        int k2 = k < 0 ? -1 : launch_shard_du(p, h->sms, h->stream);
+        int k3 = k2 < 0 ? -1 : launch_snapshot_apply(p, h->blocks_per_sm, h->sms, h->stream);
+        if (k3 < 0) return fail(h, W2V_ERR_CUDA, "adjust launch", cudaGetLastError());
+        h->launches += (uint64_t)(k + k2 + k3);
+        if (h->profiling) h->prof_launches += (uint64_t)(k + k2 + k3);
+        if ((rc = profile_mark(h)) != W2V_OK) return rc;
+    }
+    h->shard_pending = false;
+    h->step_id += 1;
+    return W2V_OK;
+}
+
 int32_t w2v_partial_dots(w2v_handle *h, const int32_t *pairs, uint64_t m, uint32_t col_lo, uint32_t col_hi,
                          float *out)
 {
@@ -466,6 +572,7 @@ int32_t w2v_set_step(w2v_handle *h, uint64_t step_id)
 {
     if (!h) return W2V_ERR_ARG;
     h->step_id = step_id;
+    h->shard_pending = false;            // the pending adjust would regenerate other negatives
     return W2V_OK;
 }
 

@@ -63,6 +63,13 @@ struct StepParams {
     uint32_t hot_rows;          // output rows [0, hot_rows) accumulate in DV (snapshot mode)
 };
 
+// F arrays of all shards (this one included) that receive a shard's partial dot products.
+constexpr int kMaxShards = 16;
+struct ShardPeers {
+    float *F[kMaxShards];
+    uint32_t n;
+};
+
 struct Scratch {
     uint64_t n_cap = 0;
     uint8_t *flags = nullptr;
@@ -77,7 +84,9 @@ struct Scratch {
 };
 
 // ---- launchers (each returns the number of kernels it launched, or -1 on a launch error) ----
-int launch_init_tables(float *U, float *V, uint64_t vocab, uint32_t d, uint32_t ld, uint64_t seed, cudaStream_t s);
+// d columns per row starting at column col_lo of vectors that have d_full columns in all
+int launch_init_tables(float *U, float *V, uint64_t vocab, uint32_t d, uint32_t ld, uint32_t d_full,
+                       uint32_t col_lo, uint64_t seed, cudaStream_t s);
 
 int launch_compact(const int32_t *tokens, uint64_t n, const SampleTables &tab, uint32_t vocab,
                    uint32_t k0, uint32_t k1, uint32_t step_lo, const Scratch &sc, DevState *st,
@@ -92,6 +101,13 @@ int launch_hogwild(const StepParams &p, uint32_t rows_in_flight, uint32_t blocks
                    cudaStream_t s);
 int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t blocks_per_sm, int sms,
                     cudaStream_t s);
+// passes 2, 2b and 3 of the snapshot plan alone: G and DU are already filled
+int launch_snapshot_apply(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s);
+
+int launch_shard_dots(const StepParams &p, const ShardPeers &peers, int sms, cudaStream_t s);
+int launch_shard_coefficients(const float *F, float *G, unsigned long long total, uint32_t n1p, float lr,
+                              int sms, cudaStream_t s);
+int launch_shard_du(const StepParams &p, int sms, cudaStream_t s);
 
 int launch_partial_dots(const float *U, const float *V, uint32_t vocab, uint32_t ld,
                         const int32_t *pairs, uint64_t m, uint32_t col_lo, uint32_t col_hi,

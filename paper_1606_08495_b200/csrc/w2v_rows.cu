@@ -10,16 +10,18 @@ namespace w2v {
 
 // U[w][4 j4 .. 4 j4 + 3] = ((r >> 8) 2^-24 - 0.5) / d, r the four words of
 // Philox(seed; w, j4, 0, 0).  Padding columns between d and the row stride are zeroed.
+// A column shard stores columns col4_off*4 .. of vectors of d_full columns: the value of a
+// column does not depend on which shard holds it.
 __global__ void __launch_bounds__(256)
-init_u_kernel(float4 *__restrict__ U4, uint64_t total4, uint32_t d4, uint32_t ld4, float d, uint32_t k0,
-              uint32_t k1)
+init_u_kernel(float4 *__restrict__ U4, uint64_t total4, uint32_t d4, uint32_t ld4, uint32_t col4_off, float d,
+              uint32_t k0, uint32_t k1)
 {
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
     for (uint64_t idx = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total4; idx += stride) {
         const uint32_t row = (uint32_t)(idx / ld4), j4 = (uint32_t)(idx % ld4);
         float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
         if (j4 < d4) {
-            const uint4 r = philox4x32_10(k0, k1, row, j4, kPurInit, 0);
+            const uint4 r = philox4x32_10(k0, k1, row, j4 + col4_off, kPurInit, 0);
             const float s = 1.0f / 16777216.0f;
             o.x = ((float)(r.x >> 8) * s - 0.5f) / d;
             o.y = ((float)(r.y >> 8) * s - 0.5f) / d;
@@ -30,14 +32,14 @@ init_u_kernel(float4 *__restrict__ U4, uint64_t total4, uint32_t d4, uint32_t ld
     }
 }
 
-int launch_init_tables(float *U, float *V, uint64_t vocab, uint32_t d, uint32_t ld, uint64_t seed,
-                       cudaStream_t s)
+int launch_init_tables(float *U, float *V, uint64_t vocab, uint32_t d, uint32_t ld, uint32_t d_full,
+                       uint32_t col_lo, uint64_t seed, cudaStream_t s)
 {
     const uint64_t total4 = vocab * (ld / 4);
     const uint64_t want = (total4 + 255) / 256;
     const int grid = (int)(want < 148ull * 32 ? (want ? want : 1) : 148ull * 32);
-    init_u_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<float4 *>(U), total4, d / 4, ld / 4, (float)d,
-                                       (uint32_t)seed, (uint32_t)(seed >> 32));
+    init_u_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<float4 *>(U), total4, d / 4, ld / 4, col_lo / 4,
+                                       (float)d_full, (uint32_t)seed, (uint32_t)(seed >> 32));
     if (cudaGetLastError() != cudaSuccess) return -1;
     if (cudaMemsetAsync(V, 0, vocab * (uint64_t)ld * sizeof(float), s) != cudaSuccess) return -1;
     return 1;

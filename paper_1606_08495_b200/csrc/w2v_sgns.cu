@@ -302,12 +302,9 @@ int launch_hogwild(const StepParams &p, uint32_t rows_in_flight, uint32_t blocks
     return 1;
 }
 
-int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t blocks_per_sm, int sms,
-                    cudaStream_t s)
+int launch_snapshot_apply(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s)
 {
     const int vpl = (int)((p.d4 + 31) / 32);
-    const int tb = pick_tb(rows_in_flight, vpl, p.negatives);
-    W2V_FOR_VPL(snap_dots(p, blocks_per_sm, sms, s))
     switch (vpl) {
         case 1: snap_adjust_v<1>(p, blocks_per_sm, sms, s); break;
         case 2: snap_adjust_v<2>(p, blocks_per_sm, sms, s); break;
@@ -318,7 +315,7 @@ int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t block
         case 7: snap_adjust_v<7>(p, blocks_per_sm, sms, s); break;
         default: snap_adjust_v<8>(p, blocks_per_sm, sms, s); break;
     }
-    int launched = 3;
+    int launched = 2;
     if (p.hot_rows) {
         const uint64_t want = ((uint64_t)p.hot_rows * 4u * p.d4 + kBlock - 1) / kBlock;
         const int grid = (int)(want < (uint64_t)sms * 8 ? want : (uint64_t)sms * 8);
@@ -331,6 +328,17 @@ int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t block
     }
     if (cudaGetLastError() != cudaSuccess) return -1;
     return launched;
+}
+
+int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t blocks_per_sm, int sms,
+                    cudaStream_t s)
+{
+    const int vpl = (int)((p.d4 + 31) / 32);
+    const int tb = pick_tb(rows_in_flight, vpl, p.negatives);
+    W2V_FOR_VPL(snap_dots(p, blocks_per_sm, sms, s))
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    const int k = launch_snapshot_apply(p, blocks_per_sm, sms, s);
+    return k < 0 ? -1 : 1 + k;
 }
 
 }  // namespace w2v
