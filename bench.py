@@ -338,6 +338,90 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def algorithmic_bytes_sharded(d, centres, pairs, negatives, shards):
+    """Column-sharded step, summed over the shards (their slice widths add up to d): dotprod reads
+    C + T slice rows; adjust reads T rows for the centre sums, writes and re-reads C scratch rows,
+    reads C rows and read-modify-writes T rows, then read-modify-writes C rows.  Each shard also adds
+    its T partial dots into `shards` arrays (8 B each) and moves 16 B per target of dots and
+    coefficients."""
+    T = pairs * (1 + negatives)
+    return 4 * d * (4 * T + 6 * centres) + (8 * shards * shards + 16 * shards) * T
+
+
+def run_sharded(args):
+    """The paper's column partition: `--shards S` shards of one model, here all on one GPU, one after
+    another (the step a rank of an S-GPU run executes is one shard's share of this)."""
+    import torch
+
+    from paper_1606_08495_b200 import binding
+    from paper_1606_08495_b200.sharded import LocalShards
+
+    if int(os.environ.get("WORLD_SIZE", "1")) != 1:
+        raise SystemExit("--mode sharded times the shards of one model on one GPU; run it without torchrun")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    S = args.shards
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    name = args.workload
+    if not name:
+        for cand in ["large", "sponsored", "medium", "small", "tiny"]:
+            c = corpus.CONFIGS[cand]
+            if 2 * c["vocab"] * c["d"] * 4 + 12 * S * c["vocab"] + 8 * (1 << 30) < free_b:
+                name = cand
+                break
+    cfg = corpus.CONFIGS[name]
+    cp = corpus.Corpus(cfg)
+    W, N, lr, d = cfg["window"], cfg["negatives"], cfg["lr"], cfg["d"]
+    K, Wu = args.steps, args.warmup
+    model = LocalShards(cfg["vocab"], d, 1, S, device=dev)
+    model.build_alias(cp.counts, cfg["subsample_t"])
+    chunks = [torch.from_numpy(cp.chunk(i)).to(dev) for i in range(Wu + K)]
+    for i in range(Wu):
+        model.step(chunks[i], W, N, lr)
+    model.sync()
+    for m in model.models:
+        binding.w2v_profile_enable(m.h, True)
+    launches0 = model.launch_count()
+    sampler = ClockSampler(physical_gpu_index(0))
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    sampler.start()
+    ev0.record()
+    centres, pairs = [], []
+    for i in range(Wu, Wu + K):
+        st = model.step(chunks[i], W, N, lr)
+        centres.append(st["centres"]); pairs.append(st["pairs"])
+    ev1.record()
+    torch.cuda.synchronize(dev)
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1)
+    launches = model.launch_count() - launches0
+    per_shard_ms = [binding.w2v_profile_read(m.h)[0] for m in model.models]
+    kernel_ms = sum(per_shard_ms)
+    tot_pairs = float(sum(pairs))
+    tot_bytes = float(sum(algorithmic_bytes_sharded(d, c, p, N, S) for c, p in zip(centres, pairs)))
+    peak, peak_kind = measured_peak()
+    achieved = tot_bytes / (kernel_ms * 1e-3) / 1e9 if kernel_ms > 0 else 0.0
+    line = {
+        "metric": METRIC, "value": tot_pairs / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": Wu,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": name, "vocab": cfg["vocab"], "d": d, "window": W, "negatives": N,
+                   "mode": "sharded", "shards": S, "columns": model.columns,
+                   "parallelism": f"{S} column shards run one after another on 1 gpu",
+                   "pairs_per_step": tot_pairs / K,
+                   "slowest_shard_ms_per_step": max(per_shard_ms) / K,
+                   "pairs_per_sec_if_each_shard_had_its_own_gpu_exchange_excluded": tot_pairs / (max(per_shard_ms) * 1e-3)},
+        "clocks": clocks, "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "kernel": "shard_dots + coefficients + shard_du + snapshot passes 2-3",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "algorithmic_bytes_per_launch": tot_bytes / K,
+                     "kernel_ms_per_launch": kernel_ms / K, "traffic": None},
+    }
+    print(json.dumps(line), flush=True)
+    model.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -353,13 +437,17 @@ def main():
     ap.add_argument("--cpu-words", type=int, default=150_000, help="word tokens in the cpu_baseline sample")
     ap.add_argument("--ref-words", type=int, default=20_000, help="word tokens per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--mode", choices=["hogwild", "snapshot"], default="hogwild",
-                    help="update mode of the timed steps (the headline number is hogwild)")
+    ap.add_argument("--mode", choices=["hogwild", "snapshot", "sharded"], default="hogwild",
+                    help="update mode of the timed steps (the headline number is hogwild); sharded = the "
+                         "paper's column partition, --shards slices of one model on one GPU")
+    ap.add_argument("--shards", type=int, default=8)
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         print("note: fewer than 3 warm-up steps; not a valid timing", file=sys.stderr)
     if args.impl == "reference":
         run_reference(args)
+    elif args.mode == "sharded":
+        run_sharded(args)
     else:
         run_gpu(args)
 
