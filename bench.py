@@ -223,7 +223,7 @@ def run_gpu(args):
     K, Wu = args.steps, args.warmup
     mode = binding.MODE_HOGWILD if args.mode == "hogwild" else binding.MODE_SNAPSHOT
 
-    row_stride = row_stride_for(d, args.row_stride)
+    row_stride = d if args.dense_rows else row_stride_for(d, args.row_stride)
     model = binding.W2V(cfg["vocab"], d, seed=1, device=dev, row_stride=row_stride)
     model.build_alias(cp.counts, cfg["subsample_t"])
     model.set_tuning(args.rows_in_flight, args.blocks_per_sm)
@@ -373,7 +373,11 @@ def run_sharded(args):
     cp = corpus.Corpus(cfg)
     W, N, lr, d = cfg["window"], cfg["negatives"], cfg["lr"], cfg["d"]
     K, Wu = args.steps, args.warmup
-    model = LocalShards(cfg["vocab"], d, 1, S, device=dev)
+    from paper_1606_08495_b200.sharded import shard_columns
+    widest = max(hi - lo for lo, hi in shard_columns(d, S))
+    aligned = (not args.dense_rows and
+               2 * cfg["vocab"] * binding.aligned_row_stride(widest) * 4 * S + 12 * S * cfg["vocab"] + 8 * (1 << 30) < free_b)
+    model = LocalShards(cfg["vocab"], d, 1, S, device=dev, aligned_rows=aligned)
     model.build_alias(cp.counts, cfg["subsample_t"])
     chunks = [torch.from_numpy(cp.chunk(i)).to(dev) for i in range(Wu + K)]
     for i in range(Wu):
@@ -408,6 +412,7 @@ def run_sharded(args):
         "data": "synthetic",
         "config": {"workload": name, "vocab": cfg["vocab"], "d": d, "window": W, "negatives": N,
                    "mode": "sharded", "shards": S, "columns": model.columns,
+                   "rows": "on 128-byte boundaries" if aligned else "dense",
                    "parallelism": f"{S} column shards run one after another on 1 gpu",
                    "pairs_per_step": tot_pairs / K,
                    "slowest_shard_ms_per_step": max(per_shard_ms) / K,
@@ -441,6 +446,7 @@ def main():
                     help="update mode of the timed steps (the headline number is hogwild); sharded = the "
                          "paper's column partition, --shards slices of one model on one GPU")
     ap.add_argument("--shards", type=int, default=8)
+    ap.add_argument("--dense-rows", action="store_true", help="no padding between table rows")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         print("note: fewer than 3 warm-up steps; not a valid timing", file=sys.stderr)

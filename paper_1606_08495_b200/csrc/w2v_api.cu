@@ -519,7 +519,7 @@ int32_t w2v_shard_adjust(w2v_handle *h, const float *F, float lr)
         if ((rc = profile_mark(h)) != W2V_OK) return rc;
         int k = launch_shard_coefficients(F, h->G, targets, h->pend_negatives + 1, lr, h->sms, h->stream);
         int k2 = k < 0 ? -1 : launch_shard_du(p, h->sms, h->stream);
-        int k3 = k2 < 0 ? -1 : launch_snapshot_apply(p, h->blocks_per_sm, h->sms, h->stream);
+        int k3 = k2 < 0 ? -1 : launch_shard_apply(p, h->blocks_per_sm, h->sms, h->stream);
         if (k3 < 0) return fail(h, W2V_ERR_CUDA, "adjust launch", cudaGetLastError());
         h->launches += (uint64_t)(k + k2 + k3);
         if (h->profiling) h->prof_launches += (uint64_t)(k + k2 + k3);

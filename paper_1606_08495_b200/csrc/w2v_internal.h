@@ -103,6 +103,10 @@ int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t block
                     cudaStream_t s);
 // passes 2, 2b and 3 of the snapshot plan alone: G and DU are already filled
 int launch_snapshot_apply(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s);
+// passes 2b and 3 alone: the fp64 sums of the most-hit rows and the centre sums are applied
+int launch_snapshot_tail(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s);
+// pass 2 (and the tail) for a column shard: narrow slices put several rows side by side in a warp
+int launch_shard_apply(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s);
 
 int launch_shard_dots(const StepParams &p, const ShardPeers &peers, int sms, cudaStream_t s);
 int launch_shard_coefficients(const float *F, float *G, unsigned long long total, uint32_t n1p, float lr,

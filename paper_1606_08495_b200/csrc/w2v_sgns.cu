@@ -315,7 +315,14 @@ int launch_snapshot_apply(const StepParams &p, uint32_t blocks_per_sm, int sms, 
         case 7: snap_adjust_v<7>(p, blocks_per_sm, sms, s); break;
         default: snap_adjust_v<8>(p, blocks_per_sm, sms, s); break;
     }
-    int launched = 2;
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    const int k = launch_snapshot_tail(p, blocks_per_sm, sms, s);
+    return k < 0 ? -1 : 1 + k;
+}
+
+int launch_snapshot_tail(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s)
+{
+    int launched = 1;
     if (p.hot_rows) {
         const uint64_t want = ((uint64_t)p.hot_rows * 4u * p.d4 + kBlock - 1) / kBlock;
         const int grid = (int)(want < (uint64_t)sms * 8 ? want : (uint64_t)sms * 8);
