@@ -257,6 +257,18 @@ int32_t w2v_write_rows(w2v_handle *h, uint32_t which, const int64_t *ids, uint64
 int32_t w2v_set_step(w2v_handle *h, uint64_t step_id);
 int32_t w2v_get_step(w2v_handle *h, uint64_t *step_id);
 
+/*
+ * Interleaved minibatch formation (Section 5.1, last paragraph: the input words of a minibatch
+ * should be well separated in the corpus, ideally in different sentences).  After this call only
+ * the tokens whose index in the chunk is congruent to phase modulo stride act as input (centre)
+ * words of w2v_sgns_step, w2v_sample_pairs and w2v_shard_dots; contexts still come from the whole
+ * sentence.  Sub-sampling, radii and negatives do not depend on the setting, so the `stride` steps
+ * phase = 0..stride-1 over the same chunk WITH THE SAME STEP NUMBER (w2v_set_step before each)
+ * use every input word of the chunk exactly once.  stride = 1 (the default) uses them all.
+ * Errors: W2V_ERR_ARG unless stride >= 1 and phase < stride.
+ */
+int32_t w2v_set_interleave(w2v_handle *h, uint32_t phase, uint32_t stride);
+
 /* Device pointers of the two tables (caller's or library-owned). */
 int32_t w2v_get_table_ptrs(w2v_handle *h, float **U, float **V);
 

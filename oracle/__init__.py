@@ -41,6 +41,7 @@ def _load():
     L.orc_create.argtypes = [u64, u32, u64, C.c_int]
     L.orc_destroy.argtypes = [vp]
     L.orc_set_step.argtypes = [vp, u64]
+    L.orc_set_interleave.argtypes = [vp, u32, u32]
     L.orc_get_step.restype = u64
     L.orc_get_step.argtypes = [vp]
     L.orc_init_row.argtypes = [vp, u64, vp]
@@ -104,6 +105,10 @@ class Oracle:
 
     def get_step(self):
         return int(self.L.orc_get_step(self.h))
+
+    def set_interleave(self, phase, stride):
+        if self.L.orc_set_interleave(self.h, int(phase), int(stride)) != 0:
+            raise ValueError("need stride >= 1 and phase < stride")
 
     def init_row(self, row):
         out = np.empty(self.d, dtype=np.float32)

@@ -36,6 +36,8 @@
  *   orc_step mode 1    the sequential limit of the lock-free operation of
  *                      Section 5.1: targets one after another, every read sees
  *                      every earlier write.
+ *   orc_set_interleave interleaved minibatch formation (Section 5.1, last
+ *                      paragraph): the input words of one call are a stride apart.
  *   orc_partial_dots   u_s(w_I) v_s(w_O)^T of Algorithm 1 for one column slice.
  *   orc_loss           minus Eq. (1) restricted to a chunk, per positive pair.
  *
@@ -168,6 +170,7 @@ typedef struct orc {
     uint32_t d;
     uint64_t seed;
     uint64_t step_id;
+    uint32_t il_phase, il_stride;   /* interleaved minibatches: centres with index % stride == phase */
     rowstore U, V;
     int have_tables;
     uint32_t *thr;     /* alias acceptance thresholds (units of 2^-32) */
@@ -261,6 +264,17 @@ void orc_destroy(orc *h)
     free(h);
 }
 void orc_set_step(orc *h, uint64_t s) { h->step_id = s; }
+/* Interleaved minibatch formation (Section 5.1, last paragraph): of the chunk's kept tokens only
+ * those whose index in the chunk is congruent to phase modulo stride act as input (centre) words;
+ * their contexts are still taken from the whole sentence.  The `stride` calls phase = 0..stride-1
+ * with the same step number cover every input word of the chunk exactly once, and the input words
+ * of one call are at least `stride` tokens apart. */
+int orc_set_interleave(orc *h, uint32_t phase, uint32_t stride)
+{
+    if (stride < 1 || phase >= stride) return -1;
+    h->il_phase = phase; h->il_stride = stride;
+    return 0;
+}
 uint64_t orc_get_step(const orc *h) { return h->step_id; }
 
 void orc_init_row(const orc *h, uint64_t row, float *out) { init_row_values(h, row, out); }
@@ -417,6 +431,7 @@ static void sample_chunk(orc *h, const int32_t *tokens, uint64_t n, uint32_t W, 
     uint64_t pair_index = 0;
     for (uint64_t q = 0; q < nk; ++q) {
         uint32_t r[4];
+        if (h->il_stride > 1 && h->cidx[q] % h->il_stride != h->il_phase) continue;
         philox4x32_10(k0, k1, h->cidx[q], step_lo, PUR_RADIUS, 0, r);
         int64_t b = 1 + (int64_t)(((uint64_t)r[0] * (uint64_t)W) >> 32);
         int had = 0;

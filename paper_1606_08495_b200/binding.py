@@ -21,7 +21,7 @@ TABLE_U, TABLE_V = 0, 1
 
 EXPORTS = (
     "w2v_create", "w2v_create_strided", "w2v_create_shard", "w2v_shard_dots", "w2v_shard_adjust",
-    "w2v_get_row_stride", "w2v_destroy", "w2v_build_alias", "w2v_get_tables", "w2v_sgns_step",
+    "w2v_get_row_stride", "w2v_set_interleave", "w2v_destroy", "w2v_build_alias", "w2v_get_tables", "w2v_sgns_step",
     "w2v_sgns_step_host", "w2v_sample_pairs", "w2v_partial_dots", "w2v_read_rows", "w2v_write_rows",
     "w2v_set_step", "w2v_get_step", "w2v_get_table_ptrs", "w2v_sync", "w2v_profile_enable",
     "w2v_profile_read", "w2v_get_launch_count", "w2v_set_tuning", "w2v_last_error",
@@ -81,6 +81,7 @@ def load():
         "w2v_read_rows": [vp, u32, vp, u64, vp],
         "w2v_write_rows": [vp, u32, vp, u64, vp],
         "w2v_set_step": [vp, u64],
+        "w2v_set_interleave": [vp, u32, u32],
         "w2v_get_step": [vp, C.POINTER(u64)],
         "w2v_get_table_ptrs": [vp, C.POINTER(vp), C.POINTER(vp)],
         "w2v_sync": [vp],
@@ -222,6 +223,10 @@ def w2v_set_step(h, step_id):
     return _check(h, load().w2v_set_step(h, int(step_id)))
 
 
+def w2v_set_interleave(h, phase, stride):
+    return _check(h, load().w2v_set_interleave(h, int(phase), int(stride)))
+
+
 def w2v_get_step(h):
     s = C.c_uint64(0)
     _check(h, load().w2v_get_step(h, C.byref(s)))
@@ -355,6 +360,9 @@ class W2V:
 
     def get_step(self):
         return w2v_get_step(self.h)
+
+    def set_interleave(self, phase, stride):
+        w2v_set_interleave(self.h, phase, stride)
 
     def sync(self):
         w2v_sync(self.h)

@@ -24,6 +24,7 @@ struct w2v_handle {
     uint64_t pend_n = 0, pend_pairs = 0;
     uint64_t seed = 0;
     uint64_t step_id = 0;
+    uint32_t il_phase = 0, il_stride = 1;   // interleaved minibatches: which tokens are input words
     int device = 0;
     int sms = 148;
     cudaStream_t stream = nullptr;
@@ -161,7 +162,7 @@ int32_t enqueue_sampling(w2v_handle *h, const int32_t *tokens, uint64_t n, uint3
     int k = launch_compact(tokens, n, tab, (uint32_t)h->vocab, k0, k1, step_lo, h->sc, h->st, h->stream);
     if (k < 0) return fail(h, W2V_ERR_CUDA, "compaction launch", cudaGetLastError());
     h->launches += (uint64_t)k;
-    k = launch_windows(n, window, k0, k1, step_lo, h->sc, h->st, h->stream);
+    k = launch_windows(n, window, k0, k1, step_lo, h->il_phase, h->il_stride, h->sc, h->st, h->stream);
     if (k < 0) return fail(h, W2V_ERR_CUDA, "window launch", cudaGetLastError());
     h->launches += (uint64_t)k;
     return W2V_OK;
@@ -576,6 +577,15 @@ int32_t w2v_set_step(w2v_handle *h, uint64_t step_id)
     return W2V_OK;
 }
 
+int32_t w2v_set_interleave(w2v_handle *h, uint32_t phase, uint32_t stride)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (stride < 1 || phase >= stride) return fail(h, W2V_ERR_ARG, "need stride >= 1 and phase < stride");
+    h->il_phase = phase; h->il_stride = stride;
+    h->shard_pending = false;
+    return W2V_OK;
+}
+
 int32_t w2v_get_step(w2v_handle *h, uint64_t *step_id)
 {
     if (!h || !step_id) return W2V_ERR_ARG;
@@ -746,7 +756,7 @@ extern "C" int32_t w2v_sample_pairs_noalloc(w2v_handle *h, const int32_t *tokens
     int k = launch_compact(tokens, n, tab, (uint32_t)h->vocab, k0, k1, step_lo, sc, st, h->stream);
     if (k < 0) return fail(h, W2V_ERR_CUDA, "compaction launch", cudaGetLastError());
     h->launches += (uint64_t)k;
-    k = launch_windows(n, window, k0, k1, step_lo, sc, st, h->stream);
+    k = launch_windows(n, window, k0, k1, step_lo, h->il_phase, h->il_stride, sc, st, h->stream);
     if (k < 0) return fail(h, W2V_ERR_CUDA, "window launch", cudaGetLastError());
     h->launches += (uint64_t)k;
     k = launch_pair_offsets(n, sc, st, h->stream);

@@ -92,7 +92,7 @@ int launch_compact(const int32_t *tokens, uint64_t n, const SampleTables &tab, u
                    uint32_t k0, uint32_t k1, uint32_t step_lo, const Scratch &sc, DevState *st,
                    cudaStream_t s);
 int launch_windows(uint64_t n, uint32_t window, uint32_t k0, uint32_t k1, uint32_t step_lo,
-                   const Scratch &sc, DevState *st, cudaStream_t s);
+                   uint32_t il_phase, uint32_t il_stride, const Scratch &sc, DevState *st, cudaStream_t s);
 int launch_pair_offsets(uint64_t n, const Scratch &sc, DevState *st, cudaStream_t s);
 int launch_emit_pairs(const StepParams &p, int32_t *centre, int32_t *context, int32_t *negs,
                       uint64_t cap, int grid, cudaStream_t s);

@@ -109,14 +109,18 @@ scatter_kernel(const int32_t *__restrict__ tokens, uint64_t n, const uint8_t *__
 // ---- windows: radius b in 1..window per centre, clipped to its sentence ------------
 __global__ void __launch_bounds__(256)
 window_kernel(const uint32_t *__restrict__ cidx, const uint32_t *__restrict__ csent, uint32_t window,
-              uint32_t k0, uint32_t k1, uint32_t step_lo, uint16_t *__restrict__ win, DevState *st)
+              uint32_t k0, uint32_t k1, uint32_t step_lo, uint32_t il_phase, uint32_t il_stride,
+              uint16_t *__restrict__ win, DevState *st)
 {
     const uint32_t nk = (uint32_t)st->n_kept;
     const uint32_t q = blockIdx.x * blockDim.x + threadIdx.x;
     uint32_t cnt = 0;
     if (q < nk) {
-        const uint32_t r = philox4x32_10(k0, k1, cidx[q], step_lo, kPurRadius, 0).x;
-        const uint32_t b = 1u + __umulhi(r, window);
+        const uint32_t i = cidx[q];
+        const uint32_t r = philox4x32_10(k0, k1, i, step_lo, kPurRadius, 0).x;
+        // interleaved minibatches: only tokens with index = phase (mod stride) are input words of
+        // this call; the others keep an empty window and serve as contexts only
+        const uint32_t b = (il_stride > 1u && i % il_stride != il_phase) ? 0u : 1u + __umulhi(r, window);
         const uint32_t sid = csent[q];
         uint32_t left = 0, right = 0;
         while (left < b && q >= left + 1u && csent[q - left - 1u] == sid) ++left;
@@ -246,11 +250,12 @@ int launch_compact(const int32_t *tokens, uint64_t n, const SampleTables &tab, u
 }
 
 int launch_windows(uint64_t n, uint32_t window, uint32_t k0, uint32_t k1, uint32_t step_lo,
-                   const Scratch &sc, DevState *st, cudaStream_t s)
+                   uint32_t il_phase, uint32_t il_stride, const Scratch &sc, DevState *st, cudaStream_t s)
 {
     if (n == 0) return 0;
     const uint32_t nb = (uint32_t)((n + 255) / 256);
-    window_kernel<<<nb, 256, 0, s>>>(sc.cidx, sc.csent, window, k0, k1, step_lo, sc.win, st);
+    window_kernel<<<nb, 256, 0, s>>>(sc.cidx, sc.csent, window, k0, k1, step_lo, il_phase, il_stride, sc.win,
+                                     st);
     if (cudaGetLastError() != cudaSuccess) return -1;
     return 1;
 }

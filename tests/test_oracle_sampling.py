@@ -169,3 +169,47 @@ def test_empty_and_degenerate_chunks():
     for toks in ([], [-1, -1, -1], [7], [7, -1, 8, -1]):
         c, x, n = o.sample_pairs(np.asarray(toks, dtype=np.int32), 2, 3)
         assert len(c) == 0 and len(x) == 0 and n.shape[0] == 0
+
+
+# ---- interleaved minibatch formation (Section 5.1, last paragraph) ----
+def test_interleaved_phases_partition_the_pairs_of_the_chunk():
+    # same step number, phases 0..stride-1: every input word of the chunk is used exactly once, with
+    # the same contexts and the same negatives as in the whole-chunk call
+    rng = np.random.default_rng(8)
+    V = 300
+    counts = rng.integers(1, 2000, size=V).astype(np.uint64)
+    o = make(V=V, counts=counts, t=5e-3, seed=12)
+    toks = []
+    for _ in range(40):
+        toks += list(rng.integers(0, V, size=rng.integers(1, 30))) + [-1]
+    whole = o.sample_pairs(toks, window=4, negatives=3)
+    whole_rows = np.concatenate([whole[0][:, None], whole[1][:, None], whole[2]], axis=1)
+    for stride in (1, 2, 7, 64):
+        parts = []
+        for phase in range(stride):
+            o.set_interleave(phase, stride)
+            c, x, n = o.sample_pairs(toks, window=4, negatives=3)
+            parts.append(np.concatenate([c[:, None], x[:, None], n], axis=1))
+        got = np.concatenate(parts, axis=0)
+        assert len(got) == len(whole_rows)
+        assert np.array_equal(got[np.lexsort(got.T[::-1])], whole_rows[np.lexsort(whole_rows.T[::-1])])
+    o.set_interleave(0, 1)
+
+
+def test_interleaved_input_words_are_a_stride_apart():
+    # distinct words, nothing dropped: a centre word identifies its position in the chunk
+    V = 500
+    o = make(V=V, counts=np.full(V, 5, dtype=np.uint64), t=0.0)
+    toks = np.arange(V, dtype=np.int32)                      # one long sentence
+    for stride, phase in ((5, 0), (5, 3), (50, 49)):
+        o.set_interleave(phase, stride)
+        c, x, _ = o.sample_pairs(toks, window=3, negatives=1)
+        assert len(c) > 0 and np.all(c % stride == phase)
+        assert np.all(np.abs(x - c) <= 3) and np.all(x != c)   # contexts still come from the whole sentence
+    o.set_interleave(0, 1)
+    for bad in ((1, 1), (5, 5), (0, 0)):
+        try:
+            o.set_interleave(*bad)
+            raise AssertionError("accepted phase >= stride")
+        except ValueError:
+            pass
