@@ -261,8 +261,13 @@ def run_gpu(args):
     barrier(); torch.cuda.synchronize(dev)
     sampler.start()
     ev0.record()
+    IL = max(1, args.interleave)
     for i in range(Wu, Wu + K):
-        binding.w2v_sgns_step(model.h, dev_chunks[i], dev_chunks[i].numel(), W, N, lr, mode, None)
+        for phase in range(IL):                       # IL > 1: interleaved minibatches, one step number
+            if IL > 1:
+                binding.w2v_set_step(model.h, i)
+                binding.w2v_set_interleave(model.h, phase, IL)
+            binding.w2v_sgns_step(model.h, dev_chunks[i], dev_chunks[i].numel(), W, N, lr, mode, None)
     ev1.record()
     torch.cuda.synchronize(dev); barrier()
     clocks = sampler.stop()
@@ -280,9 +285,13 @@ def run_gpu(args):
     ev2.record()
     for i in range(Wu + K, Wu + 2 * K):
         t = host_chunks[i]
-        binding.w2v_sgns_step_host(model.h, t, t.numel(), W, N, lr, mode, st)
-        e2e_pairs += st.pairs
-        h2d += 4 * t.numel(); d2h += 64
+        for phase in range(IL):
+            if IL > 1:
+                binding.w2v_set_step(model.h, i)
+                binding.w2v_set_interleave(model.h, phase, IL)
+            binding.w2v_sgns_step_host(model.h, t, t.numel(), W, N, lr, mode, st)
+            e2e_pairs += st.pairs
+            h2d += 4 * t.numel(); d2h += 64
     ev3.record()
     torch.cuda.synchronize(dev); barrier()
     e2e_ms = ev2.elapsed_time(ev3)
@@ -304,7 +313,7 @@ def run_gpu(args):
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": name, "vocab": cfg["vocab"], "d": d, "window": W, "negatives": N,
                        "subsample_t": cfg["subsample_t"], "tokens_per_step": int(dev_chunks[0].numel()),
-                       "mode": args.mode, "row_stride_floats": row_stride, "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
+                       "mode": args.mode, "row_stride_floats": row_stride, "interleave": IL, "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
                        "l2": "tables and gathers far larger than L2 (random rows of %.1f GB)" % (2 * cfg["vocab"] * d * 4 / 1e9)
                              if 2 * cfg["vocab"] * d * 4 > 4 * 126e6 else "tables fit in L2; no flush between steps",
                        "pairs_per_step": tot_pairs / K, "centres_per_step": sum(centres) / K,
@@ -446,6 +455,9 @@ def main():
                     help="update mode of the timed steps (the headline number is hogwild); sharded = the "
                          "paper's column partition, --shards slices of one model on one GPU")
     ap.add_argument("--shards", type=int, default=8)
+    ap.add_argument("--interleave", type=int, default=1,
+                    help="visit every chunk this many times, each time with 1/this of its input words "
+                         "(interleaved minibatch formation)")
     ap.add_argument("--dense-rows", action="store_true", help="no padding between table rows")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":

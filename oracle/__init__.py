@@ -59,6 +59,12 @@ def _load():
     L.orc_loss.argtypes = [vp, vp, u64, u32, u32, u64, vp, vp]
     L.orc_loss_pairs.restype = C.c_double
     L.orc_loss_pairs.argtypes = [vp, vp, vp, vp, u64, u32]
+    L.orc_cbow_examples.argtypes = [vp, vp, u64, u32, u32, vp, vp, vp, vp, u64, u64, vp, vp]
+    L.orc_cbow_step.argtypes = [vp, vp, u64, u32, u32, C.c_double, u32]
+    L.orc_cbow_step_examples.argtypes = [vp, vp, vp, vp, vp, u64, u32, C.c_double, u32]
+    L.orc_cbow_loss.argtypes = [vp, vp, u64, u32, u32, u64, vp, vp]
+    L.orc_cbow_loss_examples.restype = C.c_double
+    L.orc_cbow_loss_examples.argtypes = [vp, vp, vp, vp, vp, u64, u32]
     L.orc_rows_resident.restype = u64
     L.orc_rows_resident.argtypes = [vp, u32]
     _lib = L
@@ -205,6 +211,62 @@ class Oracle:
         negs = _i32(negs).reshape(len(centre), -1)
         return float(self.L.orc_loss_pairs(self.h, centre.ctypes.data, context.ctypes.data,
                                            negs.ctypes.data, len(centre), negs.shape[1]))
+
+    # -- continuous bag of words -------------------------------------------
+    def cbow_examples(self, tokens, window, negatives):
+        """(centre[E], negs[E, N], ctx_off[E + 1], ctx[sum |C|]) of the chunk's examples."""
+        tokens = _i32(tokens)
+        n = len(tokens)
+        cap_ex, cap_ctx = max(1, n), max(1, n * 2 * window)
+        centre = np.empty(cap_ex, dtype=np.int32)
+        negs = np.empty((cap_ex, negatives), dtype=np.int32)
+        ctx_off = np.zeros(cap_ex + 1, dtype=np.uint64)
+        ctx = np.empty(cap_ctx, dtype=np.int32)
+        E, M = C.c_uint64(0), C.c_uint64(0)
+        rc = self.L.orc_cbow_examples(self.h, tokens.ctypes.data, n, window, negatives, centre.ctypes.data,
+                                      negs.ctypes.data, ctx_off.ctypes.data, ctx.ctypes.data, cap_ex, cap_ctx,
+                                      C.byref(E), C.byref(M))
+        if rc != 0:
+            raise ValueError("orc_cbow_examples rejected its arguments")
+        E, M = int(E.value), int(M.value)
+        return centre[:E].copy(), negs[:E].copy(), ctx_off[:E + 1].copy(), ctx[:M].copy()
+
+    def cbow_step(self, tokens, window, negatives, lr, mode):
+        tokens = _i32(tokens)
+        rc = self.L.orc_cbow_step(self.h, tokens.ctypes.data, len(tokens), window, negatives, float(lr), mode)
+        if rc != 0:
+            raise ValueError("orc_cbow_step rejected its arguments")
+        return self.stats()
+
+    @staticmethod
+    def _examples(centre, negs, ctx_off, ctx):
+        centre = _i32(centre)
+        negs = _i32(negs).reshape(len(centre), -1)
+        ctx_off = np.ascontiguousarray(ctx_off, dtype=np.uint64)
+        ctx = _i32(ctx)
+        assert len(ctx_off) == len(centre) + 1 and int(ctx_off[-1]) == len(ctx)
+        return centre, negs, ctx_off, ctx
+
+    def cbow_step_examples(self, centre, negs, ctx_off, ctx, lr, mode):
+        centre, negs, ctx_off, ctx = self._examples(centre, negs, ctx_off, ctx)
+        rc = self.L.orc_cbow_step_examples(self.h, centre.ctypes.data, negs.ctypes.data, ctx_off.ctypes.data,
+                                           ctx.ctypes.data, len(centre), negs.shape[1], float(lr), mode)
+        assert rc == 0
+
+    def cbow_loss(self, tokens, window, negatives, step_id):
+        """(sum of -log-likelihood terms over the chunk's examples, number of examples)."""
+        tokens = _i32(tokens)
+        s, E = C.c_double(0.0), C.c_uint64(0)
+        rc = self.L.orc_cbow_loss(self.h, tokens.ctypes.data, len(tokens), window, negatives, int(step_id),
+                                  C.byref(s), C.byref(E))
+        assert rc == 0
+        return s.value, int(E.value)
+
+    def cbow_loss_examples(self, centre, negs, ctx_off, ctx):
+        centre, negs, ctx_off, ctx = self._examples(centre, negs, ctx_off, ctx)
+        return float(self.L.orc_cbow_loss_examples(self.h, centre.ctypes.data, negs.ctypes.data,
+                                                   ctx_off.ctypes.data, ctx.ctypes.data, len(centre),
+                                                   negs.shape[1]))
 
     def rows_resident(self, which):
         return int(self.L.orc_rows_resident(self.h, which))

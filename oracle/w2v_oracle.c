@@ -38,6 +38,10 @@
  *                      every earlier write.
  *   orc_set_interleave interleaved minibatch formation (Section 5.1, last
  *                      paragraph): the input words of one call are a stride apart.
+ *   orc_cbow_*         the continuous-bag-of-words variant (footnote to
+ *                      Section 5: "readily extends to CBOW"): the mean of the
+ *                      context words' input vectors predicts the centre word;
+ *                      same index sets, same two modes, exact gradient.
  *   orc_partial_dots   u_s(w_I) v_s(w_O)^T of Algorithm 1 for one column slice.
  *   orc_loss           minus Eq. (1) restricted to a chunk, per positive pair.
  *
@@ -46,7 +50,9 @@
  * c^0.75 / sum c^0.75; hand-computed 3-word examples; Eq. (4) against central
  * finite differences of Eq. (3); first-step closed form with V = 0; the
  * slice-sum identity of Algorithm 3 line "(F+,F-) <- sum_s"; hand-enumerated
- * windows.  No function here is "parity unpinned".
+ * windows; for CBOW: finite differences of its objective, the one-context case
+ * that reduces to a skip-gram pair, and the first-step closed form.
+ * No function here is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -666,6 +672,263 @@ double orc_loss_pairs(orc *h, const int32_t *centre, const int32_t *context, con
 {
     lossctx s = { h, 0.0 };
     for (uint64_t p = 0; p < P; ++p) loss_pair(&s, p, centre[p], context[p], negs + p * N, N);
+    return -s.sum;
+}
+
+/* ------------------------------------------------------------------ */
+/* Continuous bag of words (footnote to Section 5).                     */
+/* One example per kept token q that has at least one context word:     */
+/*   hbar = mean over the window's context words k of u(w_k)            */
+/*   targets: the centre word w_q (label 1) and N negatives != w_q      */
+/*   f = hbar . v(t),  g = lr (label - sigma(f))                        */
+/*   v(t) += g hbar;   every context word: u(w_k) += (sum_t g v(t)) / |C| */
+/* i.e. plus lr times the exact gradient of                             */
+/*   log s(hbar.v(w_q)) + sum_neg log s(-hbar.v(neg)).                  */
+/* Window and sub-sampling as in the skip-gram step; the negatives use  */
+/* the counter slot of offset 0 (slot = W), which no skip-gram pair has. */
+/* ------------------------------------------------------------------ */
+typedef void (*cbow_fn)(void *ctx, uint64_t ex_index, int32_t centre, const int32_t *contexts,
+                        uint32_t n_ctx, const int32_t *negs, uint32_t N);
+
+static void sample_chunk_cbow(orc *h, const int32_t *tokens, uint64_t n, uint32_t W, uint32_t N,
+                              uint64_t step_id, cbow_fn fn, void *ctx)
+{
+    uint32_t k0 = (uint32_t)h->seed;
+    uint32_t k1 = (uint32_t)(h->seed >> 32) ^ (uint32_t)(step_id >> 32);
+    uint32_t step_lo = (uint32_t)step_id;
+    if (h->cap_kept < n + 1) {
+        free(h->ctok); free(h->cidx); free(h->csent);
+        h->cap_kept = n + 1;
+        h->ctok = (int32_t *)malloc(h->cap_kept * sizeof(int32_t));
+        h->cidx = (uint32_t *)malloc(h->cap_kept * sizeof(uint32_t));
+        h->csent = (uint32_t *)malloc(h->cap_kept * sizeof(uint32_t));
+    }
+    h->st_tokens = n; h->st_kept = h->st_centres = h->st_pairs = 0;
+    h->st_draws = h->st_redraws = h->st_oov = 0;
+    uint64_t nk = 0;
+    uint32_t sent = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        int32_t w = tokens[i];
+        if (w == -1) { sent++; continue; }
+        if (w < 0 || (uint64_t)w >= h->vocab) { h->st_oov++; continue; }
+        uint32_t thr = h->keep_thr[w];
+        if (thr != 0xFFFFFFFFu) {
+            uint32_t r[4];
+            philox4x32_10(k0, k1, (uint32_t)i, step_lo, PUR_SUBSAMPLE, 0, r);
+            if (!(r[0] < thr)) continue;
+        }
+        h->ctok[nk] = w; h->cidx[nk] = (uint32_t)i; h->csent[nk] = sent;
+        nk++;
+    }
+    h->st_kept = nk;
+
+    int32_t negs[64], contexts[256];
+    uint64_t ex = 0;
+    for (uint64_t q = 0; q < nk; ++q) {
+        uint32_t r[4];
+        if (h->il_stride > 1 && h->cidx[q] % h->il_stride != h->il_phase) continue;
+        philox4x32_10(k0, k1, h->cidx[q], step_lo, PUR_RADIUS, 0, r);
+        int64_t b = 1 + (int64_t)(((uint64_t)r[0] * (uint64_t)W) >> 32);
+        uint32_t n_ctx = 0;
+        for (int64_t p = (int64_t)q - b; p <= (int64_t)q + b; ++p) {
+            if (p == (int64_t)q || p < 0 || p >= (int64_t)nk) continue;
+            if (h->csent[p] != h->csent[q]) continue;
+            contexts[n_ctx++] = h->ctok[p];
+        }
+        if (n_ctx == 0) continue;
+        int32_t wq = h->ctok[q];
+        for (uint32_t k = 0; k < N; ++k) {
+            uint32_t cand = 0;
+            int found = 0;
+            for (uint32_t a = 0; a < 16 && !found; ++a) {
+                philox4x32_10(k0, k1, h->cidx[q], step_lo, PUR_NEGATIVE | (W << 8), k | (a << 16), r);
+                cand = alias_draw(h, r);
+                h->st_draws++;
+                if (cand != (uint32_t)wq) found = 1; else h->st_redraws++;
+            }
+            if (!found) cand = (uint32_t)(((uint64_t)wq + 1) % h->vocab);
+            negs[k] = (int32_t)cand;
+        }
+        fn(ctx, ex++, wq, contexts, n_ctx, negs, N);
+        h->st_pairs += n_ctx;
+    }
+    h->st_centres = ex;
+}
+
+/* ---- the examples as lists: centre[E], negs[E*N], ctx_off[E+1], ctx[sum |C|] ---- */
+typedef struct {
+    int32_t *centre, *negs, *ctx; uint64_t *ctx_off; uint64_t cap_ex, cap_ctx, n_ctx;
+} cbowsink;
+static void sink_example(void *ctx, uint64_t ex, int32_t c, const int32_t *contexts, uint32_t n_ctx,
+                         const int32_t *negs, uint32_t N)
+{
+    cbowsink *s = (cbowsink *)ctx;
+    if (ex < s->cap_ex) {
+        s->centre[ex] = c;
+        for (uint32_t k = 0; k < N; ++k) s->negs[ex * N + k] = negs[k];
+        s->ctx_off[ex] = s->n_ctx;
+    }
+    for (uint32_t k = 0; k < n_ctx; ++k) {
+        if (s->n_ctx < s->cap_ctx) s->ctx[s->n_ctx] = contexts[k];
+        s->n_ctx++;
+    }
+    if (ex < s->cap_ex) s->ctx_off[ex + 1] = s->n_ctx;
+}
+int orc_cbow_examples(orc *h, const int32_t *tokens, uint64_t n, uint32_t W, uint32_t N,
+                      int32_t *centre, int32_t *negs, uint64_t *ctx_off, int32_t *ctx,
+                      uint64_t cap_ex, uint64_t cap_ctx, uint64_t *n_ex, uint64_t *n_ctx)
+{
+    if (!h->have_tables || W < 1 || W > 127 || N < 1 || N > 64) return -1;
+    cbowsink s = { centre, negs, ctx, ctx_off, cap_ex, cap_ctx, 0 };
+    if (cap_ex) ctx_off[0] = 0;
+    sample_chunk_cbow(h, tokens, n, W, N, h->step_id, sink_example, &s);
+    *n_ex = h->st_centres; *n_ctx = s.n_ctx;
+    return 0;
+}
+
+static void mean_context(orc *h, const int32_t *contexts, uint32_t n_ctx, double *hbar)
+{
+    uint32_t d = h->d;
+    for (uint32_t j = 0; j < d; ++j) hbar[j] = 0.0;
+    for (uint32_t k = 0; k < n_ctx; ++k) {
+        const float *u = rs_row(&h->U, h, (uint64_t)contexts[k]);
+        for (uint32_t j = 0; j < d; ++j) hbar[j] += (double)u[j];
+    }
+    for (uint32_t j = 0; j < d; ++j) hbar[j] /= (double)n_ctx;
+}
+static double dot_hv(const double *hbar, const float *v, uint32_t d)
+{
+    double s = 0.0;
+    for (uint32_t j = 0; j < d; ++j) s += hbar[j] * (double)v[j];
+    return s;
+}
+
+/* -- mode 1: one example after another, each seeing all earlier writes -- */
+typedef struct { orc *h; double lr; double *hbar, *e; } cseqctx;
+static void cbow_seq(void *ctx, uint64_t ex, int32_t c, const int32_t *contexts, uint32_t n_ctx,
+                     const int32_t *negs, uint32_t N)
+{
+    (void)ex;
+    cseqctx *s = (cseqctx *)ctx;
+    orc *h = s->h;
+    uint32_t d = h->d;
+    mean_context(h, contexts, n_ctx, s->hbar);
+    for (uint32_t j = 0; j < d; ++j) s->e[j] = 0.0;
+    for (uint32_t k = 0; k <= N; ++k) {
+        int32_t t = k == 0 ? c : negs[k - 1];
+        double label = k == 0 ? 1.0 : 0.0;
+        float *v = rs_row(&h->V, h, (uint64_t)t);
+        double g = s->lr * (label - sigmoid(dot_hv(s->hbar, v, d)));
+        for (uint32_t j = 0; j < d; ++j) s->e[j] += g * (double)v[j];
+        for (uint32_t j = 0; j < d; ++j) v[j] = (float)((double)v[j] + g * s->hbar[j]);
+    }
+    for (uint32_t k = 0; k < n_ctx; ++k) {
+        float *u = rs_row(&h->U, h, (uint64_t)contexts[k]);
+        for (uint32_t j = 0; j < d; ++j) u[j] = (float)((double)u[j] + s->e[j] / (double)n_ctx);
+    }
+}
+
+/* -- mode 0: every read sees start-of-step values, sums applied at the end -- */
+typedef struct { snapctx sn; double *hbar, *e; } csnapctx;
+static void cbow_snap(void *ctx, uint64_t ex, int32_t c, const int32_t *contexts, uint32_t n_ctx,
+                      const int32_t *negs, uint32_t N)
+{
+    (void)ex;
+    csnapctx *s = (csnapctx *)ctx;
+    orc *h = s->sn.h;
+    uint32_t d = h->d;
+    mean_context(h, contexts, n_ctx, s->hbar);
+    for (uint32_t j = 0; j < d; ++j) s->e[j] = 0.0;
+    for (uint32_t k = 0; k <= N; ++k) {
+        int32_t t = k == 0 ? c : negs[k - 1];
+        const float *v = rs_row(&h->V, h, (uint64_t)t);
+        double f = dot_hv(s->hbar, v, d);
+        double g = k == 0 ? s->sn.lr * (1.0 - sigmoid(f)) : -s->sn.lr * sigmoid(f);
+        for (uint32_t j = 0; j < d; ++j) s->e[j] += g * (double)v[j];
+        double *dv = delta_row(&s->sn, 0, t);
+        for (uint32_t j = 0; j < d; ++j) dv[j] += g * s->hbar[j];
+    }
+    for (uint32_t k = 0; k < n_ctx; ++k) {
+        double *du = delta_row(&s->sn, 1, contexts[k]);
+        for (uint32_t j = 0; j < d; ++j) du[j] += s->e[j] / (double)n_ctx;
+    }
+}
+
+typedef struct { orc *h; double sum; double *hbar; } clossctx;
+static void cbow_loss_ex(void *ctx, uint64_t ex, int32_t c, const int32_t *contexts, uint32_t n_ctx,
+                         const int32_t *negs, uint32_t N)
+{
+    (void)ex;
+    clossctx *s = (clossctx *)ctx;
+    orc *h = s->h;
+    mean_context(h, contexts, n_ctx, s->hbar);
+    s->sum += log_sigmoid(dot_hv(s->hbar, rs_row(&h->V, h, (uint64_t)c), h->d));
+    for (uint32_t k = 0; k < N; ++k)
+        s->sum += log_sigmoid(-dot_hv(s->hbar, rs_row(&h->V, h, (uint64_t)negs[k]), h->d));
+}
+
+/* runs fn over sampled examples (tokens != NULL) or over explicit lists */
+static void cbow_run(orc *h, const int32_t *tokens, uint64_t n, uint32_t W, uint32_t N, uint64_t step_id,
+                     const int32_t *centre, const int32_t *negs, const uint64_t *ctx_off,
+                     const int32_t *ctxs, uint64_t E, cbow_fn fn, void *ctx)
+{
+    if (tokens) { sample_chunk_cbow(h, tokens, n, W, N, step_id, fn, ctx); return; }
+    for (uint64_t e = 0; e < E; ++e)
+        fn(ctx, e, centre[e], ctxs + ctx_off[e], (uint32_t)(ctx_off[e + 1] - ctx_off[e]), negs + e * N, N);
+}
+
+static int cbow_step_impl(orc *h, const int32_t *tokens, uint64_t n, uint32_t W, uint32_t N,
+                          const int32_t *centre, const int32_t *negs, const uint64_t *ctx_off,
+                          const int32_t *ctxs, uint64_t E, double lr, uint32_t mode)
+{
+    double *hbar = (double *)malloc(h->d * sizeof(double)), *e = (double *)malloc(h->d * sizeof(double));
+    if (mode == 1) {
+        cseqctx s = { h, lr, hbar, e };
+        cbow_run(h, tokens, n, W, N, h->step_id, centre, negs, ctx_off, ctxs, E, cbow_seq, &s);
+    } else {
+        csnapctx s;
+        memset(&s, 0, sizeof(s));
+        s.sn.h = h; s.sn.lr = lr; s.hbar = hbar; s.e = e;
+        idmap_init(&s.sn.du_map, 4096); idmap_init(&s.sn.dv_map, 4096);
+        cbow_run(h, tokens, n, W, N, h->step_id, centre, negs, ctx_off, ctxs, E, cbow_snap, &s);
+        snap_apply(&s.sn, 1);
+        snap_apply(&s.sn, 0);
+        idmap_free(&s.sn.du_map); idmap_free(&s.sn.dv_map);
+        free(s.sn.du); free(s.sn.dv);
+    }
+    free(hbar); free(e);
+    return 0;
+}
+int orc_cbow_step(orc *h, const int32_t *tokens, uint64_t n, uint32_t W, uint32_t N, double lr, uint32_t mode)
+{
+    if (!h->have_tables || W < 1 || W > 127 || N < 1 || N > 64 || mode > 1) return -1;
+    cbow_step_impl(h, tokens, n, W, N, NULL, NULL, NULL, NULL, 0, lr, mode);
+    h->step_id++;
+    return 0;
+}
+int orc_cbow_step_examples(orc *h, const int32_t *centre, const int32_t *negs, const uint64_t *ctx_off,
+                           const int32_t *ctxs, uint64_t E, uint32_t N, double lr, uint32_t mode)
+{
+    if (mode > 1 || N > 64) return -1;
+    return cbow_step_impl(h, NULL, 0, 0, N, centre, negs, ctx_off, ctxs, E, lr, mode);
+}
+int orc_cbow_loss(orc *h, const int32_t *tokens, uint64_t n, uint32_t W, uint32_t N, uint64_t step_id,
+                  double *loss_sum, uint64_t *n_examples)
+{
+    if (!h->have_tables || W < 1 || W > 127 || N < 1 || N > 64) return -1;
+    clossctx s = { h, 0.0, (double *)malloc(h->d * sizeof(double)) };
+    sample_chunk_cbow(h, tokens, n, W, N, step_id, cbow_loss_ex, &s);
+    free(s.hbar);
+    *loss_sum = -s.sum;
+    *n_examples = h->st_centres;
+    return 0;
+}
+double orc_cbow_loss_examples(orc *h, const int32_t *centre, const int32_t *negs, const uint64_t *ctx_off,
+                              const int32_t *ctxs, uint64_t E, uint32_t N)
+{
+    clossctx s = { h, 0.0, (double *)malloc(h->d * sizeof(double)) };
+    cbow_run(h, NULL, 0, 0, N, 0, centre, negs, ctx_off, ctxs, E, cbow_loss_ex, &s);
+    free(s.hbar);
     return -s.sum;
 }
 
