@@ -177,6 +177,41 @@ int32_t w2v_sample_pairs(w2v_handle *h, const int32_t *tokens, uint64_t n, uint3
                          uint64_t cap, uint64_t *n_pairs, w2v_step_stats *stats);
 
 /*
+ * ---- Continuous bag of words (footnote to Section 5: the system "readily extends to the
+ * continuous bag of words (CBOW) variant") -------------------------------------------------------
+ * One example per kept token q that has at least one context word in its window (window,
+ * sub-sampling and dirty contexts exactly as in w2v_sgns_step):
+ *   hbar = mean of u(w_k) over the window's context words k (the input table),
+ *   targets t: the centre word w_q with label 1 and `negatives` words != w_q with label 0, drawn
+ *              from the alias table with the random counter of offset 0 (slot = window),
+ *   F = hbar.v(t), G = lr (label - s(F)), v(t) += G hbar, and every context word gets
+ *   u(w_k) += (sum_t G v(t)) / |window|   -- lr times the exact gradient of the example's log
+ *   likelihood (the open-source word2vec program adds the undivided sum; that is not followed).
+ * mode, stats, step number, scratch and errors as for w2v_sgns_step; stats->centres counts the
+ * examples and stats->pairs the (centre, context) pairs, i.e. the context rows read.
+ * Refused with W2V_ERR_STATE on a column shard.
+ */
+int32_t w2v_cbow_step(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window,
+                      uint32_t negatives, float lr, uint32_t mode, w2v_step_stats *stats);
+
+/* The same with the chunk in HOST memory (see w2v_sgns_step_host). */
+int32_t w2v_cbow_step_host(w2v_handle *h, const int32_t *tokens_host, uint64_t n, uint32_t window,
+                           uint32_t negatives, float lr, uint32_t mode, w2v_step_stats *stats);
+
+/*
+ * The examples the next w2v_cbow_step would use, without touching the tables or the step number:
+ * centre word and negatives of example e (examples ordered by centre position).  The context
+ * words of the examples are the contexts of w2v_sample_pairs, grouped by centre.
+ *   centre  device, cap int32;  negs  device, cap*negatives int32.
+ *   n_examples  host; receives the number of examples (also when > cap: W2V_ERR_CAPACITY, the
+ *               first cap are written).
+ * Synchronises the stream.
+ */
+int32_t w2v_sample_cbow(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window,
+                        uint32_t negatives, int32_t *centre, int32_t *negs, uint64_t cap,
+                        uint64_t *n_examples, w2v_step_stats *stats);
+
+/*
  * ---- Column shards: the paper's own partition (Section 5.1, Eq. (6)-(7)) ----------------------
  * Shard s of S holds columns [col_lo, col_hi) of every row of U and V.  One minibatch is
  *   1. every shard: w2v_shard_dots    -- Algorithm 1 ("dotprod") on its slice, for the index

@@ -21,7 +21,8 @@ TABLE_U, TABLE_V = 0, 1
 
 EXPORTS = (
     "w2v_create", "w2v_create_strided", "w2v_create_shard", "w2v_shard_dots", "w2v_shard_adjust",
-    "w2v_get_row_stride", "w2v_set_interleave", "w2v_destroy", "w2v_build_alias", "w2v_get_tables", "w2v_sgns_step",
+    "w2v_get_row_stride", "w2v_set_interleave", "w2v_cbow_step", "w2v_cbow_step_host", "w2v_sample_cbow",
+    "w2v_destroy", "w2v_build_alias", "w2v_get_tables", "w2v_sgns_step",
     "w2v_sgns_step_host", "w2v_sample_pairs", "w2v_partial_dots", "w2v_read_rows", "w2v_write_rows",
     "w2v_set_step", "w2v_get_step", "w2v_get_table_ptrs", "w2v_sync", "w2v_profile_enable",
     "w2v_profile_read", "w2v_get_launch_count", "w2v_set_tuning", "w2v_last_error",
@@ -75,6 +76,9 @@ def load():
         "w2v_get_tables": [vp, vp, vp, vp],
         "w2v_sgns_step": [vp, vp, u64, u32, u32, C.c_float, u32, C.POINTER(StepStats)],
         "w2v_sgns_step_host": [vp, vp, u64, u32, u32, C.c_float, u32, C.POINTER(StepStats)],
+        "w2v_cbow_step": [vp, vp, u64, u32, u32, C.c_float, u32, C.POINTER(StepStats)],
+        "w2v_cbow_step_host": [vp, vp, u64, u32, u32, C.c_float, u32, C.POINTER(StepStats)],
+        "w2v_sample_cbow": [vp, vp, u64, u32, u32, vp, vp, u64, C.POINTER(u64), C.POINTER(StepStats)],
         "w2v_sample_pairs": [vp, vp, u64, u32, u32, vp, vp, vp, u64, C.POINTER(u64), C.POINTER(StepStats)],
         "w2v_sample_pairs_noalloc": [vp, vp, u64, u32, u32, vp, vp, vp, u64, C.POINTER(u64), C.POINTER(StepStats)],
         "w2v_partial_dots": [vp, vp, u64, u32, u32, vp],
@@ -188,6 +192,24 @@ def w2v_sgns_step(h, tokens, n, window, negatives, lr, mode, stats=None, allow=(
 def w2v_sgns_step_host(h, tokens_host, n, window, negatives, lr, mode, stats=None, allow=()):
     ref = C.byref(stats) if stats is not None else None
     return _check(h, load().w2v_sgns_step_host(h, _ptr(tokens_host), int(n), window, negatives, float(lr), mode, ref), allow)
+
+
+def w2v_cbow_step(h, tokens, n, window, negatives, lr, mode, stats=None, allow=()):
+    ref = C.byref(stats) if stats is not None else None
+    return _check(h, load().w2v_cbow_step(h, _ptr(tokens), int(n), window, negatives, float(lr), mode, ref), allow)
+
+
+def w2v_cbow_step_host(h, tokens_host, n, window, negatives, lr, mode, stats=None, allow=()):
+    ref = C.byref(stats) if stats is not None else None
+    return _check(h, load().w2v_cbow_step_host(h, _ptr(tokens_host), int(n), window, negatives, float(lr), mode, ref), allow)
+
+
+def w2v_sample_cbow(h, tokens, n, window, negatives, centre, negs, cap, stats=None, allow=()):
+    nex = C.c_uint64(0)
+    ref = C.byref(stats) if stats is not None else None
+    rc = _check(h, load().w2v_sample_cbow(h, _ptr(tokens), int(n), window, negatives, _ptr(centre), _ptr(negs),
+                                          int(cap), C.byref(nex), ref), allow)
+    return rc, int(nex.value)
 
 
 def w2v_sample_pairs(h, tokens, n, window, negatives, centre, context, negs, cap, stats=None, allow=()):
@@ -321,6 +343,25 @@ class W2V:
         st = StepStats() if want_stats else None
         w2v_sgns_step_host(self.h, tokens_host, n, window, negatives, lr, mode, st, allow)
         return st.as_dict() if want_stats else None
+
+    def cbow_step(self, tokens, window, negatives, lr, mode, want_stats=True, allow=()):
+        t = self._dev_tokens(tokens)
+        st = StepStats() if want_stats else None
+        w2v_cbow_step(self.h, t, t.numel(), window, negatives, lr, mode, st, allow)
+        return st.as_dict() if want_stats else None
+
+    def sample_cbow(self, tokens, window, negatives, cap=None, allow=()):
+        """(centre[E], negs[E, N], counters) of the examples the next cbow_step would use."""
+        t = self._dev_tokens(tokens)
+        n = t.numel()
+        if cap is None:
+            cap = max(1, n)
+        centre = torch.empty(cap, dtype=torch.int32, device=self.device)
+        negs = torch.empty(cap * negatives, dtype=torch.int32, device=self.device)
+        st = StepStats()
+        rc, E = w2v_sample_cbow(self.h, t, n, window, negatives, centre, negs, cap, st, allow)
+        m = min(E, cap)
+        return centre[:m].cpu().numpy(), negs[: m * negatives].view(m, negatives).cpu().numpy(), st.as_dict()
 
     def sample_pairs(self, tokens, window, negatives, cap=None, allow=()):
         t = self._dev_tokens(tokens)

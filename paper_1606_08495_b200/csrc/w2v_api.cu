@@ -268,6 +268,63 @@ int32_t step_impl(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t win
     return W2V_OK;
 }
 
+// the continuous-bag-of-words step: same sampling, one example per centre with a context
+int32_t cbow_step_impl(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window, uint32_t negatives,
+                       float lr, uint32_t mode, w2v_step_stats *stats)
+{
+    if (mode > 1) return fail(h, W2V_ERR_ARG, "mode must be 0 (snapshot) or 1 (hogwild)");
+    if (h->is_shard) return fail(h, W2V_ERR_STATE, "a column shard has no continuous-bag-of-words step");
+    int32_t rc = enqueue_sampling(h, tokens, n, window);
+    if (rc != W2V_OK) return rc;
+    if (mode == W2V_MODE_HOGWILD) {
+        StepParams p = make_params(h, window, negatives, lr);
+        if ((rc = profile_mark(h)) != W2V_OK) return rc;
+        int k = launch_cbow_hogwild(p, h->blocks_per_sm, h->sms, h->stream);
+        if (k < 0) return fail(h, W2V_ERR_CUDA, "update kernel launch", cudaGetLastError());
+        h->launches += (uint64_t)k;
+        if (h->profiling) h->prof_launches += (uint64_t)k;
+        if ((rc = profile_mark(h)) != W2V_OK) return rc;
+    } else {
+        // coefficients are indexed by kept position, so the kept count sizes their array
+        if ((rc = read_state(h, n, nullptr)) != W2V_OK) return rc;
+        const uint64_t need_g = h->st_host->n_kept * (uint64_t)(negatives + 1);
+        if (need_g > h->G_cap) {
+            cudaFree(h->G); h->G = nullptr; h->G_cap = 0;
+            const uint64_t cap = need_g + need_g / 4 + 1024;
+            W2V_CUDA(h, dev_alloc(&h->G, cap));
+            h->G_cap = cap;
+        }
+        const uint64_t need_du = h->sc.n_cap * (uint64_t)h->d;
+        if (need_du > h->DU_cap) {
+            cudaFree(h->DU); h->DU = nullptr; h->DU_cap = 0;
+            W2V_CUDA(h, dev_alloc(&h->DU, need_du));
+            h->DU_cap = need_du;
+        }
+        const uint64_t need_dv = (uint64_t)h->hot_rows * h->d;
+        if (need_dv > h->DV_cap) {
+            cudaFree(h->DV); h->DV = nullptr; h->DV_cap = 0;
+            W2V_CUDA(h, dev_alloc(&h->DV, need_dv));
+            W2V_CUDA(h, cudaMemsetAsync(h->DV, 0, need_dv * sizeof(double), h->stream));
+            h->DV_cap = need_dv;
+        }
+        if (h->st_host->pairs > 0) {
+            StepParams p = make_params(h, window, negatives, lr);
+            if ((rc = profile_mark(h)) != W2V_OK) return rc;
+            int k = launch_cbow_snapshot(p, h->blocks_per_sm, h->sms, h->stream);
+            if (k < 0) return fail(h, W2V_ERR_CUDA, "update kernel launch", cudaGetLastError());
+            h->launches += (uint64_t)k;
+            if (h->profiling) h->prof_launches += (uint64_t)k;
+            if ((rc = profile_mark(h)) != W2V_OK) return rc;
+        }
+    }
+    h->step_id += 1;
+    if (stats) {
+        if ((rc = read_state(h, n, stats)) != W2V_OK) return rc;
+        if (stats->status & 1u) return fail(h, W2V_ERR_TOKEN_RANGE, "token ids outside [-1, vocab) were skipped");
+    }
+    return W2V_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -440,6 +497,59 @@ int32_t w2v_sample_pairs(w2v_handle *h, const int32_t *tokens, uint64_t n, uint3
     if (stats) *stats = local;
     *n_pairs = local.pairs;
     if (local.pairs > cap) return fail(h, W2V_ERR_CAPACITY, "more pairs than the output arrays hold");
+    if (local.status & 1u) return fail(h, W2V_ERR_TOKEN_RANGE, "token ids outside [-1, vocab) were skipped");
+    return W2V_OK;
+}
+
+int32_t w2v_cbow_step(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window, uint32_t negatives,
+                      float lr, uint32_t mode, w2v_step_stats *stats)
+{
+    int32_t rc = check_step_args(h, tokens, n, window, negatives);
+    if (rc != W2V_OK) return rc;
+    DeviceGuard g(h->device);
+    return cbow_step_impl(h, tokens, n, window, negatives, lr, mode, stats);
+}
+
+int32_t w2v_cbow_step_host(w2v_handle *h, const int32_t *tokens_host, uint64_t n, uint32_t window,
+                           uint32_t negatives, float lr, uint32_t mode, w2v_step_stats *stats)
+{
+    int32_t rc = check_step_args(h, tokens_host, n, window, negatives);
+    if (rc != W2V_OK) return rc;
+    DeviceGuard g(h->device);
+    if (n > h->tok_stage_cap) {
+        W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+        cudaFree(h->tok_stage); h->tok_stage = nullptr; h->tok_stage_cap = 0;
+        W2V_CUDA(h, dev_alloc(&h->tok_stage, n));
+        h->tok_stage_cap = n;
+    }
+    if (n)
+        W2V_CUDA(h, cudaMemcpyAsync(h->tok_stage, tokens_host, n * sizeof(int32_t), cudaMemcpyHostToDevice, h->stream));
+    return cbow_step_impl(h, h->tok_stage, n, window, negatives, lr, mode, stats);
+}
+
+int32_t w2v_sample_cbow(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window, uint32_t negatives,
+                        int32_t *centre, int32_t *negs, uint64_t cap, uint64_t *n_examples, w2v_step_stats *stats)
+{
+    int32_t rc = check_step_args(h, tokens, n, window, negatives);
+    if (rc != W2V_OK) return rc;
+    if (!n_examples) return fail(h, W2V_ERR_ARG, "n_examples is NULL");
+    if (cap && (!centre || !negs)) return fail(h, W2V_ERR_ARG, "output array is NULL");
+    DeviceGuard g(h->device);
+    if ((rc = enqueue_sampling(h, tokens, n, window)) != W2V_OK) return rc;
+    int k = launch_pair_offsets(n, h->sc, h->st, h->stream, true);
+    if (k < 0) return fail(h, W2V_ERR_CUDA, "example offset launch", cudaGetLastError());
+    h->launches += (uint64_t)k;
+    if (n) {
+        StepParams p = make_params(h, window, negatives, 0.f);
+        k = launch_cbow_emit(p, centre, negs, cap, h->sms * 8, h->stream);
+        if (k < 0) return fail(h, W2V_ERR_CUDA, "example list launch", cudaGetLastError());
+        h->launches += (uint64_t)k;
+    }
+    w2v_step_stats local;
+    if ((rc = read_state(h, n, &local)) != W2V_OK) return rc;
+    if (stats) *stats = local;
+    *n_examples = local.centres;
+    if (local.centres > cap) return fail(h, W2V_ERR_CAPACITY, "more examples than the output arrays hold");
     if (local.status & 1u) return fail(h, W2V_ERR_TOKEN_RANGE, "token ids outside [-1, vocab) were skipped");
     return W2V_OK;
 }

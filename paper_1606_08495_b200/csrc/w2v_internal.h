@@ -93,7 +93,14 @@ int launch_compact(const int32_t *tokens, uint64_t n, const SampleTables &tab, u
                    cudaStream_t s);
 int launch_windows(uint64_t n, uint32_t window, uint32_t k0, uint32_t k1, uint32_t step_lo,
                    uint32_t il_phase, uint32_t il_stride, const Scratch &sc, DevState *st, cudaStream_t s);
-int launch_pair_offsets(uint64_t n, const Scratch &sc, DevState *st, cudaStream_t s);
+// pair_off[q] = number of pairs of the centres before q; with examples = true, the number of
+// centres before q that have at least one context (the example number of the CBOW variant)
+int launch_pair_offsets(uint64_t n, const Scratch &sc, DevState *st, cudaStream_t s, bool examples = false);
+
+// ---- continuous bag of words (w2v_cbow.cu) ----
+int launch_cbow_hogwild(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s);
+int launch_cbow_snapshot(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s);
+int launch_cbow_emit(const StepParams &p, int32_t *centre, int32_t *negs, uint64_t cap, int grid, cudaStream_t s);
 int launch_emit_pairs(const StepParams &p, int32_t *centre, int32_t *context, int32_t *negs,
                       uint64_t cap, int grid, cudaStream_t s);
 
@@ -105,6 +112,8 @@ int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t block
 int launch_snapshot_apply(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s);
 // passes 2b and 3 alone: the fp64 sums of the most-hit rows and the centre sums are applied
 int launch_snapshot_tail(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s);
+// pass 2b alone (0 launches when no row is summed in fp64)
+int launch_apply_hot(const StepParams &p, int sms, cudaStream_t s);
 // pass 2 (and the tail) for a column shard: narrow slices put several rows side by side in a warp
 int launch_shard_apply(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s);
 

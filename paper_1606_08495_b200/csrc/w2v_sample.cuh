@@ -53,6 +53,42 @@ __device__ __forceinline__ uint32_t pair_target(uint32_t t, uint32_t w_out, uint
     return t == 0 ? w_out : r;
 }
 
+// Walks the targets of one (centre, context) pair in batches of TB rows so that TB row
+// gathers are in flight before the first dot is reduced.
+//   onTarget(t, target_row, v, f) is called once per target in order t = 0..N with the
+//   gathered row and the full dot product.
+template <int VPL, int TB, typename F>
+__device__ __forceinline__ void for_each_target(const StepParams &p, const Row<VPL> &u, uint32_t w_out,
+                                                uint32_t n0, uint32_t n1, uint32_t lane, F &&onTarget)
+{
+    const float4 *V4 = reinterpret_cast<const float4 *>(p.V);
+    const bool wide = p.negatives > 32u;
+    for (uint32_t t0 = 0; t0 <= p.negatives; t0 += TB) {
+        uint32_t tgt[TB];
+        Row<VPL> v[TB];
+        float f[TB];
+#pragma unroll
+        for (int b = 0; b < TB; ++b) {
+            const uint32_t t = t0 + b;
+            tgt[b] = pair_target(t, w_out, n0, n1, wide);
+            if (t <= p.negatives) row_load(v[b], V4 + (size_t)tgt[b] * p.ld4, p.d4, lane);
+            else row_zero(v[b]);
+        }
+#pragma unroll
+        for (int b = 0; b < TB; ++b) f[b] = row_dot_partial(u, v[b]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+            for (int b = 0; b < TB; ++b) f[b] += __shfl_xor_sync(kFullMask, f[b], o);
+        }
+#pragma unroll
+        for (int b = 0; b < TB; ++b) {
+            const uint32_t t = t0 + b;
+            if (t <= p.negatives) onTarget(t, tgt[b], v[b], f[b]);
+        }
+    }
+}
+
 __device__ __forceinline__ void flush_draw_counts(DevState *st, uint32_t draws, uint32_t redraws)
 {
     const uint32_t d = warp_sum(draws), r = warp_sum(redraws);

@@ -137,11 +137,14 @@ window_kernel(const uint32_t *__restrict__ cidx, const uint32_t *__restrict__ cs
 }
 
 // ---- pair offsets: exclusive scan of the context counts ------------------------------
-__device__ __forceinline__ uint32_t win_count(uint16_t w) { return (w & 0xFFu) + (w >> 8); }
+__device__ __forceinline__ uint32_t win_count(uint16_t w, bool examples)
+{
+    return examples ? (w != 0 ? 1u : 0u) : (w & 0xFFu) + (w >> 8);
+}
 
 __global__ void __launch_bounds__(kScanBlock)
 pair_tile_sums_kernel(const uint16_t *__restrict__ win, unsigned long long *__restrict__ cnt_tile,
-                      const DevState *st)
+                      const DevState *st, bool examples)
 {
     __shared__ uint32_t sh[33];
     const uint32_t nk = (uint32_t)st->n_kept;
@@ -149,7 +152,7 @@ pair_tile_sums_kernel(const uint16_t *__restrict__ win, unsigned long long *__re
     uint32_t s = 0;
 #pragma unroll
     for (int e = 0; e < kScanItems; ++e)
-        if (base + e < nk) s += win_count(win[base + e]);
+        if (base + e < nk) s += win_count(win[base + e], examples);
     uint32_t total;
     block_exclusive_scan<uint32_t>(s, sh, total);
     if (threadIdx.x == 0) cnt_tile[blockIdx.x] = total;
@@ -172,7 +175,7 @@ pair_scan_tiles_kernel(unsigned long long *__restrict__ cnt_tile, uint32_t n_til
 
 __global__ void __launch_bounds__(kScanBlock)
 pair_offsets_kernel(const uint16_t *__restrict__ win, const unsigned long long *__restrict__ cnt_tile,
-                    unsigned long long *__restrict__ pair_off, const DevState *st)
+                    unsigned long long *__restrict__ pair_off, const DevState *st, bool examples)
 {
     __shared__ uint32_t sh[33];
     const uint32_t nk = (uint32_t)st->n_kept;
@@ -181,7 +184,7 @@ pair_offsets_kernel(const uint16_t *__restrict__ win, const unsigned long long *
     uint32_t s = 0;
 #pragma unroll
     for (int e = 0; e < kScanItems; ++e) {
-        c[e] = base + e < nk ? win_count(win[base + e]) : 0u;
+        c[e] = base + e < nk ? win_count(win[base + e], examples) : 0u;
         s += c[e];
     }
     uint32_t total;
@@ -260,13 +263,13 @@ int launch_windows(uint64_t n, uint32_t window, uint32_t k0, uint32_t k1, uint32
     return 1;
 }
 
-int launch_pair_offsets(uint64_t n, const Scratch &sc, DevState *st, cudaStream_t s)
+int launch_pair_offsets(uint64_t n, const Scratch &sc, DevState *st, cudaStream_t s, bool examples)
 {
     const uint32_t nt = tiles_for(n);
     if (nt == 0) return 0;
-    pair_tile_sums_kernel<<<nt, kScanBlock, 0, s>>>(sc.win, sc.cnt_tile, st);
+    pair_tile_sums_kernel<<<nt, kScanBlock, 0, s>>>(sc.win, sc.cnt_tile, st, examples);
     pair_scan_tiles_kernel<<<1, 1024, 0, s>>>(sc.cnt_tile, nt);
-    pair_offsets_kernel<<<nt, kScanBlock, 0, s>>>(sc.win, sc.cnt_tile, sc.pair_off, st);
+    pair_offsets_kernel<<<nt, kScanBlock, 0, s>>>(sc.win, sc.cnt_tile, sc.pair_off, st, examples);
     if (cudaGetLastError() != cudaSuccess) return -1;
     return 3;
 }

@@ -11,42 +11,6 @@
 
 namespace w2v {
 
-// Walks the targets of one (centre, context) pair in batches of TB rows so that TB row
-// gathers are in flight before the first dot is reduced.
-//   onTarget(t, target_row, v, f) is called once per target in order t = 0..N with the
-//   gathered row and the full dot product.
-template <int VPL, int TB, typename F>
-__device__ __forceinline__ void for_each_target(const StepParams &p, const Row<VPL> &u, uint32_t w_out,
-                                                uint32_t n0, uint32_t n1, uint32_t lane, F &&onTarget)
-{
-    const float4 *V4 = reinterpret_cast<const float4 *>(p.V);
-    const bool wide = p.negatives > 32u;
-    for (uint32_t t0 = 0; t0 <= p.negatives; t0 += TB) {
-        uint32_t tgt[TB];
-        Row<VPL> v[TB];
-        float f[TB];
-#pragma unroll
-        for (int b = 0; b < TB; ++b) {
-            const uint32_t t = t0 + b;
-            tgt[b] = pair_target(t, w_out, n0, n1, wide);
-            if (t <= p.negatives) row_load(v[b], V4 + (size_t)tgt[b] * p.ld4, p.d4, lane);
-            else row_zero(v[b]);
-        }
-#pragma unroll
-        for (int b = 0; b < TB; ++b) f[b] = row_dot_partial(u, v[b]);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-            for (int b = 0; b < TB; ++b) f[b] += __shfl_xor_sync(kFullMask, f[b], o);
-        }
-#pragma unroll
-        for (int b = 0; b < TB; ++b) {
-            const uint32_t t = t0 + b;
-            if (t <= p.negatives) onTarget(t, tgt[b], v[b], f[b]);
-        }
-    }
-}
-
 // ---- Hogwild mode: one pass, updates land as they are computed ---------------------------
 template <int VPL, int TB>
 __global__ void __launch_bounds__(kBlock)
@@ -320,14 +284,23 @@ int launch_snapshot_apply(const StepParams &p, uint32_t blocks_per_sm, int sms, 
     return k < 0 ? -1 : 1 + k;
 }
 
+int launch_apply_hot(const StepParams &p, int sms, cudaStream_t s)
+{
+    if (!p.hot_rows) return 0;
+    const uint64_t want = ((uint64_t)p.hot_rows * 4u * p.d4 + kBlock - 1) / kBlock;
+    const int grid = (int)(want < (uint64_t)sms * 8 ? want : (uint64_t)sms * 8);
+    sgns_snap_apply_hot_kernel<<<grid, kBlock, 0, s>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    return 1;
+}
+
 int launch_snapshot_tail(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s)
 {
     int launched = 1;
-    if (p.hot_rows) {
-        const uint64_t want = ((uint64_t)p.hot_rows * 4u * p.d4 + kBlock - 1) / kBlock;
-        const int grid = (int)(want < (uint64_t)sms * 8 ? want : (uint64_t)sms * 8);
-        sgns_snap_apply_hot_kernel<<<grid, kBlock, 0, s>>>(p);
-        ++launched;
+    {
+        const int k = launch_apply_hot(p, sms, s);
+        if (k < 0) return -1;
+        launched += k;
     }
     {
         const int grid = grid_for(sgns_snap_apply_u_kernel, blocks_per_sm, sms);
