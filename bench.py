@@ -52,6 +52,17 @@ def algorithmic_bytes_snapshot(d, centres, pairs, negatives):
     return 4 * d * (3 * T + 6 * centres) + 8 * T
 
 
+def algorithmic_bytes_cbow(d, examples, pairs, negatives, snapshot=False):
+    """CBOW step: `pairs` context rows (one per (centre, context) pair) and E (1 + N) target rows.
+    Hogwild: every row read once and written once.  Snapshot: pass 1 reads P + T rows and writes E
+    scratch rows, pass 2 re-reads P rows and read-modify-writes T, pass 3 reads E and
+    read-modify-writes P (T = E (1 + N))."""
+    T = examples * (1 + negatives)
+    if snapshot:
+        return 4 * d * (4 * pairs + 3 * T + 2 * examples) + 8 * T
+    return 4 * d * (2 * pairs + 2 * T)
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -222,6 +233,9 @@ def run_gpu(args):
     W, N, lr, d = cfg["window"], cfg["negatives"], cfg["lr"], cfg["d"]
     K, Wu = args.steps, args.warmup
     mode = binding.MODE_HOGWILD if args.mode == "hogwild" else binding.MODE_SNAPSHOT
+    cbow = args.model == "cbow"
+    step_dev = binding.w2v_cbow_step if cbow else binding.w2v_sgns_step
+    step_host = binding.w2v_cbow_step_host if cbow else binding.w2v_sgns_step_host
 
     row_stride = d if args.dense_rows else row_stride_for(d, args.row_stride)
     model = binding.W2V(cfg["vocab"], d, seed=1, device=dev, row_stride=row_stride)
@@ -241,8 +255,12 @@ def run_gpu(args):
         model.set_step(i)
         t = dev_chunks[i]
         st = binding.StepStats()
-        binding.w2v_sample_pairs(model.h, t, t.numel(), W, N, None, None, None, 0, st,
-                                 allow=(binding.W2V_ERR_CAPACITY,))
+        if cbow:
+            binding.w2v_sample_cbow(model.h, t, t.numel(), W, N, None, None, 0, st,
+                                    allow=(binding.W2V_ERR_CAPACITY,))
+        else:
+            binding.w2v_sample_pairs(model.h, t, t.numel(), W, N, None, None, None, 0, st,
+                                     allow=(binding.W2V_ERR_CAPACITY,))
         centres.append(st.centres); pairs.append(st.pairs)
     model.set_step(0)
 
@@ -252,7 +270,7 @@ def run_gpu(args):
 
     # ---- device-timed run: inputs already resident in HBM ----
     for i in range(Wu):
-        binding.w2v_sgns_step(model.h, dev_chunks[i], dev_chunks[i].numel(), W, N, lr, mode, None)
+        step_dev(model.h, dev_chunks[i], dev_chunks[i].numel(), W, N, lr, mode, None)
     model.sync()
     binding.w2v_profile_enable(model.h, True)
     launches0 = model.launch_count()
@@ -267,7 +285,7 @@ def run_gpu(args):
             if IL > 1:
                 binding.w2v_set_step(model.h, i)
                 binding.w2v_set_interleave(model.h, phase, IL)
-            binding.w2v_sgns_step(model.h, dev_chunks[i], dev_chunks[i].numel(), W, N, lr, mode, None)
+            step_dev(model.h, dev_chunks[i], dev_chunks[i].numel(), W, N, lr, mode, None)
     ev1.record()
     torch.cuda.synchronize(dev); barrier()
     clocks = sampler.stop()
@@ -289,7 +307,7 @@ def run_gpu(args):
             if IL > 1:
                 binding.w2v_set_step(model.h, i)
                 binding.w2v_set_interleave(model.h, phase, IL)
-            binding.w2v_sgns_step_host(model.h, t, t.numel(), W, N, lr, mode, st)
+            step_host(model.h, t, t.numel(), W, N, lr, mode, st)
             e2e_pairs += st.pairs
             h2d += 4 * t.numel(); d2h += 64
     ev3.record()
@@ -297,8 +315,11 @@ def run_gpu(args):
     e2e_ms = ev2.elapsed_time(ev3)
 
     tot_pairs = float(sum(pairs))
-    model_bytes = algorithmic_bytes if args.mode == "hogwild" else algorithmic_bytes_snapshot
-    tot_bytes = float(sum(model_bytes(d, c, p, N) for c, p in zip(centres, pairs)))
+    if cbow:
+        tot_bytes = float(sum(algorithmic_bytes_cbow(d, c, p, N, args.mode == "snapshot") for c, p in zip(centres, pairs)))
+    else:
+        model_bytes = algorithmic_bytes if args.mode == "hogwild" else algorithmic_bytes_snapshot
+        tot_bytes = float(sum(model_bytes(d, c, p, N) for c, p in zip(centres, pairs)))
     ms, e2e_ms, all_pairs, all_e2e_pairs, all_launches = reduce_over_ranks(
         ms, e2e_ms, tot_pairs, float(e2e_pairs), launches, world, dev)
 
@@ -313,7 +334,7 @@ def run_gpu(args):
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": name, "vocab": cfg["vocab"], "d": d, "window": W, "negatives": N,
                        "subsample_t": cfg["subsample_t"], "tokens_per_step": int(dev_chunks[0].numel()),
-                       "mode": args.mode, "row_stride_floats": row_stride, "interleave": IL, "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
+                       "model": args.model, "mode": args.mode, "row_stride_floats": row_stride, "interleave": IL, "parallelism": f"replicas x{world}" if world > 1 else "1 gpu",
                        "l2": "tables and gathers far larger than L2 (random rows of %.1f GB)" % (2 * cfg["vocab"] * d * 4 / 1e9)
                              if 2 * cfg["vocab"] * d * 4 > 4 * 126e6 else "tables fit in L2; no flush between steps",
                        "pairs_per_step": tot_pairs / K, "centres_per_step": sum(centres) / K,
@@ -324,14 +345,14 @@ def run_gpu(args):
                     "h2d_bytes_per_step": h2d // K, "d2h_bytes_per_step": d2h // K},
             "gpu_launches": all_launches,
             "roofline": {"bound": "hbm",
-                         "kernel": "sgns_hogwild_kernel" if args.mode == "hogwild" else "sgns_snap_* (3 passes)",
+                         "kernel": ("cbow_" if cbow else "sgns_") + ("hogwild_kernel" if args.mode == "hogwild" else "snap_* (3 passes)"),
                          "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "frac_of_8TBps": achieved / 8000.0,
                          "algorithmic_bytes_per_launch": per_launch_bytes,
                          "kernel_ms_per_launch": kernel_ms / max(1, groups),
                          "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE * per_launch_bytes
-                                     if name == "large" and args.mode == "hogwild" and not args.row_stride
+                                     if name == "large" and args.mode == "hogwild" and not cbow and not args.row_stride
                                      and not args.rows_in_flight and not args.blocks_per_sm else None)},
         }
         if world == 1 and not args.no_cpu_baseline:
@@ -455,6 +476,9 @@ def main():
                     help="update mode of the timed steps (the headline number is hogwild); sharded = the "
                          "paper's column partition, --shards slices of one model on one GPU")
     ap.add_argument("--shards", type=int, default=8)
+    ap.add_argument("--model", choices=["sgns", "cbow"], default="sgns",
+                    help="skip-gram (the headline) or the continuous-bag-of-words variant; for cbow the "
+                         "metric counts (centre, context) pairs, i.e. context rows read")
     ap.add_argument("--interleave", type=int, default=1,
                     help="visit every chunk this many times, each time with 1/this of its input words "
                          "(interleaved minibatch formation)")
