@@ -20,6 +20,8 @@ struct w2v_handle {
     bool is_shard = false;
     // state between w2v_shard_dots and w2v_shard_adjust
     bool shard_pending = false;
+    int32_t *l_centre = nullptr, *l_context = nullptr, *l_negs = nullptr;   // pair list of a narrow shard's step
+    uint64_t l_cap_pairs = 0, l_cap_negs = 0;
     uint32_t pend_window = 0, pend_negatives = 0;
     uint64_t pend_n = 0, pend_pairs = 0;
     uint64_t seed = 0;
@@ -145,6 +147,7 @@ StepParams make_params(w2v_handle *h, uint32_t window, uint32_t negatives, float
     p.lr = lr;
     p.pair_off = h->sc.pair_off; p.G = h->G; p.DU = h->DU;
     p.DV = h->DV; p.hot_rows = h->DV ? h->hot_rows : 0;
+    p.l_centre = h->l_centre; p.l_context = h->l_context; p.l_negs = h->l_negs;
     return p;
 }
 
@@ -392,6 +395,7 @@ int32_t w2v_destroy(w2v_handle *h)
     cudaFree(h->st);
     if (h->st_host) cudaFreeHost(h->st_host);
     cudaFree(h->G); cudaFree(h->DU); cudaFree(h->DV); cudaFree(h->tok_stage);
+    cudaFree(h->l_centre); cudaFree(h->l_context); cudaFree(h->l_negs);
     for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
     cudaGetLastError();
     delete h;
@@ -577,6 +581,29 @@ int32_t w2v_shard_dots(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_
     const uint64_t pairs = h->st_host->pairs;
     if (pairs * (uint64_t)(negatives + 1) > cap)
         return fail(h, W2V_ERR_CAPACITY, "more targets than the arrays for the partial dot products hold");
+    if (pairs > 0 && h->d / 4 <= kNarrowD4) {
+        // narrow slice: write the index sets once, the three passes stream over them
+        if (pairs > h->l_cap_pairs) {
+            cudaFree(h->l_centre); cudaFree(h->l_context); h->l_centre = h->l_context = nullptr; h->l_cap_pairs = 0;
+            const uint64_t cap_p = pairs + pairs / 4 + 1024;
+            W2V_CUDA(h, dev_alloc(&h->l_centre, cap_p));
+            W2V_CUDA(h, dev_alloc(&h->l_context, cap_p));
+            h->l_cap_pairs = cap_p;
+        }
+        if (pairs * negatives > h->l_cap_negs) {
+            cudaFree(h->l_negs); h->l_negs = nullptr; h->l_cap_negs = 0;
+            const uint64_t cap_n = pairs * negatives + pairs * negatives / 4 + 1024;
+            W2V_CUDA(h, dev_alloc(&h->l_negs, cap_n));
+            h->l_cap_negs = cap_n;
+        }
+        StepParams pl = make_params(h, window, negatives, 0.f);
+        if ((rc = profile_mark(h)) != W2V_OK) return rc;
+        k = launch_emit_pairs(pl, h->l_centre, h->l_context, h->l_negs, pairs, h->sms * 8, h->stream);
+        if (k < 0) return fail(h, W2V_ERR_CUDA, "pair list launch", cudaGetLastError());
+        h->launches += (uint64_t)k;
+        if (h->profiling) h->prof_launches += (uint64_t)k;
+        if ((rc = profile_mark(h)) != W2V_OK) return rc;
+    }
     if (pairs > 0) {
         StepParams p = make_params(h, window, negatives, 0.f);
         if ((rc = profile_mark(h)) != W2V_OK) return rc;

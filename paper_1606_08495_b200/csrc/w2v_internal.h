@@ -59,12 +59,17 @@ struct StepParams {
     const unsigned long long *pair_off;   // first pair index of centre q
     float *G;                   // [pairs * (1 + negatives)] coefficients
     float *DU;                  // [kept * d] per-centre sums of G v(target)
+    // pair list of the step (column shards with narrow slices): written once, streamed by the passes
+    const int32_t *l_centre;    // [pairs]
+    const int32_t *l_context;   // [pairs]
+    const int32_t *l_negs;      // [pairs * negatives]
     double *DV;                 // [hot_rows * d] fp64 sums of G u(c) for the most-hit output rows
     uint32_t hot_rows;          // output rows [0, hot_rows) accumulate in DV (snapshot mode)
 };
 
 // F arrays of all shards (this one included) that receive a shard's partial dot products.
 constexpr int kMaxShards = 16;
+constexpr uint32_t kNarrowD4 = 16;     // slices of at most this many float4 use the pair-list passes
 struct ShardPeers {
     float *F[kMaxShards];
     uint32_t n;

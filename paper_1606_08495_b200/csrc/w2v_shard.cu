@@ -148,20 +148,20 @@ shard_du_kernel(StepParams p)
 }
 
 // ==== narrow slices =============================================================================
-// With 8 shards a 300-column vector leaves 36-40 columns (9-10 float4) per shard: one warp per row
-// would idle two thirds of its lanes and fetch 160 bytes per request.  Here a warp is split into
-// 32/GL groups of GL lanes (GL = 8 or 16, d/4 <= GL); each group works on its own target row, so
-// one request gathers 2 or 4 rows.  Lane sl of a group holds float4 number sl of every row.
+// With 8 shards a 300-column vector leaves 36-40 columns (9-10 float4) per shard.  One warp per
+// row would idle two thirds of its lanes, and a pass that regenerates the negatives pair by pair
+// is bound by that dependent chain (draw, alias-table read, then the rows), not by bytes.  So for
+// slices of at most 16 float4 the index sets are written once per step (the pair list of
+// w2v_sample_pairs: centre, context, negatives) and the passes stream over it.  A warp is split
+// into 32/GL groups of GL lanes (GL = 8 or 16, d/4 <= GL); each group works on its own target row
+// and lane sl of a group holds float4 number sl of every row.
 template <int GL>
 struct Narrow {
     static constexpr int NG = 32 / GL;                      // rows side by side in a warp
-    uint32_t lane, sl, grp;
-    __device__ explicit Narrow(uint32_t lane_) : lane(lane_), sl(lane_ & (GL - 1)), grp(lane_ / GL) {}
+    uint32_t sl, grp;
+    __device__ explicit Narrow(uint32_t lane) : sl(lane & (GL - 1)), grp(lane / GL) {}
 
-    __device__ float4 load(const float4 *row, uint32_t d4, bool on) const
-    {
-        return (on && sl < d4) ? __ldcg(row + sl) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
+    __device__ static float4 zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
     // sum over the lanes of a group
     __device__ static float group_sum(float x)
     {
@@ -178,70 +178,59 @@ struct Narrow {
     }
 };
 
-// target t of the pair for this lane (t may differ between the groups of a warp)
-__device__ __forceinline__ uint32_t narrow_target(uint32_t t, uint32_t w_out, uint32_t n0, uint32_t n1,
-                                                  uint32_t negatives)
+// output word of target j of the list: the context for t = 0, negative t-1 otherwise
+__device__ __forceinline__ uint32_t list_target(const StepParams &p, unsigned long long pair, uint32_t t)
 {
-    const uint32_t src = (t == 0 || t > negatives) ? 0u : t - 1u;
-    const uint32_t a = __shfl_sync(kFullMask, n0, src & 31u);
-    const uint32_t b = __shfl_sync(kFullMask, n1, src & 31u);
-    return t == 0 ? w_out : (src < 32u ? a : b);
+    return (uint32_t)(t == 0 ? __ldg(p.l_context + pair) : __ldg(p.l_negs + pair * p.negatives + (t - 1u)));
 }
 
+// Algorithm 1 over the list: one group per target, TB targets per group in flight.
 template <int GL, int TB>
 __global__ void __launch_bounds__(kBlock)
-shard_dots_narrow_kernel(StepParams p, ShardPeers peers)
+shard_dots_list_kernel(StepParams p, ShardPeers peers)
 {
     const Narrow<GL> nr(threadIdx.x & 31);
-    constexpr int NG = Narrow<GL>::NG;
-    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
-    const uint32_t nk = (uint32_t)p.st->n_kept;
+    const unsigned long long n1p = p.negatives + 1u;
+    const unsigned long long total = p.st->pairs * n1p;
+    const unsigned long long group = ((unsigned long long)blockIdx.x * blockDim.x + threadIdx.x) / GL;
+    const unsigned long long ngroups = ((unsigned long long)gridDim.x * blockDim.x) / GL;
     const float4 *U4 = reinterpret_cast<const float4 *>(p.U);
     const float4 *V4 = reinterpret_cast<const float4 *>(p.V);
-    const uint32_t n1p = p.negatives + 1u;
-    uint32_t draws = 0, redraws = 0;
-    for (uint32_t q = warp; q < nk; q += nwarps) {
-        const uint32_t w = p.win[q];
-        const uint32_t left = w & 0xFFu, right = w >> 8;
-        if (left + right == 0) continue;
-        const uint32_t c = (uint32_t)p.ctok[q];
-        const uint32_t i = p.cidx[q];
-        const float4 u = nr.load(U4 + (size_t)c * p.ld4, p.d4, true);
-        unsigned long long gi = p.pair_off[q] * n1p;
-        for (uint32_t pp = q - left; pp <= q + right; ++pp) {
-            if (pp == q) continue;
-            const uint32_t w_out = (uint32_t)p.ctok[pp];
-            uint32_t n0, n1;
-            draw_pair_negatives(p, i, pp + p.window - q, w_out, nr.lane, n0, n1, draws, redraws);
-            for (uint32_t t0 = 0; t0 < n1p; t0 += TB * NG) {
-                float f[TB];
-                float4 v[TB];
+    const bool on = nr.sl < p.d4;
+    // every lane of a warp runs the same number of rounds (the shuffles below are warp-wide)
+    for (unsigned long long j0 = group - nr.grp; j0 < total; j0 += ngroups * TB) {
+        float4 u[TB], v[TB];
+        float f[TB];
 #pragma unroll
-                for (int b = 0; b < TB; ++b) {
-                    const uint32_t t = t0 + b * NG + nr.grp;
-                    const uint32_t tgt = narrow_target(t, w_out, n0, n1, p.negatives);
-                    v[b] = nr.load(V4 + (size_t)tgt * p.ld4, p.d4, t < n1p);
-                }
-#pragma unroll
-                for (int b = 0; b < TB; ++b)
-                    f[b] = Narrow<GL>::group_sum(u.x * v[b].x + u.y * v[b].y + u.z * v[b].z + u.w * v[b].w);
-#pragma unroll
-                for (int b = 0; b < TB; ++b) {
-                    const uint32_t t = t0 + b * NG + nr.grp;
-                    if (nr.sl == 0 && t < n1p)
-                        for (uint32_t r = 0; r < peers.n; ++r) atomicAdd(peers.F[r] + gi + t, f[b]);
-                }
+        for (int b = 0; b < TB; ++b) {
+            const unsigned long long j = j0 + nr.grp + (unsigned long long)b * ngroups;
+            u[b] = v[b] = Narrow<GL>::zero();
+            if (j < total && on) {
+                const unsigned long long pair = j / n1p;
+                const uint32_t t = (uint32_t)(j - pair * n1p);
+                const uint32_t c = (uint32_t)__ldg(p.l_centre + pair);
+                const uint32_t tgt = list_target(p, pair, t);
+                u[b] = __ldg(U4 + (size_t)c * p.ld4 + nr.sl);       // U is not written during this pass
+                v[b] = __ldcg(V4 + (size_t)tgt * p.ld4 + nr.sl);
             }
-            gi += n1p;
+        }
+#pragma unroll
+        for (int b = 0; b < TB; ++b)
+            f[b] = Narrow<GL>::group_sum(u[b].x * v[b].x + u[b].y * v[b].y + u[b].z * v[b].z + u[b].w * v[b].w);
+#pragma unroll
+        for (int b = 0; b < TB; ++b) {
+            const unsigned long long j = j0 + nr.grp + (unsigned long long)b * ngroups;
+            if (nr.sl == 0 && j < total)
+                for (uint32_t r = 0; r < peers.n; ++r) atomicAdd(peers.F[r] + j, f[b]);
         }
     }
-    flush_draw_counts(p.st, draws, redraws);
 }
 
+// Algorithm 2, input rows: DU[q] = sum over the centre's targets of G v(target); a warp per centre,
+// its groups share the centre's targets.
 template <int GL, int TB>
 __global__ void __launch_bounds__(kBlock)
-shard_du_narrow_kernel(StepParams p)
+shard_du_list_kernel(StepParams p)
 {
     const Narrow<GL> nr(threadIdx.x & 31);
     constexpr int NG = Narrow<GL>::NG;
@@ -251,86 +240,68 @@ shard_du_narrow_kernel(StepParams p)
     const float4 *V4 = reinterpret_cast<const float4 *>(p.V);
     float4 *DU4 = reinterpret_cast<float4 *>(p.DU);
     const uint32_t n1p = p.negatives + 1u;
-    uint32_t draws = 0, redraws = 0;
+    const bool on = nr.sl < p.d4;
     for (uint32_t q = warp; q < nk; q += nwarps) {
         const uint32_t w = p.win[q];
-        const uint32_t left = w & 0xFFu, right = w >> 8;
-        if (left + right == 0) continue;
-        const uint32_t i = p.cidx[q];
-        float4 du = make_float4(0.f, 0.f, 0.f, 0.f);
-        unsigned long long gi = p.pair_off[q] * n1p;
-        for (uint32_t pp = q - left; pp <= q + right; ++pp) {
-            if (pp == q) continue;
-            const uint32_t w_out = (uint32_t)p.ctok[pp];
-            uint32_t n0, n1;
-            draw_pair_negatives(p, i, pp + p.window - q, w_out, nr.lane, n0, n1, draws, redraws);
-            for (uint32_t t0 = 0; t0 < n1p; t0 += TB * NG) {
-                float4 v[TB];
-                float g[TB];
+        const uint32_t cnt = (w & 0xFFu) + (w >> 8);
+        if (cnt == 0) continue;
+        const unsigned long long pair0 = p.pair_off[q];
+        const uint32_t nt = cnt * n1p;
+        float4 du = Narrow<GL>::zero();
+        for (uint32_t k0 = 0; k0 < nt; k0 += TB * NG) {
+            float4 v[TB];
+            float g[TB];
 #pragma unroll
-                for (int b = 0; b < TB; ++b) {
-                    const uint32_t t = t0 + b * NG + nr.grp;
-                    const uint32_t tgt = narrow_target(t, w_out, n0, n1, p.negatives);
-                    v[b] = nr.load(V4 + (size_t)tgt * p.ld4, p.d4, t < n1p);
-                    g[b] = t < n1p ? __ldcg(p.G + gi + t) : 0.f;
-                }
-#pragma unroll
-                for (int b = 0; b < TB; ++b) {
-                    du.x = fmaf(g[b], v[b].x, du.x); du.y = fmaf(g[b], v[b].y, du.y);
-                    du.z = fmaf(g[b], v[b].z, du.z); du.w = fmaf(g[b], v[b].w, du.w);
+            for (int b = 0; b < TB; ++b) {
+                const uint32_t k = k0 + b * NG + nr.grp;
+                v[b] = Narrow<GL>::zero();
+                g[b] = 0.f;
+                if (k < nt && on) {
+                    const uint32_t pr = k / n1p, t = k - pr * n1p;
+                    const uint32_t tgt = list_target(p, pair0 + pr, t);
+                    g[b] = __ldcg(p.G + pair0 * n1p + k);
+                    v[b] = __ldcg(V4 + (size_t)tgt * p.ld4 + nr.sl);
                 }
             }
-            gi += n1p;
+#pragma unroll
+            for (int b = 0; b < TB; ++b) {
+                du.x = fmaf(g[b], v[b].x, du.x); du.y = fmaf(g[b], v[b].y, du.y);
+                du.z = fmaf(g[b], v[b].z, du.z); du.w = fmaf(g[b], v[b].w, du.w);
+            }
         }
         du.x = Narrow<GL>::across_groups(du.x); du.y = Narrow<GL>::across_groups(du.y);
         du.z = Narrow<GL>::across_groups(du.z); du.w = Narrow<GL>::across_groups(du.w);
-        if (nr.grp == 0 && nr.sl < p.d4) DU4[(size_t)q * p.d4 + nr.sl] = du;
+        if (nr.grp == 0 && on) DU4[(size_t)q * p.d4 + nr.sl] = du;
     }
 }
 
-// pass 2 of the snapshot plan for narrow slices: v(target) += G u(c), several targets per warp
+// Algorithm 2, output rows: v(target) += G u(c) over the list, one group per target.
 template <int GL>
 __global__ void __launch_bounds__(kBlock)
-shard_adjust_v_narrow_kernel(StepParams p)
+shard_adjust_v_list_kernel(StepParams p)
 {
     const Narrow<GL> nr(threadIdx.x & 31);
-    constexpr int NG = Narrow<GL>::NG;
-    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
-    const uint32_t nk = (uint32_t)p.st->n_kept;
+    const unsigned long long n1p = p.negatives + 1u;
+    const unsigned long long total = p.st->pairs * n1p;
+    const unsigned long long group = ((unsigned long long)blockIdx.x * blockDim.x + threadIdx.x) / GL;
+    const unsigned long long ngroups = ((unsigned long long)gridDim.x * blockDim.x) / GL;
     const float4 *U4 = reinterpret_cast<const float4 *>(p.U);
     float4 *V4 = reinterpret_cast<float4 *>(p.V);
-    const uint32_t n1p = p.negatives + 1u;
-    uint32_t draws = 0, redraws = 0;
-    for (uint32_t q = warp; q < nk; q += nwarps) {
-        const uint32_t w = p.win[q];
-        const uint32_t left = w & 0xFFu, right = w >> 8;
-        if (left + right == 0) continue;
-        const uint32_t c = (uint32_t)p.ctok[q];
-        const uint32_t i = p.cidx[q];
-        const float4 u = nr.load(U4 + (size_t)c * p.ld4, p.d4, true);
-        unsigned long long gi = p.pair_off[q] * n1p;
-        for (uint32_t pp = q - left; pp <= q + right; ++pp) {
-            if (pp == q) continue;
-            const uint32_t w_out = (uint32_t)p.ctok[pp];
-            uint32_t n0, n1;
-            draw_pair_negatives(p, i, pp + p.window - q, w_out, nr.lane, n0, n1, draws, redraws);
-            for (uint32_t t0 = 0; t0 < n1p; t0 += NG) {
-                const uint32_t t = t0 + nr.grp;
-                const uint32_t tgt = narrow_target(t, w_out, n0, n1, p.negatives);
-                if (t < n1p && nr.sl < p.d4) {
-                    const float g = __ldcg(p.G + gi + t);
-                    if (tgt < p.hot_rows) {
-                        double *a = p.DV + (size_t)tgt * (4u * p.d4) + 4u * nr.sl;
-                        const double gd = (double)g;
-                        atomicAdd(a + 0, gd * (double)u.x); atomicAdd(a + 1, gd * (double)u.y);
-                        atomicAdd(a + 2, gd * (double)u.z); atomicAdd(a + 3, gd * (double)u.w);
-                    } else {
-                        red_add_f32x4(V4 + (size_t)tgt * p.ld4 + nr.sl, g * u.x, g * u.y, g * u.z, g * u.w);
-                    }
-                }
-            }
-            gi += n1p;
+    if (nr.sl >= p.d4) return;                      // no warp-wide operation below
+    for (unsigned long long j = group; j < total; j += ngroups) {
+        const unsigned long long pair = j / n1p;
+        const uint32_t t = (uint32_t)(j - pair * n1p);
+        const uint32_t c = (uint32_t)__ldg(p.l_centre + pair);
+        const uint32_t tgt = list_target(p, pair, t);
+        const float g = __ldcg(p.G + j);
+        const float4 u = __ldg(U4 + (size_t)c * p.ld4 + nr.sl);     // U is written only by pass 3
+        if (tgt < p.hot_rows) {
+            double *a = p.DV + (size_t)tgt * (4u * p.d4) + 4u * nr.sl;
+            const double gd = (double)g;
+            atomicAdd(a + 0, gd * (double)u.x); atomicAdd(a + 1, gd * (double)u.y);
+            atomicAdd(a + 2, gd * (double)u.z); atomicAdd(a + 3, gd * (double)u.w);
+        } else {
+            red_add_f32x4(V4 + (size_t)tgt * p.ld4 + nr.sl, g * u.x, g * u.y, g * u.z, g * u.w);
         }
     }
 }
@@ -361,11 +332,11 @@ static void shard_du_for(const StepParams &p, int sms, cudaStream_t s)
 int launch_shard_dots(const StepParams &p, const ShardPeers &peers, int sms, cudaStream_t s)
 {
     if (p.d4 <= 8) {
-        shard_dots_narrow_kernel<8, 2><<<shard_grid(shard_dots_narrow_kernel<8, 2>, sms), kBlock, 0, s>>>(p, peers);
+        shard_dots_list_kernel<8, 4><<<shard_grid(shard_dots_list_kernel<8, 4>, sms), kBlock, 0, s>>>(p, peers);
         return cudaGetLastError() != cudaSuccess ? -1 : 1;
     }
     if (p.d4 <= 16) {
-        shard_dots_narrow_kernel<16, 3><<<shard_grid(shard_dots_narrow_kernel<16, 3>, sms), kBlock, 0, s>>>(p, peers);
+        shard_dots_list_kernel<16, 4><<<shard_grid(shard_dots_list_kernel<16, 4>, sms), kBlock, 0, s>>>(p, peers);
         return cudaGetLastError() != cudaSuccess ? -1 : 1;
     }
 #define CALL_DOTS(V) shard_dots_for<V>(p, peers, sms, s)
@@ -398,11 +369,11 @@ int launch_shard_coefficients(const float *F, float *G, unsigned long long total
 int launch_shard_du(const StepParams &p, int sms, cudaStream_t s)
 {
     if (p.d4 <= 8) {
-        shard_du_narrow_kernel<8, 2><<<shard_grid(shard_du_narrow_kernel<8, 2>, sms), kBlock, 0, s>>>(p);
+        shard_du_list_kernel<8, 2><<<shard_grid(shard_du_list_kernel<8, 2>, sms), kBlock, 0, s>>>(p);
         return cudaGetLastError() != cudaSuccess ? -1 : 1;
     }
     if (p.d4 <= 16) {
-        shard_du_narrow_kernel<16, 3><<<shard_grid(shard_du_narrow_kernel<16, 3>, sms), kBlock, 0, s>>>(p);
+        shard_du_list_kernel<16, 3><<<shard_grid(shard_du_list_kernel<16, 3>, sms), kBlock, 0, s>>>(p);
         return cudaGetLastError() != cudaSuccess ? -1 : 1;
     }
 #define CALL_DU(V) shard_du_for<V>(p, sms, s)
@@ -425,9 +396,9 @@ int launch_shard_apply(const StepParams &p, uint32_t blocks_per_sm, int sms, cud
 {
     if (p.d4 > 16) return launch_snapshot_apply(p, blocks_per_sm, sms, s);
     if (p.d4 <= 8)
-        shard_adjust_v_narrow_kernel<8><<<shard_grid(shard_adjust_v_narrow_kernel<8>, sms), kBlock, 0, s>>>(p);
+        shard_adjust_v_list_kernel<8><<<shard_grid(shard_adjust_v_list_kernel<8>, sms), kBlock, 0, s>>>(p);
     else
-        shard_adjust_v_narrow_kernel<16><<<shard_grid(shard_adjust_v_narrow_kernel<16>, sms), kBlock, 0, s>>>(p);
+        shard_adjust_v_list_kernel<16><<<shard_grid(shard_adjust_v_list_kernel<16>, sms), kBlock, 0, s>>>(p);
     if (cudaGetLastError() != cudaSuccess) return -1;
     const int k = launch_snapshot_tail(p, blocks_per_sm, sms, s);
     return k < 0 ? -1 : 1 + k;
