@@ -20,7 +20,9 @@
  *     host memory.  The handle owns only its sampling tables and scratch.
  *   - All work is enqueued on the stream given to w2v_create.  Calls that
  *     return values to the host synchronise that stream; the others are
- *     asynchronous.
+ *     asynchronous.  A handle keeps per-step scratch and counters, so it must
+ *     not be used by two host threads at the same time; different handles
+ *     are independent.
  *   - Tables are row-major fp32: row w of U (input vectors) or V (output
  *     vectors) is d consecutive floats at offset w*d (w*row_stride for a model
  *     made by w2v_create_strided).  Row index = rank of the word by decreasing
