@@ -404,3 +404,25 @@ def test_host_token_entry_point_matches_device_entry_point():
         gpu.close()
     assert outs[0][0] == outs[1][0]
     assert row_rel_err(outs[1][1], outs[0][1]) <= 2e-6 and row_rel_err(outs[1][2], outs[0][2]) <= 2e-6
+
+
+def test_resume_from_saved_rows_and_step_number():
+    # vectors + step number are the whole training state: a model rebuilt from them continues exactly
+    cfg = corpus.scaled(TINY, vocab=3000, minibatch=2000, corpus_tokens=100_000)
+    gpu, cpu, cp = make_pair(cfg)
+    W, N, lr = cfg["window"], cfg["negatives"], cfg["lr"]
+    ids = np.arange(cfg["vocab"])
+    for i in range(2):
+        gpu.sgns_step(cp.chunk(i), W, N, lr, binding.MODE_SNAPSHOT)
+    saved_u, saved_v, saved_step = gpu.read_rows(0, ids), gpu.read_rows(1, ids), gpu.get_step()
+    for i in range(2, 4):
+        gpu.sgns_step(cp.chunk(i), W, N, lr, binding.MODE_SNAPSHOT)
+    again = binding.W2V(cfg["vocab"], cfg["d"], 11, row_stride=binding.aligned_row_stride(cfg["d"]))
+    again.build_alias(cp.counts, cfg["subsample_t"])
+    again.write_rows(0, ids, saved_u); again.write_rows(1, ids, saved_v); again.set_step(saved_step)
+    for i in range(2, 4):
+        again.sgns_step(cp.chunk(i), W, N, lr, binding.MODE_SNAPSHOT)
+    assert again.get_step() == gpu.get_step() == 4
+    assert row_rel_err(again.read_rows(0, ids), gpu.read_rows(0, ids)) <= 2e-6     # atomics' order only
+    assert row_rel_err(again.read_rows(1, ids), gpu.read_rows(1, ids)) <= 2e-6
+    gpu.close(); again.close()
