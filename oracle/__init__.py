@@ -65,6 +65,7 @@ def _load():
     L.orc_cbow_loss.argtypes = [vp, vp, u64, u32, u32, u64, vp, vp]
     L.orc_cbow_loss_examples.restype = C.c_double
     L.orc_cbow_loss_examples.argtypes = [vp, vp, vp, vp, vp, u64, u32]
+    L.orc_topk_cosine.argtypes = [vp, u32, vp, u64, u64, u64, u32, C.c_double, vp, vp]
     L.orc_rows_resident.restype = u64
     L.orc_rows_resident.argtypes = [vp, u32]
     _lib = L
@@ -267,6 +268,17 @@ class Oracle:
         return float(self.L.orc_cbow_loss_examples(self.h, centre.ctypes.data, negs.ctypes.data,
                                                    ctx_off.ctypes.data, ctx.ctypes.data, len(centre),
                                                    negs.shape[1]))
+
+    def topk_cosine(self, which, queries, cand_lo, cand_hi, K, tau):
+        """(ids[m, K] padded with -1, cosines[m, K]) of the K nearest candidate rows above tau."""
+        q = np.ascontiguousarray(queries, dtype=np.int64)
+        ids = np.empty((len(q), K), dtype=np.int64)
+        cs = np.empty((len(q), K), dtype=np.float64)
+        rc = self.L.orc_topk_cosine(self.h, int(which), q.ctypes.data, len(q), int(cand_lo), int(cand_hi), int(K),
+                                    float(tau), ids.ctypes.data, cs.ctypes.data)
+        if rc != 0:
+            raise ValueError("orc_topk_cosine rejected its arguments")
+        return ids, cs
 
     def rows_resident(self, which):
         return int(self.L.orc_rows_resident(self.h, which))

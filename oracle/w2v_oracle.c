@@ -42,6 +42,9 @@
  *                      Section 5: "readily extends to CBOW"): the mean of the
  *                      context words' input vectors predicts the centre word;
  *                      same index sets, same two modes, exact gradient.
+ *   orc_topk_cosine    retrieval by cosine similarity (Section 2: "the K queries
+ *                      with the highest similarity are retrieved"; Section 7.2:
+ *                      K nearest, kept only above a threshold tau): brute force.
  *   orc_partial_dots   u_s(w_I) v_s(w_O)^T of Algorithm 1 for one column slice.
  *   orc_loss           minus Eq. (1) restricted to a chunk, per positive pair.
  *
@@ -51,7 +54,8 @@
  * finite differences of Eq. (3); first-step closed form with V = 0; the
  * slice-sum identity of Algorithm 3 line "(F+,F-) <- sum_s"; hand-enumerated
  * windows; for CBOW: finite differences of its objective, the one-context case
- * that reduces to a skip-gram pair, and the first-step closed form.
+ * that reduces to a skip-gram pair, and the first-step closed form; for the
+ * retrieval: vectors with known angles, scale invariance, a full sort by numpy.
  * No function here is "parity unpinned".
  */
 #include <math.h>
@@ -930,6 +934,59 @@ double orc_cbow_loss_examples(orc *h, const int32_t *centre, const int32_t *negs
     cbow_run(h, NULL, 0, 0, N, 0, centre, negs, ctx_off, ctxs, E, cbow_loss_ex, &s);
     free(s.hbar);
     return -s.sum;
+}
+
+/* ------------------------------------------------------------------ */
+/* Retrieval by cosine similarity (Section 2; Section 7.2: K = 30 nearest */
+/* with cosine above tau = 0.65).  For every query row q the candidates   */
+/* are the rows cand_lo <= a < cand_hi, a != q; cos(q, a) = x_q.x_a /      */
+/* (|x_q| |x_a|) in fp64 (0 if either norm is 0).  Kept: cos > tau; of    */
+/* those the K largest, by decreasing cosine, ties by increasing id.       */
+/* out_ids is padded with -1 and out_cos with 0.                           */
+/* ------------------------------------------------------------------ */
+int orc_topk_cosine(orc *h, uint32_t which, const int64_t *queries, uint64_t m, uint64_t cand_lo,
+                    uint64_t cand_hi, uint32_t K, double tau, int64_t *out_ids, double *out_cos)
+{
+    if (which > 1 || K < 1 || cand_lo > cand_hi || cand_hi > h->vocab) return -1;
+    rowstore *rs = which ? &h->V : &h->U;
+    uint32_t d = h->d;
+    uint64_t nc = cand_hi - cand_lo;
+    double *norm = (double *)malloc((nc ? nc : 1) * sizeof(double));
+    for (uint64_t a = 0; a < nc; ++a) {
+        const float *x = rs_row(rs, h, cand_lo + a);
+        double s = 0.0;
+        for (uint32_t j = 0; j < d; ++j) s += (double)x[j] * (double)x[j];
+        norm[a] = sqrt(s);
+    }
+    for (uint64_t i = 0; i < m; ++i) {
+        int64_t *ids = out_ids + i * K;
+        double *cs = out_cos + i * K;
+        for (uint32_t k = 0; k < K; ++k) { ids[k] = -1; cs[k] = 0.0; }
+        int64_t q = queries[i];
+        if (q < 0 || (uint64_t)q >= h->vocab) continue;
+        const float *xq = rs_row(rs, h, (uint64_t)q);
+        double nq = 0.0;
+        for (uint32_t j = 0; j < d; ++j) nq += (double)xq[j] * (double)xq[j];
+        nq = sqrt(nq);
+        uint32_t have = 0;
+        for (uint64_t a = 0; a < nc; ++a) {
+            if ((int64_t)(cand_lo + a) == q) continue;
+            const float *xa = rs_row(rs, h, cand_lo + a);
+            double c = 0.0;
+            if (nq > 0.0 && norm[a] > 0.0) c = dot_rows(xq, xa, 0, d) / (nq * norm[a]);
+            if (!(c > tau)) continue;
+            /* insertion into the sorted list of the best K so far */
+            uint32_t pos = have;
+            while (pos > 0 && cs[pos - 1] < c) --pos;      /* equal cosine: the smaller id stays ahead */
+            if (pos >= K) continue;
+            uint32_t last = have < K ? have : K - 1;
+            for (uint32_t k = last; k > pos; --k) { cs[k] = cs[k - 1]; ids[k] = ids[k - 1]; }
+            cs[pos] = c; ids[pos] = (int64_t)(cand_lo + a);
+            if (have < K) ++have;
+        }
+    }
+    free(norm);
+    return 0;
 }
 
 uint64_t orc_rows_resident(const orc *h, uint32_t which)
