@@ -290,6 +290,24 @@ int32_t w2v_partial_dots(w2v_handle *h, const int32_t *pairs, uint64_t m, uint32
 int32_t w2v_read_rows(w2v_handle *h, uint32_t which, const int64_t *ids, uint64_t m, float *out);
 int32_t w2v_write_rows(w2v_handle *h, uint32_t which, const int64_t *ids, uint64_t m, const float *in);
 
+/*
+ * Retrieval by cosine similarity over the trained vectors (Section 2: "the K queries with the
+ * highest similarity are retrieved"; Section 7.2: K = 30 nearest, kept only above tau = 0.65).
+ * For every query row q: among the candidate rows cand_lo <= a < cand_hi, a != q, those with
+ * cos(q, a) = x_q.x_a / (|x_q| |x_a|) > tau (a zero row has cosine 0 with everything), and of
+ * these the K with the largest cosine, by decreasing cosine, equal cosines by increasing row.
+ *   which     W2V_TABLE_U or W2V_TABLE_V (the exported vectors are the input vectors, U).
+ *   queries   device, m int64 row numbers; one outside [0, vocab) gets an empty result.
+ *   K         1..64;  tau  any float (-2 keeps everything).
+ *   out_ids   device, m*K int64, padded with -1;  out_cos  device, m*K floats, padded with 0.
+ * Arithmetic is fp32 (cosines within about 1e-6 of exact).  Asynchronous except when scratch
+ * (1/|x| per candidate, partial lists) has to grow.  Errors: W2V_ERR_ARG, W2V_ERR_NOMEM,
+ * W2V_ERR_CUDA.  Reads the table as it is: call it between steps, not during one.
+ */
+int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, uint64_t m,
+                        uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, int64_t *out_ids,
+                        float *out_cos);
+
 /* Step number used by the next step (resume = write the rows back, set the step). */
 int32_t w2v_set_step(w2v_handle *h, uint64_t step_id);
 int32_t w2v_get_step(w2v_handle *h, uint64_t *step_id);

@@ -22,6 +22,8 @@ struct w2v_handle {
     bool shard_pending = false;
     int32_t *l_centre = nullptr, *l_context = nullptr, *l_negs = nullptr;   // pair list of a narrow shard's step
     uint64_t l_cap_pairs = 0, l_cap_negs = 0;
+    float *inv_norm = nullptr; uint64_t inv_norm_cap = 0;                      // retrieval scratch
+    float *part_cos = nullptr; long long *part_ids = nullptr; uint64_t part_cap = 0;
     uint32_t pend_window = 0, pend_negatives = 0;
     uint64_t pend_n = 0, pend_pairs = 0;
     uint64_t seed = 0;
@@ -396,6 +398,7 @@ int32_t w2v_destroy(w2v_handle *h)
     if (h->st_host) cudaFreeHost(h->st_host);
     cudaFree(h->G); cudaFree(h->DU); cudaFree(h->DV); cudaFree(h->tok_stage);
     cudaFree(h->l_centre); cudaFree(h->l_context); cudaFree(h->l_negs);
+    cudaFree(h->inv_norm); cudaFree(h->part_cos); cudaFree(h->part_ids);
     for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
     cudaGetLastError();
     delete h;
@@ -704,6 +707,53 @@ int32_t w2v_read_rows(w2v_handle *h, uint32_t which, const int64_t *ids, uint64_
 int32_t w2v_write_rows(w2v_handle *h, uint32_t which, const int64_t *ids, uint64_t m, const float *in)
 {
     return copy_rows(h, which, ids, m, const_cast<float *>(in), true);
+}
+
+int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, uint64_t m, uint64_t cand_lo,
+                        uint64_t cand_hi, uint32_t K, float tau, int64_t *out_ids, float *out_cos)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (which > 1) return fail(h, W2V_ERR_ARG, "which must be 0 (U) or 1 (V)");
+    if (K < 1 || K > 64) return fail(h, W2V_ERR_ARG, "K must be in 1..64");
+    if (!(cand_lo <= cand_hi && cand_hi <= h->vocab)) return fail(h, W2V_ERR_ARG, "need cand_lo <= cand_hi <= vocab");
+    if (m && (!queries || !out_ids || !out_cos)) return fail(h, W2V_ERR_ARG, "queries or an output array is NULL");
+    if (m >= (1ull << 31)) return fail(h, W2V_ERR_ARG, "m must be below 2^31");
+    if (m == 0) return W2V_OK;
+    DeviceGuard g(h->device);
+    const uint64_t nc = cand_hi - cand_lo;
+    if (nc > h->inv_norm_cap) {
+        W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+        cudaFree(h->inv_norm); h->inv_norm = nullptr; h->inv_norm_cap = 0;
+        W2V_CUDA(h, dev_alloc(&h->inv_norm, nc));
+        h->inv_norm_cap = nc;
+    }
+    // few query blocks: split the candidates over several blocks per query block, merge afterwards
+    const uint64_t qblocks = (m + 63) / 64, tiles = (nc + 127) / 128;
+    uint64_t splits = qblocks >= 2ull * h->sms ? 1 : (2ull * h->sms + qblocks - 1) / qblocks;
+    if (splits > 64) splits = 64;
+    if (splits > tiles) splits = tiles ? tiles : 1;
+    const uint64_t need = splits > 1 ? splits * m * K : 0;
+    if (need > h->part_cap) {
+        W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+        cudaFree(h->part_cos); cudaFree(h->part_ids); h->part_cos = nullptr; h->part_ids = nullptr; h->part_cap = 0;
+        W2V_CUDA(h, dev_alloc(&h->part_cos, need));
+        W2V_CUDA(h, dev_alloc(&h->part_ids, need));
+        h->part_cap = need;
+    }
+    const float *table = which ? h->V : h->U;
+    int32_t rc;
+    if ((rc = profile_mark(h)) != W2V_OK) return rc;
+    int k = launch_inv_norms(table, h->d, h->ld, cand_lo, nc, h->inv_norm, h->sms, h->stream);
+    if (k < 0) return fail(h, W2V_ERR_CUDA, "norm launch", cudaGetLastError());
+    int k2 = launch_topk(table, h->d, h->ld, h->vocab, reinterpret_cast<const long long *>(queries), m, cand_lo, cand_hi,
+                         K, tau, h->inv_norm, h->part_cos, h->part_ids, (uint32_t)splits, out_cos,
+                         reinterpret_cast<long long *>(out_ids), h->sms, h->stream);
+    if (k2 == -2) return fail(h, W2V_ERR_ARG, "d and K together exceed the shared memory of one block");
+    if (k2 < 0) return fail(h, W2V_ERR_CUDA, "retrieval launch", cudaGetLastError());
+    h->launches += (uint64_t)(k + k2);
+    if (h->profiling) h->prof_launches += (uint64_t)(k + k2);
+    if ((rc = profile_mark(h)) != W2V_OK) return rc;
+    return W2V_OK;
 }
 
 int32_t w2v_set_step(w2v_handle *h, uint64_t step_id)

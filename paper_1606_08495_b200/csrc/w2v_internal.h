@@ -133,6 +133,14 @@ int launch_partial_dots(const float *U, const float *V, uint32_t vocab, uint32_t
 int launch_copy_rows(float *table, uint32_t vocab, uint32_t d, uint32_t ld, const int64_t *ids, uint64_t m,
                      float *buf, bool to_table, int sms, cudaStream_t s);
 
+// ---- cosine retrieval (w2v_topk.cu) ----
+int launch_inv_norms(const float *table, uint32_t d, uint32_t ld, uint64_t lo, uint64_t count, float *inv_norm,
+                     int sms, cudaStream_t s);
+// Returns launches made, -1 on a launch error, -2 if the shape does not fit shared memory.
+int launch_topk(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, const long long *queries, uint64_t m,
+                uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, const float *inv_norm, float *part_cos,
+                long long *part_ids, uint32_t splits, float *out_cos, long long *out_ids, int sms, cudaStream_t s);
+
 // ---- host-side table construction (w2v_tables.cpp) ----
 // Returns 0, or -1 if a count is zero.  thr_alias is [vocab] pairs, keep_thr [vocab];
 // hot_prefix receives the number of leading rows that are drawn as negatives often enough to

@@ -1,0 +1,107 @@
+"""Cosine retrieval on the GPU against the CPU checker's brute force in fp64.
+
+Cosines must agree to 2e-6 (fp32 dot products of unit-scaled rows).  Where two candidates' exact
+cosines differ by less than that, either order is right, so ids are compared position by position
+only where the checker's neighbouring cosines are further apart, and otherwise through the value:
+the checker's cosine of the row the GPU returned must match the checker's cosine at that rank."""
+import numpy as np
+import pytest
+
+from oracle import Oracle
+from paper_1606_08495_b200 import binding
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-6
+
+
+def pair(V, d, seed, which=0, scale=1.0, row_stride=None, rows=None):
+    rng = np.random.default_rng(seed)
+    X = rng.normal(scale=scale, size=(V, d)).astype(np.float32) if rows is None else np.asarray(rows, dtype=np.float32)
+    gpu = binding.W2V(V, d, 1, row_stride=row_stride)
+    cpu = Oracle(V, d, 1)
+    ids = np.arange(V)
+    gpu.write_rows(which, ids, X); cpu.write_rows(which, ids, X)
+    return gpu, cpu, X
+
+
+def check(gpu, cpu, X, which, queries, lo, hi, K, tau):
+    gi, gc = gpu.topk_cosine(which, queries, lo, hi, K, tau)
+    wi, wc = cpu.topk_cosine(which, queries, lo, hi, K, tau)
+    assert gi.shape == wi.shape
+    Xd = X.astype(np.float64)
+    nrm = np.linalg.norm(Xd, axis=1)
+    for r, q in enumerate(np.asarray(queries)):
+        n_want = int((wi[r] >= 0).sum())
+        n_got = int((gi[r] >= 0).sum())
+        # the number kept can differ only through candidates within TOL of tau
+        if n_got != n_want:
+            k = min(n_got, n_want)
+            edge = wc[r][k] if n_want > n_got else None
+            assert n_want < K or n_got < K
+            assert edge is None or abs(edge - tau) <= TOL, (r, n_got, n_want)
+        for s in range(min(n_got, n_want)):
+            assert abs(gc[r, s] - wc[r, s]) <= TOL, (r, s, gc[r, s], wc[r, s])
+            if gi[r, s] != wi[r, s]:
+                a = gi[r, s]
+                exact = Xd[q] @ Xd[a] / (nrm[q] * nrm[a]) if nrm[q] > 0 and nrm[a] > 0 else 0.0
+                assert abs(exact - wc[r, s]) <= TOL and lo <= a < hi and a != q, (r, s)
+        assert np.all(gi[r, n_got:] == -1) and not gc[r, n_got:].any()
+        assert len(set(gi[r, :n_got].tolist())) == n_got
+    return gi, gc
+
+
+@pytest.mark.parametrize("V,d,K,m", [(3000, 300, 30, 200), (1000, 100, 5, 70), (5000, 64, 64, 10), (700, 4, 1, 700),
+                                     (900, 1024, 30, 40), (129, 132, 7, 129)])
+def test_topk_matches_brute_force(V, d, K, m):
+    gpu, cpu, X = pair(V, d, seed=V + d)
+    rng = np.random.default_rng(1)
+    q = rng.integers(0, V, m)
+    check(gpu, cpu, X, 0, q, 0, V, K, -2.0)
+    check(gpu, cpu, X, 0, q, V // 5, V - 7, K, 0.0)
+    gpu.close()
+
+
+def test_topk_threshold_of_the_paper_on_clustered_vectors():
+    # rows = cluster centre + noise, so that some neighbours are above tau = 0.65 and most are not
+    rng = np.random.default_rng(3)
+    V, d, C = 20_000, 300, 400
+    centres = rng.normal(size=(C, d))
+    X = (centres[rng.integers(0, C, V)] + 0.55 * rng.normal(size=(V, d))).astype(np.float32)
+    gpu, cpu, X = pair(V, d, 0, which=1, rows=X, row_stride=320)
+    q = rng.integers(0, V, 300)
+    gi, gc = check(gpu, cpu, X, 1, q, 5000, 20_000, 30, 0.65)
+    kept = (gi >= 0).sum(axis=1)
+    assert kept.max() == 30 and kept.min() < 30 and (gc[gi >= 0] > 0.65).all()
+    gpu.close()
+
+
+def test_topk_many_queries_few_candidates_and_edge_cases():
+    gpu, cpu, X = pair(5000, 32, seed=9, scale=3.0)
+    q = np.arange(5000)                                   # more query blocks than SMs: no candidate split
+    check(gpu, cpu, X, 0, q, 100, 150, 8, -2.0)
+    gi, gc = gpu.topk_cosine(0, [5, -1, 5000, 7], 0, 5000, 4, -2.0)
+    assert (gi[1] == -1).all() and (gi[2] == -1).all() and (gi[0] >= 0).all() and (gi[3] >= 0).all()
+    gi, gc = gpu.topk_cosine(0, [5], 10, 10, 4, -2.0)     # empty candidate range
+    assert (gi == -1).all() and not gc.any()
+    gi, gc = gpu.topk_cosine(0, [5], 5, 6, 4, -2.0)       # the only candidate is the query itself
+    assert (gi == -1).all()
+    for args in ((2, [1], 0, 10, 4, 0.0), (0, [1], 0, 10, 0, 0.0), (0, [1], 0, 10, 65, 0.0), (0, [1], 5, 4, 4, 0.0),
+                 (0, [1], 0, 5001, 4, 0.0)):
+        with pytest.raises(binding.W2VError) as e:
+            gpu.topk_cosine(*args)
+        assert e.value.code == binding.W2V_ERR_ARG
+    gpu.close()
+
+
+def test_topk_zero_rows_and_exact_ties():
+    rows = np.zeros((200, 8), dtype=np.float32)
+    rows[:, 0] = 1.0                                      # every row the same direction: all cosines 1
+    rows[50] = 0.0                                        # a zero row: cosine 0 with everything
+    rows[100:, 0] = np.arange(100, 200)                   # other lengths, same direction
+    gpu, cpu, X = pair(200, 8, 0, rows=rows)
+    gi, gc = gpu.topk_cosine(0, [0, 50, 150], 0, 200, 6, -2.0)
+    wi, wc = cpu.topk_cosine(0, [0, 50, 150], 0, 200, 6, -2.0)
+    assert np.array_equal(gi, wi)                         # ties go to the smaller row number
+    assert np.allclose(gc, wc, atol=TOL)
+    gpu.close()
