@@ -457,6 +457,89 @@ def run_sharded(args):
     model.close()
 
 
+def run_topk(args):
+    """Retrieval by cosine similarity (Section 2 / Section 7.2): K = 30 nearest above tau = 0.65 for a
+    batch of query rows among the last 15 % of the vocabulary (the share of the ad ids in the
+    sponsored-search-shaped workload).  One step = one w2v_topk_cosine call."""
+    import torch
+
+    from paper_1606_08495_b200 import binding
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    name = args.workload or "sponsored"
+    cfg = corpus.CONFIGS[name]
+    V, d = cfg["vocab"], cfg["d"]
+    K, tau, m = 30, 0.65, args.queries
+    lo, hi = int(V * 0.85), V
+    model = binding.W2V(V, d, seed=1, device=dev, row_stride=row_stride_for(d, args.row_stride))
+    # spread-out vectors instead of the tiny uniform initial ones: normal rows, so that cosines have the
+    # spread of unrelated trained vectors (about N(0, 1/d)); written by torch, this is input data
+    g = torch.Generator(device=dev); g.manual_seed(5)
+    Uv = model.U.view(V, model.row_stride)
+    for a in range(0, V, 1 << 20):
+        b = min(V, a + (1 << 20))
+        Uv[a:b, :d] = torch.randn(b - a, d, generator=g, device=dev)
+    q = torch.randint(0, V, (m,), generator=g, device=dev, dtype=torch.int64)
+    ids = torch.empty(m * K, dtype=torch.int64, device=dev)
+    cs = torch.empty(m * K, dtype=torch.float32, device=dev)
+    Ksteps, Wu = args.steps, args.warmup
+    for _ in range(Wu):
+        binding.w2v_topk_cosine(model.h, 0, q, m, lo, hi, K, tau, ids, cs)
+    model.sync()
+    binding.w2v_profile_enable(model.h, True)
+    launches0 = model.launch_count()
+    sampler = ClockSampler(physical_gpu_index(0))
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    sampler.start()
+    ev0.record()
+    for _ in range(Ksteps):
+        binding.w2v_topk_cosine(model.h, 0, q, m, lo, hi, K, tau, ids, cs)
+    ev1.record()
+    torch.cuda.synchronize(dev)
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1)
+    kernel_ms, _ = binding.w2v_profile_read(model.h)
+    launches = model.launch_count() - launches0
+    # end to end: query ids from pinned host memory, results back to the host
+    qh = q.cpu().pin_memory()
+    ids_h = torch.empty(m * K, dtype=torch.int64).pin_memory()
+    cs_h = torch.empty(m * K, dtype=torch.float32).pin_memory()
+    ev2, ev3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev2.record()
+    for _ in range(Ksteps):
+        q.copy_(qh, non_blocking=True)
+        binding.w2v_topk_cosine(model.h, 0, q, m, lo, hi, K, tau, ids, cs)
+        ids_h.copy_(ids, non_blocking=True); cs_h.copy_(cs, non_blocking=True)
+    ev3.record()
+    torch.cuda.synchronize(dev)
+    e2e_ms = ev2.elapsed_time(ev3)
+    cosines = float(m) * (hi - lo) * Ksteps
+    flops = 2.0 * d * cosines
+    sm_mhz = clocks.get("sm_max_mhz") or 1965.0
+    peak = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12          # fp32 FMA lanes x 2 flop x clock, TFLOP/s
+    achieved = flops / (kernel_ms * 1e-3) / 1e12 if kernel_ms > 0 else 0.0
+    line = {
+        "metric": "cosine_similarities_per_sec", "value": cosines / (ms * 1e-3), "unit": "cosines/s", "n_gpus": 1,
+        "steps": Ksteps, "warmup": Wu, "ms_per_step": ms / Ksteps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": name + " (retrieval)", "vocab": V, "d": d, "queries_per_step": m,
+                   "candidates": hi - lo, "K": K, "tau": tau, "row_stride_floats": model.row_stride,
+                   "l2": "3 M candidate rows (3.8 GB) streamed per call, far larger than L2"},
+        "clocks": clocks,
+        "e2e": {"value": cosines / (e2e_ms * 1e-3), "unit": "cosines/s", "h2d_bytes_per_step": 8 * m,
+                "d2h_bytes_per_step": 12 * m * K},
+        "gpu_launches": launches,
+        "roofline": {"bound": "alu", "kernel": "topk_cosine_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "TFLOP/s", "frac": achieved / peak,
+                     "peak_kind": "148 SMs x 128 fp32 FMA lanes x 2 flop x max SM clock",
+                     "flops_per_launch": flops / Ksteps, "kernel_ms_per_launch": kernel_ms / Ksteps, "traffic": None},
+    }
+    print(json.dumps(line), flush=True)
+    model.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -472,7 +555,8 @@ def main():
     ap.add_argument("--cpu-words", type=int, default=150_000, help="word tokens in the cpu_baseline sample")
     ap.add_argument("--ref-words", type=int, default=20_000, help="word tokens per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--mode", choices=["hogwild", "snapshot", "sharded"], default="hogwild",
+    ap.add_argument("--queries", type=int, default=8192, help="query rows per call of --mode topk")
+    ap.add_argument("--mode", choices=["hogwild", "snapshot", "sharded", "topk"], default="hogwild",
                     help="update mode of the timed steps (the headline number is hogwild); sharded = the "
                          "paper's column partition, --shards slices of one model on one GPU")
     ap.add_argument("--shards", type=int, default=8)
@@ -490,6 +574,8 @@ def main():
         run_reference(args)
     elif args.mode == "sharded":
         run_sharded(args)
+    elif args.mode == "topk":
+        run_topk(args)
     else:
         run_gpu(args)
 

@@ -728,10 +728,7 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
         h->inv_norm_cap = nc;
     }
     // few query blocks: split the candidates over several blocks per query block, merge afterwards
-    const uint64_t qblocks = (m + 63) / 64, tiles = (nc + 127) / 128;
-    uint64_t splits = qblocks >= 2ull * h->sms ? 1 : (2ull * h->sms + qblocks - 1) / qblocks;
-    if (splits > 64) splits = 64;
-    if (splits > tiles) splits = tiles ? tiles : 1;
+    const uint64_t splits = topk_splits(m, nc, h->sms);
     const uint64_t need = splits > 1 ? splits * m * K : 0;
     if (need > h->part_cap) {
         W2V_CUDA(h, cudaStreamSynchronize(h->stream));

@@ -134,6 +134,7 @@ int launch_copy_rows(float *table, uint32_t vocab, uint32_t d, uint32_t ld, cons
                      float *buf, bool to_table, int sms, cudaStream_t s);
 
 // ---- cosine retrieval (w2v_topk.cu) ----
+uint32_t topk_splits(uint64_t m, uint64_t n_candidates, int sms);
 int launch_inv_norms(const float *table, uint32_t d, uint32_t ld, uint64_t lo, uint64_t count, float *inv_norm,
                      int sms, cudaStream_t s);
 // Returns launches made, -1 on a launch error, -2 if the shape does not fit shared memory.

@@ -3,7 +3,7 @@
 // similarity are retrieved"; Section 7.2: K = 30 nearest, kept only above tau = 0.65).
 //
 // For a block of BQ query rows the kernel streams the candidate rows in tiles of BC, forms the
-// BQ x BC dot products in registers (a 16 x 16 thread grid, each thread a (BQ/16) x 8 patch; both
+// BQ x BC dot products in registers (a 16 x 32 thread grid, each thread (BQ/16) x 8 of them; both
 // operands staged through shared memory, k-major), scales them by the inverse norms and feeds the
 // ones that can still enter a query's list into that query's sorted top-K list in shared memory.
 // All arithmetic is fp32 on the CUDA cores: cosines agree with a double-precision evaluation to
@@ -13,11 +13,12 @@
 
 namespace w2v {
 
-constexpr int kTopkBC = 128;          // candidate rows per tile
+constexpr int kTopkBC = 256;          // candidate rows per tile
 constexpr int kTopkKC = 16;           // columns per shared-memory chunk
 constexpr int kTopkPad = 4;           // keeps 16-byte alignment of the k-major rows
-constexpr int kTopkThreads = 256;
-constexpr int kTopkPush = 16;         // at most 16 threads offer a candidate to one query per round
+constexpr int kTopkThreads = 512;     // 16 query groups x 32 candidate groups
+constexpr int kTopkTX = 32;           // threads along the candidates
+constexpr int kTopkPush = kTopkTX;    // at most one offer per candidate thread to a query per round
 
 // 1 / |x| per candidate row (0 for a zero row): one warp per row.
 __global__ void __launch_bounds__(kBlock)
@@ -95,11 +96,13 @@ topk_cosine_kernel(TopkParams p)
     constexpr int TQ = BQ / 16;                              // query rows per thread
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t d = 4u * p.d4;
-    // layout: Qs[d][BQ] | Cs[KC][BC+pad] | list_sc[BQ][K] | list_id[BQ][K] | push_c[BQ][16] | push_i[BQ][16]
+    // layout: Qs[nch*KC][BQ] | Cs[2][KC][BC+pad] | list_sc[BQ][K] | list_id[BQ][K] | push_c[BQ][16] | push_i[BQ][16]
     //         | qinv[BQ] | thr[BQ] | have[BQ] | npush[BQ] | qrow[BQ]
+    const uint32_t nch = (d + kTopkKC - 1) / kTopkKC;       // column chunks; Qs is zero-padded to nch * KC rows
     float *Qs = reinterpret_cast<float *>(smem_raw);
-    float *Cs = Qs + (size_t)d * BQ;
-    long long *list_id = reinterpret_cast<long long *>(Cs + kTopkKC * (kTopkBC + kTopkPad));
+    float *Cs = Qs + (size_t)nch * kTopkKC * BQ;            // two buffers of KC x (BC + pad)
+    constexpr int kCsBuf = kTopkKC * (kTopkBC + kTopkPad);
+    long long *list_id = reinterpret_cast<long long *>(Cs + 2 * kCsBuf);
     long long *push_i = list_id + (size_t)BQ * p.K;
     long long *qrow = push_i + BQ * kTopkPush;
     float *list_sc = reinterpret_cast<float *>(qrow + BQ);
@@ -110,7 +113,7 @@ topk_cosine_kernel(TopkParams p)
     uint32_t *npush = have + BQ;
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    const uint32_t tx = tid & 15, ty = tid >> 4;
+    const uint32_t tx = tid & (kTopkTX - 1), ty = tid / kTopkTX;
     const uint64_t q0 = (uint64_t)blockIdx.x * BQ;
     // this block's share of the candidates: whole tiles
     const uint64_t nc = p.cand_hi - p.cand_lo;
@@ -131,6 +134,7 @@ topk_cosine_kernel(TopkParams p)
         Qs[(4 * j4 + 0) * BQ + i] = x.x; Qs[(4 * j4 + 1) * BQ + i] = x.y;
         Qs[(4 * j4 + 2) * BQ + i] = x.z; Qs[(4 * j4 + 3) * BQ + i] = x.w;
     }
+    for (uint32_t e = d * BQ + tid; e < nch * kTopkKC * BQ; e += kTopkThreads) Qs[e] = 0.f;
     __syncthreads();
     for (uint32_t i = wid; i < (uint32_t)BQ; i += kTopkThreads / 32) {
         float s = 0.f;
@@ -140,53 +144,88 @@ topk_cosine_kernel(TopkParams p)
     }
     __syncthreads();
 
-    for (uint64_t tile = t_lo; tile < t_hi; ++tile) {
-        const uint64_t c0 = tile * kTopkBC;                  // first candidate of the tile (relative)
-        float acc[TQ][8];
+    // Candidate columns are staged chunk by chunk (KC columns of BC rows, transposed); the global
+    // loads of chunk g+1 are in flight while chunk g is multiplied.
+    constexpr int kRep = (kTopkBC * kTopkKC / 4) / kTopkThreads;
+    const uint64_t total_g = (t_hi - t_lo) * nch;
+    auto gload = [&](uint64_t tile, uint32_t chunk, float4 (&x)[kRep]) {
+        const uint64_t c0 = tile * kTopkBC;
+        const uint32_t k0 = chunk * kTopkKC;
 #pragma unroll
-        for (int a = 0; a < TQ; ++a)
-#pragma unroll
-            for (int b = 0; b < 8; ++b) acc[a][b] = 0.f;
-        for (uint32_t k0 = 0; k0 < d; k0 += kTopkKC) {
-            // stage candidate columns k0 .. k0+KC of the tile, transposed
-            __syncthreads();
-#pragma unroll
-            for (int rep = 0; rep < (kTopkBC * kTopkKC / 4) / kTopkThreads; ++rep) {
-                const uint32_t f = tid + rep * kTopkThreads;
-                const uint32_t row = f / (kTopkKC / 4), kq = f % (kTopkKC / 4);
-                float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (c0 + row < nc && k0 + 4 * kq < d)
-                    x = __ldcg(reinterpret_cast<const float4 *>(p.table) + (size_t)(p.cand_lo + c0 + row) * p.ld4 +
-                               (k0 / 4 + kq));
-                float *dst = Cs + (4 * kq) * (kTopkBC + kTopkPad) + row;
-                dst[0] = x.x; dst[kTopkBC + kTopkPad] = x.y;
-                dst[2 * (kTopkBC + kTopkPad)] = x.z; dst[3 * (kTopkBC + kTopkPad)] = x.w;
-            }
-            __syncthreads();
-            const uint32_t kn = d - k0 < (uint32_t)kTopkKC ? d - k0 : (uint32_t)kTopkKC;
-            for (uint32_t k = 0; k < kn; ++k) {
-                float qv[TQ];
-#pragma unroll
-                for (int a = 0; a < TQ; ++a) qv[a] = Qs[(k0 + k) * BQ + ty * TQ + a];
-                const float4 c_lo = *reinterpret_cast<const float4 *>(Cs + k * (kTopkBC + kTopkPad) + tx * 8);
-                const float4 c_hi = *reinterpret_cast<const float4 *>(Cs + k * (kTopkBC + kTopkPad) + tx * 8 + 4);
-                const float cv[8] = {c_lo.x, c_lo.y, c_lo.z, c_lo.w, c_hi.x, c_hi.y, c_hi.z, c_hi.w};
-#pragma unroll
-                for (int a = 0; a < TQ; ++a)
-#pragma unroll
-                    for (int b = 0; b < 8; ++b) acc[a][b] = fmaf(qv[a], cv[b], acc[a][b]);
-            }
+        for (int rep = 0; rep < kRep; ++rep) {
+            const uint32_t f = tid + rep * kTopkThreads;
+            const uint32_t row = f / (kTopkKC / 4), kq = f % (kTopkKC / 4);
+            x[rep] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c0 + row < nc && k0 + 4 * kq < d)
+                x[rep] = __ldcg(reinterpret_cast<const float4 *>(p.table) + (size_t)(p.cand_lo + c0 + row) * p.ld4 +
+                                (k0 / 4 + kq));
         }
+    };
+    auto sstore = [&](float *buf, const float4 (&x)[kRep]) {
+#pragma unroll
+        for (int rep = 0; rep < kRep; ++rep) {
+            const uint32_t f = tid + rep * kTopkThreads;
+            const uint32_t row = f / (kTopkKC / 4), kq = f % (kTopkKC / 4);
+            float *dst = buf + (4 * kq) * (kTopkBC + kTopkPad) + row;
+            dst[0] = x[rep].x; dst[kTopkBC + kTopkPad] = x[rep].y;
+            dst[2 * (kTopkBC + kTopkPad)] = x[rep].z; dst[3 * (kTopkBC + kTopkPad)] = x[rep].w;
+        }
+    };
+    float acc[TQ][8];
+    {
+        float4 x0[kRep];
+        if (total_g) { gload(t_lo, 0, x0); sstore(Cs, x0); }
+    }
+    __syncthreads();
+    uint64_t tile = t_lo;
+    uint32_t chunk = 0;
+    for (uint64_t g = 0; g < total_g; ++g, ++chunk) {
+        if (chunk == nch) { chunk = 0; ++tile; }
+        const uint64_t c0 = tile * kTopkBC;                      // first candidate of the tile (relative)
+        const float *cbuf = Cs + (g & 1) * kCsBuf;
+        float4 xn[kRep];
+        const bool more = g + 1 < total_g;
+        if (more) gload(chunk + 1 == nch ? tile + 1 : tile, chunk + 1 == nch ? 0u : chunk + 1, xn);
+        if (chunk == 0) {
+#pragma unroll
+            for (int a = 0; a < TQ; ++a)
+#pragma unroll
+                for (int b = 0; b < 8; ++b) acc[a][b] = 0.f;
+        }
+        const float *qbase = Qs + (size_t)chunk * kTopkKC * BQ + ty * TQ;
+#pragma unroll
+        for (int k = 0; k < kTopkKC; ++k) {
+            float qv[TQ];
+            if constexpr (TQ == 4) {
+                const float4 q4 = *reinterpret_cast<const float4 *>(qbase + k * BQ);
+                qv[0] = q4.x; qv[1] = q4.y; qv[2] = q4.z; qv[3] = q4.w;
+            } else {
+#pragma unroll
+                for (int a = 0; a < TQ; ++a) qv[a] = qbase[k * BQ + a];
+            }
+            // a thread's 8 candidates are columns 4 tx .. 4 tx + 3 and BC/2 + 4 tx .. : the threads
+            // of a warp read 512 contiguous bytes per load, without bank conflicts
+            const float4 c_lo = *reinterpret_cast<const float4 *>(cbuf + k * (kTopkBC + kTopkPad) + tx * 4);
+            const float4 c_hi = *reinterpret_cast<const float4 *>(cbuf + k * (kTopkBC + kTopkPad) + kTopkBC / 2 + tx * 4);
+            const float cv[8] = {c_lo.x, c_lo.y, c_lo.z, c_lo.w, c_hi.x, c_hi.y, c_hi.z, c_hi.w};
+#pragma unroll
+            for (int a = 0; a < TQ; ++a)
+#pragma unroll
+                for (int b = 0; b < 8; ++b) acc[a][b] = fmaf(qv[a], cv[b], acc[a][b]);
+        }
+        if (more) sstore(Cs + ((g + 1) & 1) * kCsBuf, xn);
+        __syncthreads();
+        if (chunk != nch - 1) continue;
         // ---- cosines; offer what can still enter a list, one candidate column per round ----
         float inv_c[8];
 #pragma unroll
         for (int b = 0; b < 8; ++b) {
-            const uint64_t c = c0 + tx * 8 + b;
+            const uint64_t c = c0 + (b < 4 ? tx * 4 + b : kTopkBC / 2 + tx * 4 + (b - 4));
             inv_c[b] = c < nc ? p.inv_norm[c] : 0.f;
         }
 #pragma unroll
         for (int b = 0; b < 8; ++b) {
-            const uint64_t c = c0 + tx * 8 + b;
+            const uint64_t c = c0 + (b < 4 ? tx * 4 + b : kTopkBC / 2 + tx * 4 + (b - 4));
             const long long cid = (long long)(p.cand_lo + c);
             int pushed = 0;
 #pragma unroll
@@ -194,7 +233,7 @@ topk_cosine_kernel(TopkParams p)
                 const uint32_t i = ty * TQ + a;
                 const float cs = acc[a][b] * qinv[i] * inv_c[b];
                 if (c < nc && qrow[i] >= 0 && cid != qrow[i] && cs > p.tau && (have[i] < p.K || cs >= thr[i])) {
-                    const uint32_t slot = atomicAdd(&npush[i], 1u);      // < 16: one offer per tx thread
+                    const uint32_t slot = atomicAdd(&npush[i], 1u);      // < kTopkPush: one offer per tx thread
                     push_c[i * kTopkPush + slot] = cs;
                     push_i[i * kTopkPush + slot] = cid;
                     pushed = 1;
@@ -263,10 +302,29 @@ topk_merge_kernel(const float *__restrict__ part_cos, const long long *__restric
 // ---- launchers --------------------------------------------------------------------------------
 size_t topk_smem_bytes(uint32_t d, uint32_t K, int BQ)
 {
-    size_t b = (size_t)d * BQ * 4 + (size_t)kTopkKC * (kTopkBC + kTopkPad) * 4;     // Qs, Cs
+    const size_t nch = (d + kTopkKC - 1) / kTopkKC;
+    size_t b = nch * kTopkKC * BQ * 4 + 2 * (size_t)kTopkKC * (kTopkBC + kTopkPad) * 4;  // Qs (padded), two Cs
     b += (size_t)BQ * K * 8 + (size_t)BQ * kTopkPush * 8 + (size_t)BQ * 8;          // list_id, push_i, qrow
     b += (size_t)BQ * K * 4 + (size_t)BQ * kTopkPush * 4 + (size_t)BQ * 4 * 4;      // list_sc, push_c, qinv/thr/have/npush
     return b;
+}
+
+// How many ways to split the candidates so that the grid fills whole waves of one block per SM:
+// the smallest split count (at most 64, at most one per tile) whose last wave is at least 95 % full,
+// else the fullest one.
+uint32_t topk_splits(uint64_t m, uint64_t n_candidates, int sms)
+{
+    const uint64_t qblocks = (m + 63) / 64, tiles = (n_candidates + kTopkBC - 1) / kTopkBC;
+    uint64_t max_s = tiles < 64 ? (tiles ? tiles : 1) : 64;
+    uint32_t best = 1;
+    double best_fill = 0.0;
+    for (uint64_t sp = 1; sp <= max_s; ++sp) {
+        const uint64_t blocks = qblocks * sp, waves = (blocks + sms - 1) / sms;
+        const double fill = (double)blocks / (double)(waves * sms);
+        if (fill > best_fill + 1e-9) { best_fill = fill; best = (uint32_t)sp; }
+        if (fill >= 0.95) return (uint32_t)sp;
+    }
+    return best;
 }
 
 int launch_inv_norms(const float *table, uint32_t d, uint32_t ld, uint64_t lo, uint64_t count, float *inv_norm,
