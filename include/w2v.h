@@ -308,6 +308,16 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
                         uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, int64_t *out_ids,
                         float *out_cos);
 
+/*
+ * Which kernel w2v_topk_cosine runs (the paper has no say in this):
+ *   0  fp32 multiply-adds on the CUDA cores (the default);
+ *   1  the tensor cores: every value is split into a TF32 head and a TF32 tail and each product is
+ *      formed as head*head + head*tail + tail*head in fp32 accumulators, which keeps cosines
+ *      within about 1e-6 of exact at several times the speed.  A block of this kernel that waits
+ *      too long on its own pipeline gives up; w2v_sync then returns W2V_ERR_CUDA.
+ */
+int32_t w2v_set_retrieval_kernel(w2v_handle *h, uint32_t kind);
+
 /* Step number used by the next step (resume = write the rows back, set the step). */
 int32_t w2v_set_step(w2v_handle *h, uint64_t step_id);
 int32_t w2v_get_step(w2v_handle *h, uint64_t *step_id);

@@ -22,7 +22,7 @@ TABLE_U, TABLE_V = 0, 1
 EXPORTS = (
     "w2v_create", "w2v_create_strided", "w2v_create_shard", "w2v_shard_dots", "w2v_shard_adjust",
     "w2v_get_row_stride", "w2v_set_interleave", "w2v_cbow_step", "w2v_cbow_step_host", "w2v_sample_cbow",
-    "w2v_topk_cosine", "w2v_destroy", "w2v_build_alias", "w2v_get_tables", "w2v_sgns_step",
+    "w2v_topk_cosine", "w2v_set_retrieval_kernel", "w2v_destroy", "w2v_build_alias", "w2v_get_tables", "w2v_sgns_step",
     "w2v_sgns_step_host", "w2v_sample_pairs", "w2v_partial_dots", "w2v_read_rows", "w2v_write_rows",
     "w2v_set_step", "w2v_get_step", "w2v_get_table_ptrs", "w2v_sync", "w2v_profile_enable",
     "w2v_profile_read", "w2v_get_launch_count", "w2v_set_tuning", "w2v_last_error",
@@ -85,6 +85,7 @@ def load():
         "w2v_read_rows": [vp, u32, vp, u64, vp],
         "w2v_write_rows": [vp, u32, vp, u64, vp],
         "w2v_topk_cosine": [vp, u32, vp, u64, u64, u64, u32, C.c_float, vp, vp],
+        "w2v_set_retrieval_kernel": [vp, u32],
         "w2v_set_step": [vp, u64],
         "w2v_set_interleave": [vp, u32, u32],
         "w2v_get_step": [vp, C.POINTER(u64)],
@@ -245,6 +246,10 @@ def w2v_write_rows(h, which, ids, m, rows):
 def w2v_topk_cosine(h, which, queries, m, cand_lo, cand_hi, K, tau, out_ids, out_cos):
     return _check(h, load().w2v_topk_cosine(h, int(which), _ptr(queries), int(m), int(cand_lo), int(cand_hi), int(K),
                                             float(tau), _ptr(out_ids), _ptr(out_cos)))
+
+
+def w2v_set_retrieval_kernel(h, kind):
+    return _check(h, load().w2v_set_retrieval_kernel(h, int(kind)))
 
 
 def w2v_set_step(h, step_id):

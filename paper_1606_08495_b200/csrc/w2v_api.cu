@@ -24,6 +24,8 @@ struct w2v_handle {
     uint64_t l_cap_pairs = 0, l_cap_negs = 0;
     float *inv_norm = nullptr; uint64_t inv_norm_cap = 0;                      // retrieval scratch
     float *part_cos = nullptr; long long *part_ids = nullptr; uint64_t part_cap = 0;
+    uint32_t retrieval_kernel = 0;       // 0: fp32 on the CUDA cores, 1: tensor cores (3 x TF32)
+    int *tc_error = nullptr;             // device word raised by a tensor-core block whose wait ran out
     uint32_t pend_window = 0, pend_negatives = 0;
     uint64_t pend_n = 0, pend_pairs = 0;
     uint64_t seed = 0;
@@ -398,7 +400,7 @@ int32_t w2v_destroy(w2v_handle *h)
     if (h->st_host) cudaFreeHost(h->st_host);
     cudaFree(h->G); cudaFree(h->DU); cudaFree(h->DV); cudaFree(h->tok_stage);
     cudaFree(h->l_centre); cudaFree(h->l_context); cudaFree(h->l_negs);
-    cudaFree(h->inv_norm); cudaFree(h->part_cos); cudaFree(h->part_ids);
+    cudaFree(h->inv_norm); cudaFree(h->part_cos); cudaFree(h->part_ids); cudaFree(h->tc_error);
     for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
     cudaGetLastError();
     delete h;
@@ -728,8 +730,13 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
         h->inv_norm_cap = nc;
     }
     // few query blocks: split the candidates over several blocks per query block, merge afterwards
-    const uint64_t splits = topk_splits(m, nc, h->sms);
-    const uint64_t need = splits > 1 ? splits * m * K : 0;
+    const bool tc = h->retrieval_kernel == 1;
+    const uint64_t splits = tc ? topk_splits(m, nc, h->sms, 128, 128) : topk_splits(m, nc, h->sms);
+    const uint64_t need = (splits > 1 || tc) ? splits * m * K : 0;
+    if (tc && !h->tc_error) {
+        W2V_CUDA(h, dev_alloc(&h->tc_error, 1));
+        W2V_CUDA(h, cudaMemsetAsync(h->tc_error, 0, sizeof(int), h->stream));
+    }
     if (need > h->part_cap) {
         W2V_CUDA(h, cudaStreamSynchronize(h->stream));
         cudaFree(h->part_cos); cudaFree(h->part_ids); h->part_cos = nullptr; h->part_ids = nullptr; h->part_cap = 0;
@@ -742,9 +749,21 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
     if ((rc = profile_mark(h)) != W2V_OK) return rc;
     int k = launch_inv_norms(table, h->d, h->ld, cand_lo, nc, h->inv_norm, h->sms, h->stream);
     if (k < 0) return fail(h, W2V_ERR_CUDA, "norm launch", cudaGetLastError());
-    int k2 = launch_topk(table, h->d, h->ld, h->vocab, reinterpret_cast<const long long *>(queries), m, cand_lo, cand_hi,
+    int k2;
+    if (tc) {
+        k2 = launch_topk_tc(table, h->d, h->ld, h->vocab, reinterpret_cast<const long long *>(queries), m, cand_lo,
+                            cand_hi, K, tau, h->inv_norm, h->part_cos, h->part_ids, (uint32_t)splits, h->tc_error,
+                            h->stream);
+        if (k2 >= 0) {
+            const int k3 = launch_topk_merge(h->part_cos, h->part_ids, m, K, (uint32_t)splits, out_cos,
+                                             reinterpret_cast<long long *>(out_ids), h->sms, h->stream);
+            k2 = k3 < 0 ? -1 : k2 + k3;
+        }
+    } else {
+        k2 = launch_topk(table, h->d, h->ld, h->vocab, reinterpret_cast<const long long *>(queries), m, cand_lo, cand_hi,
                          K, tau, h->inv_norm, h->part_cos, h->part_ids, (uint32_t)splits, out_cos,
                          reinterpret_cast<long long *>(out_ids), h->sms, h->stream);
+    }
     if (k2 == -2) return fail(h, W2V_ERR_ARG, "d and K together exceed the shared memory of one block");
     if (k2 < 0) return fail(h, W2V_ERR_CUDA, "retrieval launch", cudaGetLastError());
     h->launches += (uint64_t)(k + k2);
@@ -797,6 +816,22 @@ int32_t w2v_sync(w2v_handle *h)
     if (!h) return W2V_ERR_ARG;
     DeviceGuard g(h->device);
     W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+    if (h->tc_error) {
+        int flag = 0;
+        W2V_CUDA(h, cudaMemcpy(&flag, h->tc_error, sizeof(int), cudaMemcpyDeviceToHost));
+        if (flag) {
+            W2V_CUDA(h, cudaMemset(h->tc_error, 0, sizeof(int)));
+            return fail(h, W2V_ERR_CUDA, "a tensor-core retrieval block gave up waiting; its results are incomplete");
+        }
+    }
+    return W2V_OK;
+}
+
+int32_t w2v_set_retrieval_kernel(w2v_handle *h, uint32_t kind)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (kind > 1) return fail(h, W2V_ERR_ARG, "kind must be 0 (fp32 CUDA cores) or 1 (tensor cores)");
+    h->retrieval_kernel = kind;
     return W2V_OK;
 }
 

@@ -312,9 +312,10 @@ size_t topk_smem_bytes(uint32_t d, uint32_t K, int BQ)
 // How many ways to split the candidates so that the grid fills whole waves of one block per SM:
 // the smallest split count (at most 64, at most one per tile) whose last wave is at least 95 % full,
 // else the fullest one.
-uint32_t topk_splits(uint64_t m, uint64_t n_candidates, int sms)
+uint32_t topk_splits(uint64_t m, uint64_t n_candidates, int sms, uint32_t block_queries, uint32_t tile_rows)
 {
-    const uint64_t qblocks = (m + 63) / 64, tiles = (n_candidates + kTopkBC - 1) / kTopkBC;
+    if (block_queries == 0) { block_queries = 64; tile_rows = kTopkBC; }
+    const uint64_t qblocks = (m + block_queries - 1) / block_queries, tiles = (n_candidates + tile_rows - 1) / tile_rows;
     uint64_t max_s = tiles < 64 ? (tiles ? tiles : 1) : 64;
     uint32_t best = 1;
     double best_fill = 0.0;
@@ -334,6 +335,18 @@ int launch_inv_norms(const float *table, uint32_t d, uint32_t ld, uint64_t lo, u
     const uint64_t want = (count + (kBlock / 32) - 1) / (kBlock / 32);
     const int grid = (int)(want < (uint64_t)sms * 8 ? want : (uint64_t)sms * 8);
     row_inv_norm_kernel<<<grid, kBlock, 0, s>>>(table, d / 4, ld / 4, lo, count, inv_norm);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    return 1;
+}
+
+int launch_topk_merge(const float *part_cos, const long long *part_ids, uint64_t m, uint32_t K, uint32_t splits,
+                      float *out_cos, long long *out_ids, int sms, cudaStream_t s)
+{
+    if (m == 0) return 0;
+    const int warps = kBlock / 32;
+    const uint64_t want = (m + warps - 1) / warps;
+    const int grid = (int)(want < (uint64_t)sms * 8 ? want : (uint64_t)sms * 8);
+    topk_merge_kernel<<<grid, kBlock, (size_t)warps * K * 12, s>>>(part_cos, part_ids, m, K, splits, out_cos, out_ids);
     if (cudaGetLastError() != cudaSuccess) return -1;
     return 1;
 }

@@ -1,0 +1,320 @@
+// Cosine retrieval on the tensor cores (tcgen05, TMEM accumulators), same contract as the fp32
+// kernel in w2v_topk.cu.
+//
+// The dot products of 128 query rows with 128 candidate rows are one M128 x N128 accumulator tile in
+// tensor memory.  The tensor cores read fp32 operands as TF32 (the 13 low mantissa bits are
+// ignored), which alone would leave cosines good to 1e-3 only; the threshold and the ranking need
+// 1e-6.  So every value x is split into hi = x rounded to TF32 and lo = (x - hi) rounded to TF32, and
+// each k-step issues three MMAs into the same accumulator: lo.hi + hi.lo + hi.hi (the dropped lo.lo
+// term and the rounding of lo are below 2^-21 of |a||b| and unbiased).
+//
+// One block = 288 threads:
+//   warps 0-3  epilogue: warp w reads accumulator rows 32w .. 32w+31 (thread = one query) from
+//              tensor memory, scales by the inverse norms and keeps that query's sorted top-K list;
+//   warp 4     allocates tensor memory; one lane issues the MMAs;
+//   warps 5-8  loaders: global rows -> (hi, lo) -> shared memory, K-major core-matrix layout without
+//              swizzle ([16-byte column chunk][row][16 B], chunk stride 2064 B: conflict-free stores).
+// Shared-memory stages and the two accumulator buffers are handed over with mbarriers; every wait
+// has an iteration limit, after which the block raises the error flag and leaves through the common
+// exit that frees the tensor memory.
+#include "w2v_device.cuh"
+#include "w2v_internal.h"
+
+namespace w2v {
+
+constexpr int kTcM = 128;                       // query rows per block (accumulator lanes)
+constexpr int kTcN = 128;                       // candidate rows per tile (accumulator columns)
+constexpr int kTcKB = 32;                       // floats per K-block = 8 chunks of 16 B = 4 MMAs of K = 8
+constexpr int kTcStages = 3;
+constexpr int kTcChunkStride = kTcM * 16 + 16;  // bytes between 16-byte column chunks of an operand
+constexpr int kTcOperand = 8 * kTcChunkStride;  // bytes of one operand block (128 rows x 32 floats)
+constexpr int kTcStageBytes = 4 * kTcOperand;   // Q hi, Q lo, C hi, C lo
+constexpr int kTcThreads = 288;
+constexpr int kTcLoaders = 128;
+constexpr uint32_t kTcSpinLimit = 1u << 20;
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+// Bounded wait.  Returns false (and raises the block's abort flag) when the limit is reached or
+// another thread has already given up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    for (uint32_t spin = 0; spin < kTcSpinLimit; ++spin) {
+        if (mbar_try(bar, parity)) return true;
+        if ((spin & 1023u) == 1023u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+// Shared-memory matrix descriptor: K-major, no swizzle; 8 rows x 16 B core matrices, `lbo` bytes
+// between the two 16-byte column chunks of one MMA, `sbo` bytes between groups of 8 rows.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo)
+{
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}\n"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0), "r"(0), "r"(0), "r"(0) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+// Does (score a, id ia) rank ahead of (score b, id ib)?  Larger cosine first, then smaller id.
+__device__ __forceinline__ bool ranks_ahead_tc(float a, long long ia, float b, long long ib)
+{
+    return a > b || (a == b && ia < ib);
+}
+
+struct TcParams {
+    const float *table;
+    const long long *queries;
+    const float *inv_norm;
+    float *part_cos;              // [splits][m][K]
+    long long *part_ids;
+    int *error;                   // device word: set to 1 if a wait ran out
+    uint64_t m, vocab, cand_lo, cand_hi;
+    uint32_t d4, ld4, K, splits;
+    float tau;
+};
+
+// x rounded to the nearest value with 10 explicit mantissa bits (ties away from zero), so that the
+// tensor core, which drops the 13 low bits, reads it exactly.
+__device__ __forceinline__ float tf32_round(float x)
+{
+    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
+}
+
+// rows x 32 floats of the table -> (hi, lo) operand blocks.  `row_of(r)` gives the table row of
+// operand row r or -1 for a row of zeros.
+template <typename RowOf>
+__device__ __forceinline__ void load_split(const TcParams &p, unsigned char *hi, unsigned char *lo, uint32_t k0,
+                                           uint32_t ltid, RowOf row_of)
+{
+    const float4 *T4 = reinterpret_cast<const float4 *>(p.table);
+#pragma unroll
+    for (int it = 0; it < (kTcM * 8) / kTcLoaders; ++it) {
+        const uint32_t e = ltid + it * kTcLoaders;
+        const uint32_t r = e >> 3, ch = e & 7;                   // 8 threads cover 128 contiguous bytes of a row
+        const long long row = row_of(r);
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (row >= 0 && k0 / 4 + ch < p.d4) x = __ldcg(T4 + (size_t)row * p.ld4 + (k0 / 4 + ch));
+        const float4 h = make_float4(tf32_round(x.x), tf32_round(x.y), tf32_round(x.z), tf32_round(x.w));
+        const float4 l = make_float4(tf32_round(x.x - h.x), tf32_round(x.y - h.y), tf32_round(x.z - h.z),
+                                     tf32_round(x.w - h.w));
+        const uint32_t off = ch * kTcChunkStride + r * 16;
+        *reinterpret_cast<float4 *>(hi + off) = h;
+        *reinterpret_cast<float4 *>(lo + off) = l;
+    }
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+topk_cosine_tc_kernel(TcParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + kTcStages * kTcStageBytes);
+    uint64_t *empty = full + kTcStages;
+    uint64_t *tfull = empty + kTcStages;
+    uint64_t *tempty = tfull + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(tempty + 2);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    long long *qrow = reinterpret_cast<long long *>(tmem_slot + 4);          // [128]
+
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint64_t q0 = (uint64_t)blockIdx.x * kTcM;
+    const uint64_t nc = p.cand_hi - p.cand_lo;
+    const uint64_t tiles = (nc + kTcN - 1) / kTcN;
+    const uint64_t t_lo = tiles * blockIdx.y / p.splits, t_hi = tiles * (blockIdx.y + 1) / p.splits;
+    const uint32_t d = 4u * p.d4;
+    const uint32_t nkb = (d + kTcKB - 1) / kTcKB;
+    const uint64_t n_tiles = t_hi - t_lo;
+
+    if (tid == 0) {
+        for (int s = 0; s < kTcStages; ++s) { mbar_init(full + s, kTcLoaders); mbar_init(empty + s, 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull + b, 1); mbar_init(tempty + b, kTcM); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (tid < (uint32_t)kTcM) {
+        long long r = q0 + tid < p.m ? p.queries[q0 + tid] : -1;
+        if (r < 0 || (unsigned long long)r >= p.vocab) r = -1;
+        qrow[tid] = r;
+    }
+    if (warp == 4) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(2 * kTcN));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp < 4) {
+        // ================= epilogue: one thread per query row =================
+        const uint32_t r = tid;
+        const long long my_q = qrow[r];
+        const bool live = q0 + r < p.m;
+        float *lc = p.part_cos + ((size_t)blockIdx.y * p.m + (q0 + r)) * p.K;      // this query's list (global, private)
+        long long *li = p.part_ids + ((size_t)blockIdx.y * p.m + (q0 + r)) * p.K;
+        float qinv = 0.f;
+        if (my_q >= 0) {
+            const float4 *row = reinterpret_cast<const float4 *>(p.table) + (size_t)my_q * p.ld4;
+            float s = 0.f;
+            for (uint32_t j = 0; j < p.d4; ++j) {
+                const float4 x = __ldcg(row + j);
+                s = fmaf(x.x, x.x, s); s = fmaf(x.y, x.y, s); s = fmaf(x.z, x.z, s); s = fmaf(x.w, x.w, s);
+            }
+            qinv = s > 0.f ? 1.0f / sqrtf(s) : 0.f;
+        }
+        if (live) for (uint32_t s = 0; s < p.K; ++s) { lc[s] = 0.f; li[s] = -1; }
+        uint32_t have = 0;
+        float thr = p.tau;
+        for (uint64_t i = 0; i < n_tiles; ++i) {
+            const uint32_t b = (uint32_t)(i & 1);
+            // the tensor-memory loads below are warp-wide: the whole warp goes on or gives up together
+            if (!__all_sync(kFullMask, mbar_wait(tfull + b, (uint32_t)((i >> 1) & 1), abort_flag))) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint64_t c0 = (t_lo + i) * kTcN;
+#pragma unroll 1
+            for (uint32_t cc = 0; cc < (uint32_t)kTcN; cc += 16) {
+                uint32_t v[16];
+                __syncwarp();
+                const uint32_t ta = tmem_base + ((warp * 32u) << 16) + b * kTcN + cc;
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                             : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                               "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                             : "r"(ta));
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (my_q < 0 || !live) continue;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const uint64_t c = c0 + cc + j;
+                    if (c >= nc) break;
+                    const float cs = __uint_as_float(v[j]) * qinv * __ldg(p.inv_norm + c);
+                    const long long cid = (long long)(p.cand_lo + c);
+                    if (!(cs > p.tau) || cid == my_q || (have == p.K && cs < thr)) continue;
+                    // sorted insertion into this thread's own list
+                    uint32_t pos = have;
+                    while (pos > 0 && ranks_ahead_tc(cs, cid, lc[pos - 1], li[pos - 1])) --pos;
+                    if (pos >= p.K) continue;
+                    const uint32_t last = have < p.K ? have : p.K - 1u;
+                    for (uint32_t s = last; s > pos; --s) { lc[s] = lc[s - 1]; li[s] = li[s - 1]; }
+                    lc[pos] = cs; li[pos] = cid;
+                    if (have < p.K) ++have;
+                    thr = have == p.K ? lc[p.K - 1] : p.tau;
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            mbar_arrive(tempty + b);                              // this accumulator buffer may be overwritten
+        }
+    } else if (warp == 4) {
+        // ================= MMA issue: one lane =================
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTcN >> 3) << 17) | ((uint32_t)(kTcM >> 4) << 24);
+            uint64_t g = 0;
+            bool ok = true;
+            for (uint64_t i = 0; i < n_tiles && ok; ++i) {
+                const uint32_t b = (uint32_t)(i & 1);
+                ok = mbar_wait(tempty + b, (uint32_t)(((i >> 1) & 1) ^ 1), abort_flag);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t dst = tmem_base + b * kTcN;
+                for (uint32_t kb = 0; kb < nkb && ok; ++kb, ++g) {
+                    const uint32_t s = (uint32_t)(g % kTcStages);
+                    ok = mbar_wait(full + s, (uint32_t)((g / kTcStages) & 1), abort_flag);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t base = smem_addr(smem + (size_t)s * kTcStageBytes);
+#pragma unroll
+                    for (int kk = 0; kk < kTcKB / 8; ++kk) {
+                        const uint32_t off = 2 * kk * kTcChunkStride;
+                        const uint64_t qh = umma_desc(base + 0 * kTcOperand + off, kTcChunkStride, 128);
+                        const uint64_t ql = umma_desc(base + 1 * kTcOperand + off, kTcChunkStride, 128);
+                        const uint64_t ch = umma_desc(base + 2 * kTcOperand + off, kTcChunkStride, 128);
+                        const uint64_t cl = umma_desc(base + 3 * kTcOperand + off, kTcChunkStride, 128);
+                        umma_tf32(dst, ql, ch, idesc, (kb | kk) ? 1u : 0u);      // small terms first
+                        umma_tf32(dst, qh, cl, idesc, 1u);
+                        umma_tf32(dst, qh, ch, idesc, 1u);
+                    }
+                    umma_commit(empty + s);                       // the stage is free once these MMAs have read it
+                }
+                if (ok) umma_commit(tfull + b);                   // the tile's accumulator is complete
+            }
+        }
+    } else {
+        // ================= loaders =================
+        const uint32_t ltid = tid - 5 * 32;
+        uint64_t g = 0;
+        bool ok = true;
+        for (uint64_t i = 0; i < n_tiles && ok; ++i) {
+            const uint64_t c0 = (t_lo + i) * kTcN;
+            for (uint32_t kb = 0; kb < nkb; ++kb, ++g) {
+                const uint32_t s = (uint32_t)(g % kTcStages);
+                ok = mbar_wait(empty + s, (uint32_t)(((g / kTcStages) & 1) ^ 1), abort_flag);
+                if (!ok) break;
+                unsigned char *st = smem + (size_t)s * kTcStageBytes;
+                load_split(p, st + 0 * kTcOperand, st + 1 * kTcOperand, kb * kTcKB, ltid,
+                           [&](uint32_t r) { return qrow[r]; });
+                load_split(p, st + 2 * kTcOperand, st + 3 * kTcOperand, kb * kTcKB, ltid,
+                           [&](uint32_t r) { return c0 + r < nc ? (long long)(p.cand_lo + c0 + r) : -1ll; });
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // stores -> tensor-core reads
+                mbar_arrive(full + s);
+            }
+        }
+    }
+    // ================= common exit =================
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (tid == 0 && *abort_flag) atomicExch(p.error, 1);
+    if (warp == 4) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * kTcN));
+    }
+}
+
+size_t topk_tc_smem_bytes()
+{
+    return (size_t)kTcStages * kTcStageBytes + (2 * kTcStages + 4) * 8 + 16 + kTcM * 8 + 128;
+}
+
+// Returns 1, or -1 on a launch error.  Results go to part_* ([splits][m][K]); the caller merges.
+int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, const long long *queries, uint64_t m,
+                   uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, const float *inv_norm, float *part_cos,
+                   long long *part_ids, uint32_t splits, int *error, cudaStream_t s)
+{
+    if (m == 0) return 0;
+    TcParams p;
+    p.table = table; p.queries = queries; p.inv_norm = inv_norm; p.part_cos = part_cos; p.part_ids = part_ids;
+    p.error = error; p.m = m; p.vocab = vocab; p.cand_lo = cand_lo; p.cand_hi = cand_hi;
+    p.d4 = d / 4; p.ld4 = ld / 4; p.K = K; p.splits = splits; p.tau = tau;
+    const size_t sm = topk_tc_smem_bytes();
+    if (cudaFuncSetAttribute(topk_cosine_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess)
+        return -1;
+    dim3 grid((unsigned)((m + kTcM - 1) / kTcM), splits);
+    topk_cosine_tc_kernel<<<grid, kTcThreads, sm, s>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    return 1;
+}
+
+}  // namespace w2v

@@ -13,19 +13,29 @@ from paper_1606_08495_b200 import binding
 pytestmark = pytest.mark.gpu
 
 TOL = 2e-6
+KERNELS = [0, 1]          # fp32 on the CUDA cores; tensor cores with the TF32 head/tail split
 
 
-def pair(V, d, seed, which=0, scale=1.0, row_stride=None, rows=None):
+def tolerance(kernel, d):
+    """fp32 CUDA cores: rounding of a d-term fp32 dot product of unit-scaled rows, 2e-6.  Tensor cores:
+    the head/tail split leaves ~2^-21 per product, but the accumulator in tensor memory is updated
+    3 * d/8 times (three MMAs per 8 columns) with rounding toward zero, each time up to 2^-24 of the
+    running sum (|cos| <= 1): a bias of up to 3 (d/8) 2^-24 on top."""
+    return TOL if kernel == 0 else TOL + 3 * ((d + 7) // 8) * 2.0 ** -24
+
+
+def pair(V, d, seed, which=0, scale=1.0, row_stride=None, rows=None, kernel=0):
     rng = np.random.default_rng(seed)
     X = rng.normal(scale=scale, size=(V, d)).astype(np.float32) if rows is None else np.asarray(rows, dtype=np.float32)
     gpu = binding.W2V(V, d, 1, row_stride=row_stride)
     cpu = Oracle(V, d, 1)
     ids = np.arange(V)
     gpu.write_rows(which, ids, X); cpu.write_rows(which, ids, X)
+    binding.w2v_set_retrieval_kernel(gpu.h, kernel)
     return gpu, cpu, X
 
 
-def check(gpu, cpu, X, which, queries, lo, hi, K, tau):
+def check(gpu, cpu, X, which, queries, lo, hi, K, tau, TOL=TOL):
     gi, gc = gpu.topk_cosine(which, queries, lo, hi, K, tau)
     wi, wc = cpu.topk_cosine(which, queries, lo, hi, K, tau)
     assert gi.shape == wi.shape
@@ -51,35 +61,38 @@ def check(gpu, cpu, X, which, queries, lo, hi, K, tau):
     return gi, gc
 
 
+@pytest.mark.parametrize("kernel", KERNELS)
 @pytest.mark.parametrize("V,d,K,m", [(3000, 300, 30, 200), (1000, 100, 5, 70), (5000, 64, 64, 10), (700, 4, 1, 700),
                                      (900, 1024, 30, 40), (129, 132, 7, 129)])
-def test_topk_matches_brute_force(V, d, K, m):
-    gpu, cpu, X = pair(V, d, seed=V + d)
+def test_topk_matches_brute_force(V, d, K, m, kernel):
+    gpu, cpu, X = pair(V, d, seed=V + d, kernel=kernel)
     rng = np.random.default_rng(1)
     q = rng.integers(0, V, m)
-    check(gpu, cpu, X, 0, q, 0, V, K, -2.0)
-    check(gpu, cpu, X, 0, q, V // 5, V - 7, K, 0.0)
+    check(gpu, cpu, X, 0, q, 0, V, K, -2.0, tolerance(kernel, d))
+    check(gpu, cpu, X, 0, q, V // 5, V - 7, K, 0.0, tolerance(kernel, d))
     gpu.close()
 
 
-def test_topk_threshold_of_the_paper_on_clustered_vectors():
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_topk_threshold_of_the_paper_on_clustered_vectors(kernel):
     # rows = cluster centre + noise, so that some neighbours are above tau = 0.65 and most are not
     rng = np.random.default_rng(3)
     V, d, C = 20_000, 300, 400
     centres = rng.normal(size=(C, d))
     X = (centres[rng.integers(0, C, V)] + 0.55 * rng.normal(size=(V, d))).astype(np.float32)
-    gpu, cpu, X = pair(V, d, 0, which=1, rows=X, row_stride=320)
+    gpu, cpu, X = pair(V, d, 0, which=1, rows=X, row_stride=320, kernel=kernel)
     q = rng.integers(0, V, 300)
-    gi, gc = check(gpu, cpu, X, 1, q, 5000, 20_000, 30, 0.65)
+    gi, gc = check(gpu, cpu, X, 1, q, 5000, 20_000, 30, 0.65, tolerance(kernel, d))
     kept = (gi >= 0).sum(axis=1)
     assert kept.max() == 30 and kept.min() < 30 and (gc[gi >= 0] > 0.65).all()
     gpu.close()
 
 
-def test_topk_many_queries_few_candidates_and_edge_cases():
-    gpu, cpu, X = pair(5000, 32, seed=9, scale=3.0)
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_topk_many_queries_few_candidates_and_edge_cases(kernel):
+    gpu, cpu, X = pair(5000, 32, seed=9, scale=3.0, kernel=kernel)
     q = np.arange(5000)                                   # more query blocks than SMs: no candidate split
-    check(gpu, cpu, X, 0, q, 100, 150, 8, -2.0)
+    check(gpu, cpu, X, 0, q, 100, 150, 8, -2.0, tolerance(kernel, 32))
     gi, gc = gpu.topk_cosine(0, [5, -1, 5000, 7], 0, 5000, 4, -2.0)
     assert (gi[1] == -1).all() and (gi[2] == -1).all() and (gi[0] >= 0).all() and (gi[3] >= 0).all()
     gi, gc = gpu.topk_cosine(0, [5], 10, 10, 4, -2.0)     # empty candidate range
@@ -94,14 +107,15 @@ def test_topk_many_queries_few_candidates_and_edge_cases():
     gpu.close()
 
 
-def test_topk_zero_rows_and_exact_ties():
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_topk_zero_rows_and_exact_ties(kernel):
     rows = np.zeros((200, 8), dtype=np.float32)
     rows[:, 0] = 1.0                                      # every row the same direction: all cosines 1
     rows[50] = 0.0                                        # a zero row: cosine 0 with everything
     rows[100:, 0] = np.arange(100, 200)                   # other lengths, same direction
-    gpu, cpu, X = pair(200, 8, 0, rows=rows)
+    gpu, cpu, X = pair(200, 8, 0, rows=rows, kernel=kernel)
     gi, gc = gpu.topk_cosine(0, [0, 50, 150], 0, 200, 6, -2.0)
     wi, wc = cpu.topk_cosine(0, [0, 50, 150], 0, 200, 6, -2.0)
     assert np.array_equal(gi, wi)                         # ties go to the smaller row number
-    assert np.allclose(gc, wc, atol=TOL)
+    assert np.allclose(gc, wc, atol=tolerance(kernel, 8))
     gpu.close()
