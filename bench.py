@@ -473,6 +473,8 @@ def run_topk(args):
     K, tau, m = 30, 0.65, args.queries
     lo, hi = int(V * 0.85), V
     model = binding.W2V(V, d, seed=1, device=dev, row_stride=row_stride_for(d, args.row_stride))
+    tensor = args.retrieval_kernel == "tensor"
+    binding.w2v_set_retrieval_kernel(model.h, 1 if tensor else 0)
     # spread-out vectors instead of the tiny uniform initial ones: normal rows, so that cosines have the
     # spread of unrelated trained vectors (about N(0, 1/d)); written by torch, this is input data
     g = torch.Generator(device=dev); g.manual_seed(5)
@@ -518,22 +520,36 @@ def run_topk(args):
     cosines = float(m) * (hi - lo) * Ksteps
     flops = 2.0 * d * cosines
     sm_mhz = clocks.get("sm_max_mhz") or 1965.0
-    peak = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12          # fp32 FMA lanes x 2 flop x clock, TFLOP/s
     achieved = flops / (kernel_ms * 1e-3) / 1e12 if kernel_ms > 0 else 0.0
+    if tensor:
+        # useful flops against the tensor peak of the type the MMAs run in: measured dense bf16 x the
+        # nominal tf32 / bf16 ratio (1.1 / 2.25 PFLOP/s); each useful product costs three TF32 MMAs
+        try:
+            with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+                bf16, kind = float(json.load(f)["bf16_tflops_sustained"]), "measured sustained bf16 x 1.1/2.25"
+        except Exception:
+            bf16, kind = 1400.0, "fallback sustained bf16 x 1.1/2.25"
+        peak, bound = bf16 * 1.1 / 2.25, "tensor"
+        peak_kind = kind + " (tf32); the kernel issues 3 MMA flops per useful flop"
+    else:
+        peak, bound = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12, "alu"     # fp32 FMA lanes x 2 flop x clock, TFLOP/s
+        peak_kind = "148 SMs x 128 fp32 FMA lanes x 2 flop x max SM clock"
     line = {
         "metric": "cosine_similarities_per_sec", "value": cosines / (ms * 1e-3), "unit": "cosines/s", "n_gpus": 1,
         "steps": Ksteps, "warmup": Wu, "ms_per_step": ms / Ksteps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": name + " (retrieval)", "vocab": V, "d": d, "queries_per_step": m,
                    "candidates": hi - lo, "K": K, "tau": tau, "row_stride_floats": model.row_stride,
+                   "kernel": "tcgen05 tf32, head/tail split (3 MMAs per product)" if tensor else "fp32 CUDA cores",
                    "l2": "3 M candidate rows (3.8 GB) streamed per call, far larger than L2"},
         "clocks": clocks,
         "e2e": {"value": cosines / (e2e_ms * 1e-3), "unit": "cosines/s", "h2d_bytes_per_step": 8 * m,
                 "d2h_bytes_per_step": 12 * m * K},
         "gpu_launches": launches,
-        "roofline": {"bound": "alu", "kernel": "topk_cosine_kernel", "achieved": achieved, "peak": peak,
-                     "unit": "TFLOP/s", "frac": achieved / peak,
-                     "peak_kind": "148 SMs x 128 fp32 FMA lanes x 2 flop x max SM clock",
+        "roofline": {"bound": bound, "kernel": "topk_cosine_tc_kernel" if tensor else "topk_cosine_kernel",
+                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                     "mma_tflops_issued": 3 * achieved if tensor else None,
+                     "peak_kind": peak_kind,
                      "flops_per_launch": flops / Ksteps, "kernel_ms_per_launch": kernel_ms / Ksteps, "traffic": None},
     }
     print(json.dumps(line), flush=True)
@@ -556,6 +572,7 @@ def main():
     ap.add_argument("--ref-words", type=int, default=20_000, help="word tokens per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--queries", type=int, default=8192, help="query rows per call of --mode topk")
+    ap.add_argument("--retrieval-kernel", choices=["fp32", "tensor"], default="tensor")
     ap.add_argument("--mode", choices=["hogwild", "snapshot", "sharded", "topk"], default="hogwild",
                     help="update mode of the timed steps (the headline number is hogwild); sharded = the "
                          "paper's column partition, --shards slices of one model on one GPU")

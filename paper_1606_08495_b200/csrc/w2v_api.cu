@@ -24,7 +24,7 @@ struct w2v_handle {
     uint64_t l_cap_pairs = 0, l_cap_negs = 0;
     float *inv_norm = nullptr; uint64_t inv_norm_cap = 0;                      // retrieval scratch
     float *part_cos = nullptr; long long *part_ids = nullptr; uint64_t part_cap = 0;
-    uint32_t retrieval_kernel = 0;       // 0: fp32 on the CUDA cores, 1: tensor cores (3 x TF32)
+    uint32_t retrieval_kernel = 1;       // 0: fp32 on the CUDA cores, 1: tensor cores (3 x TF32)
     int *tc_error = nullptr;             // device word raised by a tensor-core block whose wait ran out
     uint32_t pend_window = 0, pend_negatives = 0;
     uint64_t pend_n = 0, pend_pairs = 0;

@@ -8,11 +8,11 @@
 // each k-step issues three MMAs into the same accumulator: lo.hi + hi.lo + hi.hi (the dropped lo.lo
 // term and the rounding of lo are below 2^-21 of |a||b| and unbiased).
 //
-// One block = 288 threads:
+// One block = 544 threads:
 //   warps 0-3  epilogue: warp w reads accumulator rows 32w .. 32w+31 (thread = one query) from
 //              tensor memory, scales by the inverse norms and keeps that query's sorted top-K list;
 //   warp 4     allocates tensor memory; one lane issues the MMAs;
-//   warps 5-8  loaders: global rows -> (hi, lo) -> shared memory, K-major core-matrix layout without
+//   warps 5-16 loaders (three groups of 4 warps, one per stage of the ring): global rows -> (hi, lo) -> shared memory, K-major core-matrix layout without
 //              swizzle ([16-byte column chunk][row][16 B], chunk stride 2064 B: conflict-free stores).
 // Shared-memory stages and the two accumulator buffers are handed over with mbarriers; every wait
 // has an iteration limit, after which the block raises the error flag and leaves through the common
@@ -29,8 +29,9 @@ constexpr int kTcStages = 3;
 constexpr int kTcChunkStride = kTcM * 16 + 16;  // bytes between 16-byte column chunks of an operand
 constexpr int kTcOperand = 8 * kTcChunkStride;  // bytes of one operand block (128 rows x 32 floats)
 constexpr int kTcStageBytes = 4 * kTcOperand;   // Q hi, Q lo, C hi, C lo
-constexpr int kTcThreads = 288;
-constexpr int kTcLoaders = 128;
+constexpr int kTcLoaders = 128;                 // threads that fill one stage together
+constexpr int kTcGroups = 3;                    // loader groups; group j fills stages j, j + 3, ...: all three stages can be in flight
+constexpr int kTcThreads = 5 * 32 + kTcGroups * kTcLoaders;
 constexpr uint32_t kTcSpinLimit = 1u << 20;
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -107,26 +108,38 @@ __device__ __forceinline__ float tf32_round(float x)
     return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
 }
 
-// rows x 32 floats of the table -> (hi, lo) operand blocks.  `row_of(r)` gives the table row of
-// operand row r or -1 for a row of zeros.
-template <typename RowOf>
-__device__ __forceinline__ void load_split(const TcParams &p, unsigned char *hi, unsigned char *lo, uint32_t k0,
-                                           uint32_t ltid, RowOf row_of)
+// One stage: 128 query rows and 128 candidate rows x 32 floats of the table -> (hi, lo) operand
+// blocks.  All of a thread's global loads are issued before the first value is used.
+__device__ __forceinline__ void load_stage(const TcParams &p, unsigned char *st, uint32_t k0, uint32_t ltid,
+                                           const long long *qrow, uint64_t c0, uint64_t nc)
 {
+    constexpr int kPer = (kTcM * 8) / kTcLoaders;                // float4 per thread and operand
     const float4 *T4 = reinterpret_cast<const float4 *>(p.table);
+    float4 x[2][kPer];
 #pragma unroll
-    for (int it = 0; it < (kTcM * 8) / kTcLoaders; ++it) {
+    for (int it = 0; it < kPer; ++it) {
         const uint32_t e = ltid + it * kTcLoaders;
         const uint32_t r = e >> 3, ch = e & 7;                   // 8 threads cover 128 contiguous bytes of a row
-        const long long row = row_of(r);
-        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (row >= 0 && k0 / 4 + ch < p.d4) x = __ldcg(T4 + (size_t)row * p.ld4 + (k0 / 4 + ch));
-        const float4 h = make_float4(tf32_round(x.x), tf32_round(x.y), tf32_round(x.z), tf32_round(x.w));
-        const float4 l = make_float4(tf32_round(x.x - h.x), tf32_round(x.y - h.y), tf32_round(x.z - h.z),
-                                     tf32_round(x.w - h.w));
-        const uint32_t off = ch * kTcChunkStride + r * 16;
-        *reinterpret_cast<float4 *>(hi + off) = h;
-        *reinterpret_cast<float4 *>(lo + off) = l;
+        const bool col_ok = k0 / 4 + ch < p.d4;
+        const long long rq = qrow[r];
+        const long long rc = c0 + r < nc ? (long long)(p.cand_lo + c0 + r) : -1ll;
+        x[0][it] = (rq >= 0 && col_ok) ? __ldcg(T4 + (size_t)rq * p.ld4 + (k0 / 4 + ch)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        x[1][it] = (rc >= 0 && col_ok) ? __ldcg(T4 + (size_t)rc * p.ld4 + (k0 / 4 + ch)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int o = 0; o < 2; ++o) {
+#pragma unroll
+        for (int it = 0; it < kPer; ++it) {
+            const uint32_t e = ltid + it * kTcLoaders;
+            const uint32_t r = e >> 3, ch = e & 7;
+            const float4 v = x[o][it];
+            const float4 h = make_float4(tf32_round(v.x), tf32_round(v.y), tf32_round(v.z), tf32_round(v.w));
+            const float4 l = make_float4(tf32_round(v.x - h.x), tf32_round(v.y - h.y), tf32_round(v.z - h.z),
+                                         tf32_round(v.w - h.w));
+            const uint32_t off = ch * kTcChunkStride + r * 16;
+            *reinterpret_cast<float4 *>(st + (2 * o) * kTcOperand + off) = h;
+            *reinterpret_cast<float4 *>(st + (2 * o + 1) * kTcOperand + off) = l;
+        }
     }
 }
 
@@ -264,20 +277,18 @@ topk_cosine_tc_kernel(TcParams p)
         }
     } else {
         // ================= loaders =================
-        const uint32_t ltid = tid - 5 * 32;
+        const uint32_t group = (tid - 5 * 32) / kTcLoaders, ltid = (tid - 5 * 32) % kTcLoaders;
         uint64_t g = 0;
         bool ok = true;
         for (uint64_t i = 0; i < n_tiles && ok; ++i) {
             const uint64_t c0 = (t_lo + i) * kTcN;
             for (uint32_t kb = 0; kb < nkb; ++kb, ++g) {
+                if (g % kTcGroups != group) continue;
                 const uint32_t s = (uint32_t)(g % kTcStages);
                 ok = mbar_wait(empty + s, (uint32_t)(((g / kTcStages) & 1) ^ 1), abort_flag);
                 if (!ok) break;
                 unsigned char *st = smem + (size_t)s * kTcStageBytes;
-                load_split(p, st + 0 * kTcOperand, st + 1 * kTcOperand, kb * kTcKB, ltid,
-                           [&](uint32_t r) { return qrow[r]; });
-                load_split(p, st + 2 * kTcOperand, st + 3 * kTcOperand, kb * kTcKB, ltid,
-                           [&](uint32_t r) { return c0 + r < nc ? (long long)(p.cand_lo + c0 + r) : -1ll; });
+                load_stage(p, st, kb * kTcKB, ltid, qrow, c0, nc);
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // stores -> tensor-core reads
                 mbar_arrive(full + s);
             }
