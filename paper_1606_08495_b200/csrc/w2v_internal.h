@@ -137,10 +137,12 @@ int launch_copy_rows(float *table, uint32_t vocab, uint32_t d, uint32_t ld, cons
 uint32_t topk_splits(uint64_t m, uint64_t n_candidates, int sms, uint32_t block_queries = 0, uint32_t tile_rows = 0);
 int launch_topk_merge(const float *part_cos, const long long *part_ids, uint64_t m, uint32_t K, uint32_t splits,
                       float *out_cos, long long *out_ids, int sms, cudaStream_t s);
-// tensor-core variant (w2v_topk_tc.cu): partial lists only, 128 queries per block, tiles of 128 candidates
+// tensor-core variant (w2v_topk_tc.cu): partial lists only, 128 queries per block, tiles of 256 candidates
+size_t topk_tc_qsplit_bytes(uint64_t m, uint32_t d);
 int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, const long long *queries, uint64_t m,
-                   uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, const float *inv_norm, float *part_cos,
-                   long long *part_ids, uint32_t splits, int *error, cudaStream_t s);
+                   uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, const float *inv_norm,
+                   unsigned char *qsplit, float *part_cos, long long *part_ids, uint32_t splits, int *error,
+                   cudaStream_t s);
 int launch_inv_norms(const float *table, uint32_t d, uint32_t ld, uint64_t lo, uint64_t count, float *inv_norm,
                      int sms, cudaStream_t s);
 // Returns launches made, -1 on a launch error, -2 if the shape does not fit shared memory.

@@ -1,18 +1,19 @@
 // Cosine retrieval on the tensor cores (tcgen05, TMEM accumulators), same contract as the fp32
 // kernel in w2v_topk.cu.
 //
-// The dot products of 128 query rows with 128 candidate rows are one M128 x N128 accumulator tile in
+// The dot products of 128 query rows with 256 candidate rows are one M128 x N256 accumulator tile in
 // tensor memory.  The tensor cores read fp32 operands as TF32 (the 13 low mantissa bits are
 // ignored), which alone would leave cosines good to 1e-3 only; the threshold and the ranking need
 // 1e-6.  So every value x is split into hi = x rounded to TF32 and lo = (x - hi) rounded to TF32, and
 // each k-step issues three MMAs into the same accumulator: lo.hi + hi.lo + hi.hi (the dropped lo.lo
 // term and the rounding of lo are below 2^-21 of |a||b| and unbiased).
 //
-// One block = 544 threads:
+// One block = 672 threads:
 //   warps 0-3  epilogue: warp w reads accumulator rows 32w .. 32w+31 (thread = one query) from
 //              tensor memory, scales by the inverse norms and keeps that query's sorted top-K list;
 //   warp 4     allocates tensor memory; one lane issues the MMAs;
-//   warps 5-16 loaders (three groups of 4 warps, one per stage of the ring): global rows -> (hi, lo) -> shared memory, K-major core-matrix layout without
+//   warps 5-20 loaders (two groups of 8 warps, one per stage of the ring): candidate rows -> (hi, lo) -> shared memory
+//              (the query side is split once by a pre-pass and arrives by cp.async.bulk), K-major core-matrix layout without
 //              swizzle ([16-byte column chunk][row][16 B], chunk stride 2064 B: conflict-free stores).
 // Shared-memory stages and the two accumulator buffers are handed over with mbarriers; every wait
 // has an iteration limit, after which the block raises the error flag and leaves through the common
@@ -23,14 +24,16 @@
 namespace w2v {
 
 constexpr int kTcM = 128;                       // query rows per block (accumulator lanes)
-constexpr int kTcN = 128;                       // candidate rows per tile (accumulator columns)
+constexpr int kTcN = 256;                       // candidate rows per tile (accumulator columns)
 constexpr int kTcKB = 32;                       // floats per K-block = 8 chunks of 16 B = 4 MMAs of K = 8
-constexpr int kTcStages = 3;
-constexpr int kTcChunkStride = kTcM * 16 + 16;  // bytes between 16-byte column chunks of an operand
-constexpr int kTcOperand = 8 * kTcChunkStride;  // bytes of one operand block (128 rows x 32 floats)
-constexpr int kTcStageBytes = 4 * kTcOperand;   // Q hi, Q lo, C hi, C lo
-constexpr int kTcLoaders = 128;                 // threads that fill one stage together
-constexpr int kTcGroups = 3;                    // loader groups; group j fills stages j, j + 3, ...: all three stages can be in flight
+constexpr int kTcStages = 2;
+constexpr int kTcChunkStride = kTcM * 16 + 16;  // bytes between 16-byte column chunks of a query operand
+constexpr int kTcOperand = 8 * kTcChunkStride;  // bytes of one query operand block (128 rows x 32 floats)
+constexpr int kTcChunkStrideC = kTcN * 16 + 16; // the same for a candidate operand (256 rows)
+constexpr int kTcOperandC = 8 * kTcChunkStrideC;
+constexpr int kTcStageBytes = 2 * kTcOperand + 2 * kTcOperandC;   // Q hi, Q lo, C hi, C lo
+constexpr int kTcLoaders = 256;                 // threads that fill one stage together
+constexpr int kTcGroups = 2;                    // loader groups; group j fills stages j, j + 2, ...
 constexpr int kTcThreads = 5 * 32 + kTcGroups * kTcLoaders;
 constexpr uint32_t kTcSpinLimit = 1u << 20;
 
@@ -89,10 +92,26 @@ __device__ __forceinline__ bool ranks_ahead_tc(float a, long long ia, float b, l
     return a > b || (a == b && ia < ib);
 }
 
+// One candidate for a thread's own sorted list (in global memory, private to the thread).
+__device__ __noinline__ void list_offer(float *lc, long long *li, uint32_t &have, float &thr, uint32_t K, float tau,
+                                        float cs, long long cid, long long self)
+{
+    if (!(cs > tau) || cid == self || (have == K && cs < thr)) return;
+    uint32_t pos = have;
+    while (pos > 0 && ranks_ahead_tc(cs, cid, lc[pos - 1], li[pos - 1])) --pos;
+    if (pos >= K) return;
+    const uint32_t last = have < K ? have : K - 1u;
+    for (uint32_t s = last; s > pos; --s) { lc[s] = lc[s - 1]; li[s] = li[s - 1]; }
+    lc[pos] = cs; li[pos] = cid;
+    if (have < K) ++have;
+    thr = have == K ? lc[K - 1] : tau;
+}
+
 struct TcParams {
     const float *table;
     const long long *queries;
     const float *inv_norm;
+    const unsigned char *qsplit;  // [query blocks][K-blocks][hi, lo] operand blocks, laid out as in shared memory
     float *part_cos;              // [splits][m][K]
     long long *part_ids;
     int *error;                   // device word: set to 1 if a wait ran out
@@ -108,39 +127,74 @@ __device__ __forceinline__ float tf32_round(float x)
     return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
 }
 
-// One stage: 128 query rows and 128 candidate rows x 32 floats of the table -> (hi, lo) operand
-// blocks.  All of a thread's global loads are issued before the first value is used.
-__device__ __forceinline__ void load_stage(const TcParams &p, unsigned char *st, uint32_t k0, uint32_t ltid,
-                                           const long long *qrow, uint64_t c0, uint64_t nc)
+__device__ __forceinline__ void split_store(unsigned char *hi, unsigned char *lo, uint32_t r, uint32_t ch, float4 v,
+                                            uint32_t chunk_stride)
 {
-    constexpr int kPer = (kTcM * 8) / kTcLoaders;                // float4 per thread and operand
+    const float4 h = make_float4(tf32_round(v.x), tf32_round(v.y), tf32_round(v.z), tf32_round(v.w));
+    const float4 l = make_float4(tf32_round(v.x - h.x), tf32_round(v.y - h.y), tf32_round(v.z - h.z),
+                                 tf32_round(v.w - h.w));
+    const uint32_t off = ch * chunk_stride + r * 16;
+    *reinterpret_cast<float4 *>(hi + off) = h;
+    *reinterpret_cast<float4 *>(lo + off) = l;
+}
+
+// The query side is the same for every candidate tile: it is split once, into global scratch that
+// has the layout of the shared-memory operand blocks, and the main kernel copies it in bulk.
+// One block per (query block, K-block).
+__global__ void __launch_bounds__(256)
+topk_split_queries_kernel(const float *__restrict__ table, const long long *__restrict__ queries, uint64_t m,
+                          uint64_t vocab, uint32_t d4, uint32_t ld4, uint32_t nkb, unsigned char *__restrict__ qsplit)
+{
+    const uint32_t qb = blockIdx.x / nkb, kb = blockIdx.x % nkb;
+    unsigned char *hi = qsplit + ((size_t)qb * nkb + kb) * 2 * kTcOperand, *lo = hi + kTcOperand;
+    const float4 *T4 = reinterpret_cast<const float4 *>(table);
+    for (uint32_t e = threadIdx.x; e < (uint32_t)kTcM * 8; e += blockDim.x) {
+        const uint32_t r = e >> 3, ch = e & 7;
+        const uint64_t qi = (uint64_t)qb * kTcM + r;
+        long long row = qi < m ? queries[qi] : -1;
+        if (row < 0 || (unsigned long long)row >= vocab) row = -1;
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (row >= 0 && kb * 8 + ch < d4) x = __ldcg(T4 + (size_t)row * ld4 + (kb * 8 + ch));
+        split_store(hi, lo, r, ch, x, kTcChunkStride);
+    }
+    // the 16 padding bytes at the end of each chunk are copied too: keep them defined
+    if (threadIdx.x < 8) {
+        *reinterpret_cast<float4 *>(hi + threadIdx.x * kTcChunkStride + kTcM * 16) = make_float4(0.f, 0.f, 0.f, 0.f);
+        *reinterpret_cast<float4 *>(lo + threadIdx.x * kTcChunkStride + kTcM * 16) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+}
+
+// One stage of candidates: 128 rows x 32 floats of the table -> (hi, lo) operand blocks, in two
+// halves so that the global loads can be issued before the stage's slot in shared memory is free.
+constexpr int kTcPer = (kTcN * 8) / kTcLoaders;                  // float4 per loader thread and stage
+
+__device__ __forceinline__ void candidates_issue(const TcParams &p, float4 (&x)[kTcPer], uint32_t k0, uint32_t ltid,
+                                                 uint64_t c0, uint64_t nc)
+{
     const float4 *T4 = reinterpret_cast<const float4 *>(p.table);
-    float4 x[2][kPer];
 #pragma unroll
-    for (int it = 0; it < kPer; ++it) {
+    for (int it = 0; it < kTcPer; ++it) {
         const uint32_t e = ltid + it * kTcLoaders;
         const uint32_t r = e >> 3, ch = e & 7;                   // 8 threads cover 128 contiguous bytes of a row
-        const bool col_ok = k0 / 4 + ch < p.d4;
-        const long long rq = qrow[r];
-        const long long rc = c0 + r < nc ? (long long)(p.cand_lo + c0 + r) : -1ll;
-        x[0][it] = (rq >= 0 && col_ok) ? __ldcg(T4 + (size_t)rq * p.ld4 + (k0 / 4 + ch)) : make_float4(0.f, 0.f, 0.f, 0.f);
-        x[1][it] = (rc >= 0 && col_ok) ? __ldcg(T4 + (size_t)rc * p.ld4 + (k0 / 4 + ch)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        x[it] = (c0 + r < nc && k0 / 4 + ch < p.d4) ? __ldcg(T4 + (size_t)(p.cand_lo + c0 + r) * p.ld4 + (k0 / 4 + ch))
+                                                    : make_float4(0.f, 0.f, 0.f, 0.f);
     }
+}
+
+__device__ __forceinline__ void candidates_store(unsigned char *hi, unsigned char *lo, const float4 (&x)[kTcPer],
+                                                 uint32_t ltid)
+{
 #pragma unroll
-    for (int o = 0; o < 2; ++o) {
-#pragma unroll
-        for (int it = 0; it < kPer; ++it) {
-            const uint32_t e = ltid + it * kTcLoaders;
-            const uint32_t r = e >> 3, ch = e & 7;
-            const float4 v = x[o][it];
-            const float4 h = make_float4(tf32_round(v.x), tf32_round(v.y), tf32_round(v.z), tf32_round(v.w));
-            const float4 l = make_float4(tf32_round(v.x - h.x), tf32_round(v.y - h.y), tf32_round(v.z - h.z),
-                                         tf32_round(v.w - h.w));
-            const uint32_t off = ch * kTcChunkStride + r * 16;
-            *reinterpret_cast<float4 *>(st + (2 * o) * kTcOperand + off) = h;
-            *reinterpret_cast<float4 *>(st + (2 * o + 1) * kTcOperand + off) = l;
-        }
+    for (int it = 0; it < kTcPer; ++it) {
+        const uint32_t e = ltid + it * kTcLoaders;
+        split_store(hi, lo, e >> 3, e & 7, x[it], kTcChunkStrideC);
     }
+}
+
+__device__ __forceinline__ void bulk_to_smem(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
 
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -154,6 +208,7 @@ topk_cosine_tc_kernel(TcParams p)
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(tempty + 2);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     long long *qrow = reinterpret_cast<long long *>(tmem_slot + 4);          // [128]
+    float *inv_c = reinterpret_cast<float *>(qrow + kTcM);                   // [4 warps][2][kTcN]
 
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint64_t q0 = (uint64_t)blockIdx.x * kTcM;
@@ -206,37 +261,41 @@ topk_cosine_tc_kernel(TcParams p)
         float thr = p.tau;
         for (uint64_t i = 0; i < n_tiles; ++i) {
             const uint32_t b = (uint32_t)(i & 1);
+            const uint64_t c0 = (t_lo + i) * kTcN;
+            // inverse norms of the tile's candidates (0 past the end of the range), staged in shared
+            // memory while the tile's MMAs are still running
+            float *icn = inv_c + (warp * 2 + b) * kTcN;             // one copy per warp: no block-wide barrier here
+            for (uint32_t j = lane; j < (uint32_t)kTcN; j += 32) icn[j] = c0 + j < nc ? __ldg(p.inv_norm + c0 + j) : 0.f;
+            __syncwarp();
             // the tensor-memory loads below are warp-wide: the whole warp goes on or gives up together
             if (!__all_sync(kFullMask, mbar_wait(tfull + b, (uint32_t)((i >> 1) & 1), abort_flag))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint64_t c0 = (t_lo + i) * kTcN;
+            const bool mine = my_q >= 0 && live;
 #pragma unroll 1
-            for (uint32_t cc = 0; cc < (uint32_t)kTcN; cc += 16) {
-                uint32_t v[16];
+            for (uint32_t cc = 0; cc < (uint32_t)kTcN; cc += 32) {
+                uint32_t v[32];
                 __syncwarp();
                 const uint32_t ta = tmem_base + ((warp * 32u) << 16) + b * kTcN + cc;
-                asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                             "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                             "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
                              : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                               "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                               "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                               "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                               "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
                              : "r"(ta));
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (my_q < 0 || !live) continue;
+                if (!mine) continue;
+                // fast filter: which of the 32 cosines reach the current cut at all?
+                float cut = have < p.K ? p.tau : fmaxf(p.tau, thr);
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const uint64_t c = c0 + cc + j;
-                    if (c >= nc) break;
-                    const float cs = __uint_as_float(v[j]) * qinv * __ldg(p.inv_norm + c);
-                    const long long cid = (long long)(p.cand_lo + c);
-                    if (!(cs > p.tau) || cid == my_q || (have == p.K && cs < thr)) continue;
-                    // sorted insertion into this thread's own list
-                    uint32_t pos = have;
-                    while (pos > 0 && ranks_ahead_tc(cs, cid, lc[pos - 1], li[pos - 1])) --pos;
-                    if (pos >= p.K) continue;
-                    const uint32_t last = have < p.K ? have : p.K - 1u;
-                    for (uint32_t s = last; s > pos; --s) { lc[s] = lc[s - 1]; li[s] = li[s - 1]; }
-                    lc[pos] = cs; li[pos] = cid;
-                    if (have < p.K) ++have;
-                    thr = have == p.K ? lc[p.K - 1] : p.tau;
+                for (int j = 0; j < 32; ++j) {
+                    const float cs = __uint_as_float(v[j]) * qinv * icn[cc + j];
+                    if (cs >= cut) {                               // rare: exact test and sorted insertion
+                        const uint64_t c = c0 + cc + j;
+                        if (c < nc) list_offer(lc, li, have, thr, p.K, p.tau, cs, (long long)(p.cand_lo + c), my_q);
+                        cut = have < p.K ? p.tau : fmaxf(p.tau, thr);
+                    }
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -261,11 +320,11 @@ topk_cosine_tc_kernel(TcParams p)
                     const uint32_t base = smem_addr(smem + (size_t)s * kTcStageBytes);
 #pragma unroll
                     for (int kk = 0; kk < kTcKB / 8; ++kk) {
-                        const uint32_t off = 2 * kk * kTcChunkStride;
+                        const uint32_t off = 2 * kk * kTcChunkStride, offc = 2 * kk * kTcChunkStrideC;
                         const uint64_t qh = umma_desc(base + 0 * kTcOperand + off, kTcChunkStride, 128);
                         const uint64_t ql = umma_desc(base + 1 * kTcOperand + off, kTcChunkStride, 128);
-                        const uint64_t ch = umma_desc(base + 2 * kTcOperand + off, kTcChunkStride, 128);
-                        const uint64_t cl = umma_desc(base + 3 * kTcOperand + off, kTcChunkStride, 128);
+                        const uint64_t ch = umma_desc(base + 2 * kTcOperand + offc, kTcChunkStrideC, 128);
+                        const uint64_t cl = umma_desc(base + 2 * kTcOperand + kTcOperandC + offc, kTcChunkStrideC, 128);
                         umma_tf32(dst, ql, ch, idesc, (kb | kk) ? 1u : 0u);      // small terms first
                         umma_tf32(dst, qh, cl, idesc, 1u);
                         umma_tf32(dst, qh, ch, idesc, 1u);
@@ -277,21 +336,28 @@ topk_cosine_tc_kernel(TcParams p)
         }
     } else {
         // ================= loaders =================
+        // group j fills stages j, j + kTcGroups, ...; the loads of a stage are issued before its slot
+        // is waited for, so they overlap the MMAs that still read the slot
         const uint32_t group = (tid - 5 * 32) / kTcLoaders, ltid = (tid - 5 * 32) % kTcLoaders;
-        uint64_t g = 0;
-        bool ok = true;
-        for (uint64_t i = 0; i < n_tiles && ok; ++i) {
-            const uint64_t c0 = (t_lo + i) * kTcN;
-            for (uint32_t kb = 0; kb < nkb; ++kb, ++g) {
-                if (g % kTcGroups != group) continue;
-                const uint32_t s = (uint32_t)(g % kTcStages);
-                ok = mbar_wait(empty + s, (uint32_t)(((g / kTcStages) & 1) ^ 1), abort_flag);
-                if (!ok) break;
-                unsigned char *st = smem + (size_t)s * kTcStageBytes;
-                load_stage(p, st, kb * kTcKB, ltid, qrow, c0, nc);
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // stores -> tensor-core reads
-                mbar_arrive(full + s);
+        const uint64_t total_g = n_tiles * nkb;
+        float4 x[kTcPer];
+        uint64_t g = group;
+        if (g < total_g) candidates_issue(p, x, (uint32_t)(g % nkb) * kTcKB, ltid, (t_lo + g / nkb) * kTcN, nc);
+        while (g < total_g) {
+            const uint32_t s = (uint32_t)(g % kTcStages), kb = (uint32_t)(g % nkb);
+            if (!mbar_wait(empty + s, (uint32_t)(((g / kTcStages) & 1) ^ 1), abort_flag)) break;
+            unsigned char *st = smem + (size_t)s * kTcStageBytes;
+            if (ltid == 0) {
+                // the query side arrives by bulk copy; its bytes complete the same barrier
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                             ::"r"(smem_addr(full + s)), "r"(2u * kTcOperand) : "memory");
+                bulk_to_smem(st, p.qsplit + ((size_t)blockIdx.x * nkb + kb) * 2 * kTcOperand, 2u * kTcOperand, full + s);
             }
+            candidates_store(st + 2 * kTcOperand, st + 2 * kTcOperand + kTcOperandC, x, ltid);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");         // stores -> tensor-core reads
+            if (ltid != 0) mbar_arrive(full + s);
+            g += kTcGroups;
+            if (g < total_g) candidates_issue(p, x, (uint32_t)(g % nkb) * kTcKB, ltid, (t_lo + g / nkb) * kTcN, nc);
         }
     }
     // ================= common exit =================
@@ -306,16 +372,28 @@ topk_cosine_tc_kernel(TcParams p)
 
 size_t topk_tc_smem_bytes()
 {
-    return (size_t)kTcStages * kTcStageBytes + (2 * kTcStages + 4) * 8 + 16 + kTcM * 8 + 128;
+    return (size_t)kTcStages * kTcStageBytes + (2 * kTcStages + 4) * 8 + 16 + kTcM * 8 + 8 * kTcN * 4 + 128;
 }
 
-// Returns 1, or -1 on a launch error.  Results go to part_* ([splits][m][K]); the caller merges.
+// Returns the launches made, or -1 on a launch error.  Results go to part_* ([splits][m][K]); the caller merges.
+size_t topk_tc_qsplit_bytes(uint64_t m, uint32_t d)
+{
+    const uint64_t qblocks = (m + kTcM - 1) / kTcM, nkb = (d + kTcKB - 1) / kTcKB;
+    return (size_t)(qblocks * nkb * 2 * kTcOperand);
+}
+
 int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, const long long *queries, uint64_t m,
-                   uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, const float *inv_norm, float *part_cos,
-                   long long *part_ids, uint32_t splits, int *error, cudaStream_t s)
+                   uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, const float *inv_norm,
+                   unsigned char *qsplit, float *part_cos, long long *part_ids, uint32_t splits, int *error,
+                   cudaStream_t s)
 {
     if (m == 0) return 0;
+    const uint32_t nkb = (d + kTcKB - 1) / kTcKB;
+    const unsigned qblocks = (unsigned)((m + kTcM - 1) / kTcM);
+    topk_split_queries_kernel<<<qblocks * nkb, 256, 0, s>>>(table, queries, m, vocab, d / 4, ld / 4, nkb, qsplit);
+    if (cudaGetLastError() != cudaSuccess) return -1;
     TcParams p;
+    p.qsplit = qsplit;
     p.table = table; p.queries = queries; p.inv_norm = inv_norm; p.part_cos = part_cos; p.part_ids = part_ids;
     p.error = error; p.m = m; p.vocab = vocab; p.cand_lo = cand_lo; p.cand_hi = cand_hi;
     p.d4 = d / 4; p.ld4 = ld / 4; p.K = K; p.splits = splits; p.tau = tau;
@@ -325,7 +403,7 @@ int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, 
     dim3 grid((unsigned)((m + kTcM - 1) / kTcM), splits);
     topk_cosine_tc_kernel<<<grid, kTcThreads, sm, s>>>(p);
     if (cudaGetLastError() != cudaSuccess) return -1;
-    return 1;
+    return 2;
 }
 
 }  // namespace w2v
