@@ -8,11 +8,11 @@
 // each k-step issues three MMAs into the same accumulator: lo.hi + hi.lo + hi.hi (the dropped lo.lo
 // term and the rounding of lo are below 2^-21 of |a||b| and unbiased).
 //
-// One block = 672 threads:
+// One block = 416 threads:
 //   warps 0-3  epilogue: warp w reads accumulator rows 32w .. 32w+31 (thread = one query) from
 //              tensor memory, scales by the inverse norms and keeps that query's sorted top-K list;
 //   warp 4     allocates tensor memory; one lane issues the MMAs;
-//   warps 5-20 loaders (two groups of 8 warps, one per stage of the ring): candidate rows -> (hi, lo) -> shared memory
+//   warps 5-12 loaders (two groups of 4 warps, one per stage of the ring): candidate rows -> (hi, lo) -> shared memory
 //              (the query side is split once by a pre-pass and arrives by cp.async.bulk), K-major core-matrix layout without
 //              swizzle ([16-byte column chunk][row][16 B], chunk stride 2064 B: conflict-free stores).
 // Shared-memory stages and the two accumulator buffers are handed over with mbarriers; every wait
@@ -32,7 +32,7 @@ constexpr int kTcOperand = 8 * kTcChunkStride;  // bytes of one query operand bl
 constexpr int kTcChunkStrideC = kTcN * 16 + 16; // the same for a candidate operand (256 rows)
 constexpr int kTcOperandC = 8 * kTcChunkStrideC;
 constexpr int kTcStageBytes = 2 * kTcOperand + 2 * kTcOperandC;   // Q hi, Q lo, C hi, C lo
-constexpr int kTcLoaders = 256;                 // threads that fill one stage together
+constexpr int kTcLoaders = 128;                 // threads that fill one stage together
 constexpr int kTcGroups = 2;                    // loader groups; group j fills stages j, j + 2, ...
 constexpr int kTcThreads = 5 * 32 + kTcGroups * kTcLoaders;
 constexpr uint32_t kTcSpinLimit = 1u << 20;
