@@ -7,7 +7,8 @@
 // operands staged through shared memory, k-major), scales them by the inverse norms and feeds the
 // ones that can still enter a query's list into that query's sorted top-K list in shared memory.
 // All arithmetic is fp32 on the CUDA cores: cosines agree with a double-precision evaluation to
-// ~1e-6, which the threshold and the ranking need; the tensor cores' TF32 inputs would not give that.
+// ~1e-6.  (w2v_topk_tc.cu is the tensor-core kernel for the same contract; this one is selected with
+// w2v_set_retrieval_kernel(h, 0).)  The merge kernel and the split plan below serve both.
 #include "w2v_device.cuh"
 #include "w2v_internal.h"
 
