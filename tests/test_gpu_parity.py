@@ -426,3 +426,34 @@ def test_resume_from_saved_rows_and_step_number():
     assert row_rel_err(again.read_rows(0, ids), gpu.read_rows(0, ids)) <= 2e-6     # atomics' order only
     assert row_rel_err(again.read_rows(1, ids), gpu.read_rows(1, ids)) <= 2e-6
     gpu.close(); again.close()
+
+
+def test_sampled_indices_random_chunk_structures():
+    # seeded random chunks: sentence lengths from 0 up, runs of sentinels, out-of-vocabulary ids, every
+    # window and negative count, with and without sub-sampling, several step numbers and interleavings
+    rng = np.random.default_rng(77)
+    V = 400
+    counts = rng.integers(1, 10**5, size=V).astype(np.uint64)
+    for case in range(40):
+        t = [0.0, 1e-3, 1e-2][case % 3]
+        gpu, cpu, _ = make_pair(dict(vocab=V, d=8), counts=counts, t=t, seed=1000 + case)
+        toks = []
+        for _ in range(int(rng.integers(0, 60))):
+            n = int(rng.integers(0, 70))
+            sent = rng.integers(0, V, size=n)
+            if n and rng.random() < 0.3:
+                sent[rng.integers(0, n)] = V + int(rng.integers(0, 5))         # out of vocabulary
+            if n and rng.random() < 0.1:
+                sent[rng.integers(0, n)] = -int(rng.integers(2, 9))
+            toks += list(sent) + [-1] * int(rng.integers(0 if n else 1, 3))
+        toks = np.asarray(toks, dtype=np.int32)
+        W, N = int(rng.integers(1, 20)), int(rng.integers(1, 40))
+        step = int(rng.integers(0, 2**40))
+        stride = int(rng.integers(1, 6)); phase = int(rng.integers(0, stride))
+        for m in (gpu, cpu):
+            m.set_step(step); m.set_interleave(phase, stride)
+        assert_same_pairs(gpu, cpu, toks, W, N)
+        c0, n0, _, ctx0 = cpu.cbow_examples(toks, W, N)
+        c1, n1, _ = gpu.sample_cbow(toks, W, N, allow=(binding.W2V_ERR_TOKEN_RANGE,)) if len(toks) else (c0, n0, None)
+        assert np.array_equal(c0, c1) and np.array_equal(n0, n1)
+        gpu.close()
