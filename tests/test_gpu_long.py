@@ -1,7 +1,7 @@
 """Hogwild-mode training at the lengths the acceptance criterion names: one pass over the small
 corpus (17 M tokens) and a 20 M-token prefix of the medium corpus, held-out loss of the GPU result
 against the sequential CPU checker's, three GPU repeats.  The checker needs several minutes per run
-on one core, so these are skipped unless W2V_LONG_TESTS=1; the design doc records the last results."""
+on one core, so these are skipped unless W2V_LONG_TESTS=1."""
 import os
 
 import numpy as np
