@@ -128,3 +128,21 @@ def test_shard_call_order_and_capacity_errors():
         with pytest.raises(binding.W2VError):
             binding.W2V(10, 16, 1, columns=(lo, hi))
     gpu.close()
+
+
+def test_sharded_step_with_interleaved_minibatches():
+    cfg = corpus.scaled(TINY, vocab=2000, d=100, minibatch=1500, corpus_tokens=100_000)
+    gpu, cpu, cp = make_sharded(cfg, 4)
+    W, N, lr, stride = cfg["window"], cfg["negatives"], 0.05, 5
+    toks = cp.chunk(0)
+    for phase in range(stride):
+        cpu.set_step(0); cpu.set_interleave(phase, stride)
+        for m in gpu.models:
+            m.set_step(0); m.set_interleave(phase, stride)
+        st = gpu.step(toks, W, N, lr)
+        so = cpu.step(toks, W, N, lr, 0)
+        assert st["pairs"] == so["pairs"] and st["centres"] == so["centres"]
+    ids = np.arange(cfg["vocab"])
+    assert row_rel_err(gpu.read_rows(0, ids), cpu.read_rows(0, ids)) <= SNAPSHOT_TOL
+    assert row_rel_err(gpu.read_rows(1, ids), cpu.read_rows(1, ids)) <= SNAPSHOT_TOL
+    gpu.close()
