@@ -229,6 +229,8 @@ def run_gpu(args):
     free_b, _ = torch.cuda.mem_get_info(dev)
     name = pick_workload(args.workload, free_b, args.row_stride)
     cfg = corpus.CONFIGS[name]
+    if args.tokens_per_step:
+        cfg = corpus.scaled(cfg, minibatch=args.tokens_per_step)
     cp = corpus.Corpus(cfg)
     W, N, lr, d = cfg["window"], cfg["negatives"], cfg["lr"], cfg["d"]
     K, Wu = args.steps, args.warmup
@@ -576,6 +578,8 @@ def main():
     ap.add_argument("--mode", choices=["hogwild", "snapshot", "sharded", "topk"], default="hogwild",
                     help="update mode of the timed steps (the headline number is hogwild); sharded = the "
                          "paper's column partition, --shards slices of one model on one GPU")
+    ap.add_argument("--tokens-per-step", type=int, default=0,
+                    help="word tokens per chunk (0 = the workload's own minibatch)")
     ap.add_argument("--shards", type=int, default=8)
     ap.add_argument("--model", choices=["sgns", "cbow"], default="sgns",
                     help="skip-gram (the headline) or the continuous-bag-of-words variant; for cbow the "
