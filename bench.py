@@ -409,7 +409,7 @@ def run_sharded(args):
     widest = max(hi - lo for lo, hi in shard_columns(d, S))
     aligned = (not args.dense_rows and
                2 * cfg["vocab"] * binding.aligned_row_stride(widest) * 4 * S + 12 * S * cfg["vocab"] + 8 * (1 << 30) < free_b)
-    model = LocalShards(cfg["vocab"], d, 1, S, device=dev, aligned_rows=aligned)
+    model = LocalShards(cfg["vocab"], d, 1, S, device=dev, aligned_rows=aligned, exchange=args.exchange)
     model.build_alias(cp.counts, cfg["subsample_t"])
     chunks = [torch.from_numpy(cp.chunk(i)).to(dev) for i in range(Wu + K)]
     for i in range(Wu):
@@ -444,7 +444,7 @@ def run_sharded(args):
         "data": "synthetic",
         "config": {"workload": name, "vocab": cfg["vocab"], "d": d, "window": W, "negatives": N,
                    "mode": "sharded", "shards": S, "columns": model.columns,
-                   "rows": "on 128-byte boundaries" if aligned else "dense",
+                   "rows": "on 128-byte boundaries" if aligned else "dense", "exchange": args.exchange,
                    "parallelism": f"{S} column shards run one after another on 1 gpu",
                    "pairs_per_step": tot_pairs / K,
                    "slowest_shard_ms_per_step": max(per_shard_ms) / K,
@@ -588,6 +588,9 @@ def main():
                     help="visit every chunk this many times, each time with 1/this of its input words "
                          "(interleaved minibatch formation)")
     ap.add_argument("--dense-rows", action="store_true", help="no padding between table rows")
+    ap.add_argument("--exchange", choices=["p2p", "allreduce"], default="p2p",
+                    help="--mode sharded: partial dots added into every shard's array by the producing kernel, "
+                         "or stored per shard and summed afterwards")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         print("note: fewer than 3 warm-up steps; not a valid timing", file=sys.stderr)

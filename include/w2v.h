@@ -242,7 +242,8 @@ int32_t w2v_create_shard(uint64_t vocab, uint32_t d_full, uint32_t col_lo, uint3
  * Algorithm 1 on this handle's columns for the chunk's index sets (sampled exactly as
  * w2v_sgns_step would).  Target number j = pair*(1+negatives) + t (t = 0 the context word,
  * t >= 1 negative t-1; pairs in the order of w2v_sample_pairs) gets its partial dot product
- * ADDED to F_peers[r][j] for every r < n_peers.
+ * ADDED to F_peers[r][j] for every r < n_peers; with n_peers == 1 it is STORED to F_peers[0][j]
+ * (the array then needs no zeroing; entries past the last target are left alone).
  *   tokens   device, n int32.
  *   F_peers  host array of n_peers (1..16) device pointers, each to cap floats that the caller
  *            zeroed before the first shard of this step adds to them; pointers into other

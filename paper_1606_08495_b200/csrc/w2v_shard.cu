@@ -83,10 +83,16 @@ shard_dots_kernel(StepParams p, ShardPeers peers)
                 [&](uint32_t t, const Row<VPL> &, float f) {
                     if (lane == (t & 31u)) { if (t < 32u) f0 = f; else f1 = f; }
                 });
-            for (uint32_t r = 0; r < peers.n; ++r) {
-                float *F = peers.F[r] + gi;
-                if (lane < n1p) atomicAdd(F + lane, f0);
-                if (lane + 32u < n1p) atomicAdd(F + lane + 32u, f1);
+            if (peers.n == 1) {                       // a single array: nobody else adds to it, plain stores
+                float *F = peers.F[0] + gi;
+                if (lane < n1p) F[lane] = f0;
+                if (lane + 32u < n1p) F[lane + 32u] = f1;
+            } else {
+                for (uint32_t r = 0; r < peers.n; ++r) {
+                    float *F = peers.F[r] + gi;
+                    if (lane < n1p) atomicAdd(F + lane, f0);
+                    if (lane + 32u < n1p) atomicAdd(F + lane + 32u, f1);
+                }
             }
             gi += n1p;
         }
@@ -220,8 +226,10 @@ shard_dots_list_kernel(StepParams p, ShardPeers peers)
 #pragma unroll
         for (int b = 0; b < TB; ++b) {
             const unsigned long long j = j0 + nr.grp + (unsigned long long)b * ngroups;
-            if (nr.sl == 0 && j < total)
-                for (uint32_t r = 0; r < peers.n; ++r) atomicAdd(peers.F[r] + j, f[b]);
+            if (nr.sl == 0 && j < total) {
+                if (peers.n == 1) peers.F[0][j] = f[b];           // a single array: plain stores
+                else for (uint32_t r = 0; r < peers.n; ++r) atomicAdd(peers.F[r] + j, f[b]);
+            }
         }
     }
 }

@@ -51,7 +51,13 @@ def _targets_capacity(n_tokens: int, window: int, negatives: int) -> int:
 class LocalShards:
     """S column shards of one model on one GPU (the ranks of the multi-GPU run, one after another)."""
 
-    def __init__(self, vocab, d, seed, shards, device="cuda:0", aligned_rows=False):
+    def __init__(self, vocab, d, seed, shards, device="cuda:0", aligned_rows=False, exchange="p2p"):
+        """exchange="p2p": every shard's kernel adds into every shard's array (peer pointers);
+        "allreduce": every shard stores its partials in its own array and the arrays are summed
+        afterwards, as an all-reduce would (here: a torch sum on the one GPU)."""
+        if exchange not in ("p2p", "allreduce"):
+            raise ValueError("exchange must be 'p2p' or 'allreduce'")
+        self.exchange = exchange
         self.vocab, self.d, self.seed = int(vocab), int(d), int(seed)
         self.columns = shard_columns(d, shards)
         self.device = torch.device(device)
@@ -85,13 +91,23 @@ class LocalShards:
         t = self.models[0]._dev_tokens(tokens)
         n = t.numel()
         self._ensure(_targets_capacity(n, window, negatives))
-        for f in self.F:
-            f.zero_()
         st = binding.StepStats()
-        for m in self.models:                                   # every shard adds into every shard's array
-            binding.w2v_shard_dots(m.h, t, n, window, negatives, self.F, self.cap, st)
-        for m, f in zip(self.models, self.F):                   # stream order stands in for the barrier
-            binding.w2v_shard_adjust(m.h, f, lr)
+        if self.exchange == "p2p":
+            for f in self.F:
+                f.zero_()
+            for m in self.models:                               # every shard adds into every shard's array
+                binding.w2v_shard_dots(m.h, t, n, window, negatives, self.F, self.cap, st)
+            for m, f in zip(self.models, self.F):               # stream order stands in for the barrier
+                binding.w2v_shard_adjust(m.h, f, lr)
+        else:
+            for m, f in zip(self.models, self.F):               # partials into the shard's own array
+                binding.w2v_shard_dots(m.h, t, n, window, negatives, [f], self.cap, st)
+            targets = st.pairs * (1 + negatives)
+            total = self.F[0][:targets]
+            for f in self.F[1:]:                                # the all-reduce, on one GPU
+                total += f[:targets]
+            for m in self.models:
+                binding.w2v_shard_adjust(m.h, total, lr)
         return st.as_dict()
 
     def read_rows(self, which, ids):
@@ -163,8 +179,7 @@ class DistributedShard:
             raise ValueError("chunk larger than the capacity this shard was created with")
         st = binding.StepStats()
         if self.exchange == "allreduce":
-            self.F.zero_()
-            binding.w2v_shard_dots(m.h, t, n, window, negatives, [self.F], self.cap, st)
+            binding.w2v_shard_dots(m.h, t, n, window, negatives, [self.F], self.cap, st)    # one array: stored
             targets = st.pairs * (1 + negatives)
             if targets:
                 self.dist.all_reduce(self.F[:targets], op=self.dist.ReduceOp.SUM, group=self.group)

@@ -19,9 +19,9 @@ SNAPSHOT_TOL = 1e-5
 TINY = corpus.CONFIGS["tiny"]
 
 
-def make_sharded(cfg, shards, seed=11, aligned=False):
+def make_sharded(cfg, shards, seed=11, aligned=False, exchange="p2p"):
     cp = corpus.Corpus(cfg)
-    gpu = LocalShards(cfg["vocab"], cfg["d"], seed, shards, aligned_rows=aligned)
+    gpu = LocalShards(cfg["vocab"], cfg["d"], seed, shards, aligned_rows=aligned, exchange=exchange)
     cpu = Oracle(cfg["vocab"], cfg["d"], seed)
     gpu.build_alias(cp.counts, cfg["subsample_t"])
     cpu.build_tables(cp.counts, cfg["subsample_t"])
@@ -39,11 +39,12 @@ def test_shards_hold_the_columns_of_the_whole_initial_model(d, shards):
     gpu.close()
 
 
+@pytest.mark.parametrize("exchange", ["p2p", "allreduce"])
 @pytest.mark.parametrize("d,shards,aligned", [(100, 1, False), (100, 2, False), (100, 3, True), (300, 8, False),
                                               (300, 10, True), (64, 16, False)])
-def test_sharded_step_equals_snapshot_step(d, shards, aligned):
+def test_sharded_step_equals_snapshot_step(d, shards, aligned, exchange):
     cfg = corpus.scaled(TINY, vocab=3000, d=d, minibatch=2000, corpus_tokens=100_000)
-    gpu, cpu, cp = make_sharded(cfg, shards, aligned=aligned)
+    gpu, cpu, cp = make_sharded(cfg, shards, aligned=aligned, exchange=exchange)
     W, N, lr = cfg["window"], cfg["negatives"], cfg["lr"]
     for i in range(3):
         toks = cp.chunk(i)
