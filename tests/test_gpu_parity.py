@@ -23,7 +23,7 @@ MEDIUM_CUT = corpus.scaled(corpus.CONFIGS["medium"], vocab=200_000, corpus_token
 
 
 # ---------------------------------------------------------------- initialisation and tables
-@pytest.mark.parametrize("vocab,d", [(1000, 100), (333, 4), (70, 300), (64, 1024), (5000, 200)])
+@pytest.mark.parametrize("vocab,d", [(1000, 100), (333, 4), (70, 300), (64, 1024), (5000, 200), (20000, 256)])
 def test_initial_tables_bit_exact(vocab, d):
     gpu = binding.W2V(vocab, d, seed=0xDEADBEEF12345)
     cpu = Oracle(vocab, d, seed=0xDEADBEEF12345)
