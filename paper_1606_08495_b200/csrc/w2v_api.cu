@@ -162,11 +162,18 @@ int32_t enqueue_sampling(w2v_handle *h, const int32_t *tokens, uint64_t n, uint3
     int32_t rc = ensure_scratch(h, n);
     if (rc != W2V_OK) return rc;
     h->shard_pending = false;            // the scratch a pending w2v_shard_adjust would need is overwritten
-    W2V_CUDA(h, cudaMemsetAsync(h->st, 0, sizeof(DevState), h->stream));
     const uint32_t k0 = (uint32_t)h->seed;
     const uint32_t k1 = (uint32_t)(h->seed >> 32) ^ (uint32_t)(h->step_id >> 32);
     const uint32_t step_lo = (uint32_t)h->step_id;
     SampleTables tab{h->keep_thr, h->alias};
+    if (n > 0 && n <= kSmallChunk) {
+        int k = launch_sample_small(tokens, n, tab, (uint32_t)h->vocab, k0, k1, step_lo, window, h->il_phase,
+                                    h->il_stride, h->sc, h->st, h->stream);
+        if (k < 0) return fail(h, W2V_ERR_CUDA, "sampling launch", cudaGetLastError());
+        h->launches += (uint64_t)k;
+        return W2V_OK;
+    }
+    W2V_CUDA(h, cudaMemsetAsync(h->st, 0, sizeof(DevState), h->stream));
     int k = launch_compact(tokens, n, tab, (uint32_t)h->vocab, k0, k1, step_lo, h->sc, h->st, h->stream);
     if (k < 0) return fail(h, W2V_ERR_CUDA, "compaction launch", cudaGetLastError());
     h->launches += (uint64_t)k;

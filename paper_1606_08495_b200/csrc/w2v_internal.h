@@ -100,6 +100,11 @@ int launch_windows(uint64_t n, uint32_t window, uint32_t k0, uint32_t k1, uint32
                    uint32_t il_phase, uint32_t il_stride, const Scratch &sc, DevState *st, cudaStream_t s);
 // pair_off[q] = number of pairs of the centres before q; with examples = true, the number of
 // centres before q that have at least one context (the example number of the CBOW variant)
+// chunks of at most kSmallChunk tokens: counters cleared, sub-sampling, compaction and windows in one launch
+constexpr uint64_t kSmallChunk = 8192;
+int launch_sample_small(const int32_t *tokens, uint64_t n, const SampleTables &tab, uint32_t vocab, uint32_t k0,
+                        uint32_t k1, uint32_t step_lo, uint32_t window, uint32_t il_phase, uint32_t il_stride,
+                        const Scratch &sc, DevState *st, cudaStream_t s);
 int launch_pair_offsets(uint64_t n, const Scratch &sc, DevState *st, cudaStream_t s, bool examples = false);
 
 // ---- continuous bag of words (w2v_cbow.cu) ----

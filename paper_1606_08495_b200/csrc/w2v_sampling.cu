@@ -231,6 +231,89 @@ emit_pairs_kernel(StepParams p, int32_t *__restrict__ centre, int32_t *__restric
     flush_draw_counts(p.st, draws, redraws);
 }
 
+// ---- small chunks: the whole integer half in one launch -------------------------------------
+// A chunk of at most kSmallChunk tokens is classified, compacted and given its windows by a single
+// block (the counters are cleared here too), so that a small step is two launches instead of six:
+// with chunks this small the step is bound by launches, not by the GPU.
+constexpr int kSmallBlock = 1024;
+constexpr int kSmallItems = 8;
+
+__global__ void __launch_bounds__(kSmallBlock)
+sample_small_kernel(const int32_t *__restrict__ tokens, uint32_t n, SampleTables tab, uint32_t vocab, uint32_t k0,
+                    uint32_t k1, uint32_t step_lo, uint32_t window, uint32_t il_phase, uint32_t il_stride,
+                    int32_t *__restrict__ ctok, uint32_t *__restrict__ cidx, uint32_t *__restrict__ csent,
+                    uint16_t *__restrict__ win, DevState *st)
+{
+    __shared__ uint32_t sh[33];
+    __shared__ uint32_t s_pairs, s_centres, s_oov;
+    const uint32_t base = threadIdx.x * kSmallItems;
+    if (threadIdx.x == 0) { s_pairs = 0; s_centres = 0; s_oov = 0; }
+    uint8_t f[kSmallItems];
+    uint32_t kept = 0, sent = 0, oov = 0;
+#pragma unroll
+    for (int e = 0; e < kSmallItems; ++e) {
+        const uint32_t i = base + e;
+        f[e] = 0;
+        if (i >= n) continue;
+        const int32_t w = tokens[i];
+        if (w == -1) {
+            f[e] = kFlagSentinel; ++sent;
+        } else if (w < 0 || (uint32_t)w >= vocab) {
+            ++oov;
+        } else {
+            const uint32_t thr = __ldg(tab.keep_thr + w);
+            bool keep = true;
+            if (thr != 0xFFFFFFFFu) keep = philox4x32_10(k0, k1, i, step_lo, kPurSubsample, 0).x < thr;
+            if (keep) { f[e] = kFlagKept; ++kept; }
+        }
+    }
+    uint32_t total;
+    const uint32_t ex = block_exclusive_scan<uint32_t>(kept | (sent << 16), sh, total);
+    uint32_t pos = ex & 0xFFFFu, sid = ex >> 16;
+#pragma unroll
+    for (int e = 0; e < kSmallItems; ++e) {
+        if (f[e] & kFlagKept) {
+            const uint32_t i = base + e;
+            ctok[pos] = tokens[i]; cidx[pos] = i; csent[pos] = sid;
+            ++pos;
+        }
+        sid += (f[e] & kFlagSentinel) >> 1;
+    }
+    if (oov) atomicAdd(&s_oov, oov);
+    __syncthreads();                                   // the compacted chunk is complete (block-wide)
+    const uint32_t nk = total & 0xFFFFu;
+    uint32_t pairs = 0, centres = 0;
+    for (uint32_t q = threadIdx.x; q < nk; q += kSmallBlock) {
+        const uint32_t i = cidx[q];
+        const uint32_t r = philox4x32_10(k0, k1, i, step_lo, kPurRadius, 0).x;
+        const uint32_t b = (il_stride > 1u && i % il_stride != il_phase) ? 0u : 1u + __umulhi(r, window);
+        const uint32_t sd = csent[q];
+        uint32_t left = 0, right = 0;
+        while (left < b && q >= left + 1u && csent[q - left - 1u] == sd) ++left;
+        while (right < b && q + right + 1u < nk && csent[q + right + 1u] == sd) ++right;
+        win[q] = (uint16_t)(left | (right << 8));
+        pairs += left + right;
+        centres += (left + right) ? 1u : 0u;
+    }
+    pairs = warp_sum(pairs); centres = warp_sum(centres);
+    if ((threadIdx.x & 31) == 0 && pairs) { atomicAdd(&s_pairs, pairs); atomicAdd(&s_centres, centres); }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        st->n_kept = nk; st->n_sent = total >> 16; st->centres = s_centres; st->pairs = s_pairs;
+        st->neg_draws = 0; st->neg_redraws = 0; st->oov = s_oov; st->status = s_oov ? 1u : 0u; st->pad = 0;
+    }
+}
+
+int launch_sample_small(const int32_t *tokens, uint64_t n, const SampleTables &tab, uint32_t vocab, uint32_t k0,
+                        uint32_t k1, uint32_t step_lo, uint32_t window, uint32_t il_phase, uint32_t il_stride,
+                        const Scratch &sc, DevState *st, cudaStream_t s)
+{
+    sample_small_kernel<<<1, kSmallBlock, 0, s>>>(tokens, (uint32_t)n, tab, vocab, k0, k1, step_lo, window, il_phase,
+                                                  il_stride, sc.ctok, sc.cidx, sc.csent, sc.win, st);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    return 1;
+}
+
 // ---- launchers ---------------------------------------------------------------------------
 static inline uint32_t tiles_for(uint64_t n) { return (uint32_t)((n + kScanTile - 1) / kScanTile); }
 
