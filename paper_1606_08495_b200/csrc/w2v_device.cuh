@@ -99,6 +99,38 @@ __device__ __forceinline__ void row_load(Row<VPL> &r, const float4 *base, uint32
     }
 }
 
+// Row touch: one 4-byte load per 64-byte DRAM burst of a row brings the whole row into L2 at
+// the price of one register per 2 KB of row (a full gather costs one per 16 bytes), so many
+// more rows can be in flight per warp.  NCH = touches per lane.  The last touch is the row's
+// last word: a row that does not start on a 64-byte boundary spans one burst more.
+template <int NCH>
+__device__ __forceinline__ void row_touch(uint32_t (&x)[NCH], const float4 *base, uint32_t d4, uint32_t lane)
+{
+    const char *b = reinterpret_cast<const char *>(base);
+    const uint32_t bytes = d4 * 16u, n = (bytes + 63u) / 64u + 1u;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+        const uint32_t idx = lane + 32u * c;
+        x[c] = 0u;
+        if (idx < n) {
+            const uint32_t off = idx * 64u < bytes ? idx * 64u : bytes - 4u;
+            asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(x[c]) : "l"(b + off));
+        }
+    }
+}
+
+// An offset that is always zero (`zero` is a kernel argument equal to 0) but that the hardware
+// can only compute once the touches have landed: added to the address of the additions that
+// follow, it makes them wait for the row to be in L2.
+template <int NCH>
+__device__ __forceinline__ uint32_t touch_fence(const uint32_t (&x)[NCH], uint32_t zero)
+{
+    uint32_t a = x[0];
+#pragma unroll
+    for (int c = 1; c < NCH; ++c) a |= x[c];
+    return a & zero;
+}
+
 template <int VPL>
 __device__ __forceinline__ float row_dot_partial(const Row<VPL> &a, const Row<VPL> &b)
 {

@@ -65,6 +65,7 @@ struct StepParams {
     const int32_t *l_negs;      // [pairs * negatives]
     double *DV;                 // [hot_rows * d] fp64 sums of G u(c) for the most-hit output rows
     uint32_t hot_rows;          // output rows [0, hot_rows) accumulate in DV (snapshot mode)
+    uint32_t zero;              // always 0; ANDed with a loaded word it ties a later address to that load's arrival
 };
 
 // F arrays of all shards (this one included) that receive a shard's partial dot products.

@@ -53,40 +53,86 @@ __device__ __forceinline__ uint32_t pair_target(uint32_t t, uint32_t w_out, uint
     return t == 0 ? w_out : r;
 }
 
-// Walks the targets of one (centre, context) pair in batches of TB rows so that TB row
-// gathers are in flight before the first dot is reduced.
-//   onTarget(t, target_row, v, f) is called once per target in order t = 0..N with the
-//   gathered row and the full dot product.
+// One batch of TB targets of a pair, t0..t0+TB-1: all TB row gathers are issued before the
+// first dot is reduced.  `off` (in float4) is added to every row address; it is zero, see
+// touch_fence.  onTarget(t, target_row, v, f) is called once per target with the gathered row
+// and the full dot product.
+template <int VPL, int TB, typename F>
+__device__ __forceinline__ void target_batch(const StepParams &p, const Row<VPL> &u, uint32_t w_out,
+                                             uint32_t n0, uint32_t n1, uint32_t lane, uint32_t t0,
+                                             uint32_t off, F &&onTarget)
+{
+    const float4 *V4 = reinterpret_cast<const float4 *>(p.V);
+    const bool wide = p.negatives > 32u;
+    uint32_t tgt[TB];
+    Row<VPL> v[TB];
+    float f[TB];
+#pragma unroll
+    for (int b = 0; b < TB; ++b) {
+        const uint32_t t = t0 + b;
+        tgt[b] = pair_target(t, w_out, n0, n1, wide);
+        if (t <= p.negatives) row_load(v[b], V4 + (size_t)tgt[b] * p.ld4 + off, p.d4, lane);
+        else row_zero(v[b]);
+    }
+#pragma unroll
+    for (int b = 0; b < TB; ++b) f[b] = row_dot_partial(u, v[b]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+        for (int b = 0; b < TB; ++b) f[b] += __shfl_xor_sync(kFullMask, f[b], o);
+    }
+#pragma unroll
+    for (int b = 0; b < TB; ++b) {
+        const uint32_t t = t0 + b;
+        if (t <= p.negatives) onTarget(t, tgt[b], v[b], f[b]);
+    }
+}
+
+// Walks the targets of one (centre, context) pair, t = 0..N in order, in batches of TB rows.
 template <int VPL, int TB, typename F>
 __device__ __forceinline__ void for_each_target(const StepParams &p, const Row<VPL> &u, uint32_t w_out,
                                                 uint32_t n0, uint32_t n1, uint32_t lane, F &&onTarget)
 {
+    for (uint32_t t0 = 0; t0 <= p.negatives; t0 += TB)
+        target_batch<VPL, TB>(p, u, w_out, n0, n1, lane, t0, 0u, onTarget);
+}
+
+// The same walk with the rows of the later batches (targets TB .. TB+kTouchAhead-1) touched
+// before the first batch is gathered: they arrive in L2 while the first batch is worked on, at
+// one register per row instead of the VPL*4 of a full gather, and the later batches wait for
+// them through the address offset.
+constexpr int kTouchAhead = 12;
+
+template <int VPL, int TB, typename F>
+__device__ __forceinline__ void for_each_target_touched(const StepParams &p, const Row<VPL> &u, uint32_t w_out,
+                                                        uint32_t n0, uint32_t n1, uint32_t lane, F &&onTarget)
+{
+    constexpr int NCH = (VPL + 3) / 4;
     const float4 *V4 = reinterpret_cast<const float4 *>(p.V);
     const bool wide = p.negatives > 32u;
-    for (uint32_t t0 = 0; t0 <= p.negatives; t0 += TB) {
-        uint32_t tgt[TB];
-        Row<VPL> v[TB];
-        float f[TB];
+    uint32_t any = 0u;
+    {
+        uint32_t x[kTouchAhead][NCH];
 #pragma unroll
-        for (int b = 0; b < TB; ++b) {
-            const uint32_t t = t0 + b;
-            tgt[b] = pair_target(t, w_out, n0, n1, wide);
-            if (t <= p.negatives) row_load(v[b], V4 + (size_t)tgt[b] * p.ld4, p.d4, lane);
-            else row_zero(v[b]);
+        for (int b = 0; b < kTouchAhead; ++b) {
+            const uint32_t t = (uint32_t)(TB + b);
+            const uint32_t tgt = pair_target(t, w_out, n0, n1, wide);
+            if (t <= p.negatives) row_touch<NCH>(x[b], V4 + (size_t)tgt * p.ld4, p.d4, lane);
+            else {
+#pragma unroll
+                for (int k = 0; k < NCH; ++k) x[b][k] = 0u;
+            }
         }
+        target_batch<VPL, TB>(p, u, w_out, n0, n1, lane, 0u, 0u, onTarget);
 #pragma unroll
-        for (int b = 0; b < TB; ++b) f[b] = row_dot_partial(u, v[b]);
+        for (int b = 0; b < kTouchAhead; ++b) {
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-            for (int b = 0; b < TB; ++b) f[b] += __shfl_xor_sync(kFullMask, f[b], o);
-        }
-#pragma unroll
-        for (int b = 0; b < TB; ++b) {
-            const uint32_t t = t0 + b;
-            if (t <= p.negatives) onTarget(t, tgt[b], v[b], f[b]);
+            for (int k = 0; k < NCH; ++k) any |= x[b][k];
         }
     }
+    const uint32_t off = any & p.zero;
+    for (uint32_t t0 = TB; t0 <= p.negatives; t0 += TB)
+        target_batch<VPL, TB>(p, u, w_out, n0, n1, lane, t0, off, onTarget);
 }
 
 __device__ __forceinline__ void flush_draw_counts(DevState *st, uint32_t draws, uint32_t redraws)
