@@ -472,11 +472,11 @@ def run_topk(args):
     name = args.workload or "sponsored"
     cfg = corpus.CONFIGS[name]
     V, d = cfg["vocab"], cfg["d"]
-    K, tau, m = 30, 0.65, args.queries
+    K, tau, m = 30, args.tau, args.queries
     lo, hi = int(V * 0.85), V
     model = binding.W2V(V, d, seed=1, device=dev, row_stride=row_stride_for(d, args.row_stride))
-    tensor = args.retrieval_kernel == "tensor"
-    binding.w2v_set_retrieval_kernel(model.h, 1 if tensor else 0)
+    tensor = args.retrieval_kernel != "fp32"
+    binding.w2v_set_retrieval_kernel(model.h, {"fp32": 0, "tensor": 1, "screen": 2}[args.retrieval_kernel])
     # spread-out vectors instead of the tiny uniform initial ones: normal rows, so that cosines have the
     # spread of unrelated trained vectors (about N(0, 1/d)); written by torch, this is input data
     g = torch.Generator(device=dev); g.manual_seed(5)
@@ -532,7 +532,9 @@ def run_topk(args):
         except Exception:
             bf16, kind = 1400.0, "fallback sustained bf16 x 1.1/2.25"
         peak, bound = bf16 * 1.1 / 2.25, "tensor"
-        peak_kind = kind + " (tf32); the kernel issues 3 MMA flops per useful flop"
+        mma_per_product = 3 if args.retrieval_kernel == "tensor" else 1
+        peak_kind = kind + (" (tf32); the kernel issues 3 MMA flops per useful flop" if mma_per_product == 3 else
+                            " (tf32); one MMA flop per useful flop, plus fp32 dot products for the candidates near the cut")
     else:
         peak, bound = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12, "alu"     # fp32 FMA lanes x 2 flop x clock, TFLOP/s
         peak_kind = "148 SMs x 128 fp32 FMA lanes x 2 flop x max SM clock"
@@ -542,15 +544,18 @@ def run_topk(args):
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": name + " (retrieval)", "vocab": V, "d": d, "queries_per_step": m,
                    "candidates": hi - lo, "K": K, "tau": tau, "row_stride_floats": model.row_stride,
-                   "kernel": "tcgen05 tf32, head/tail split (3 MMAs per product)" if tensor else "fp32 CUDA cores",
+                   "kernel": {"tensor": "tcgen05 tf32, head/tail split (3 MMAs per product)",
+                              "screen": "tcgen05 tf32 screen (1 MMA per product) + exact fp32 cosines near the cut",
+                              "fp32": "fp32 CUDA cores"}[args.retrieval_kernel],
                    "l2": "3 M candidate rows (3.8 GB) streamed per call, far larger than L2"},
         "clocks": clocks,
         "e2e": {"value": cosines / (e2e_ms * 1e-3), "unit": "cosines/s", "h2d_bytes_per_step": 8 * m,
                 "d2h_bytes_per_step": 12 * m * K},
         "gpu_launches": launches,
-        "roofline": {"bound": bound, "kernel": "topk_cosine_tc_kernel" if tensor else "topk_cosine_kernel",
+        "roofline": {"bound": bound, "kernel": {"tensor": "topk_cosine_tc_kernel", "screen": "topk_cosine_screen_kernel",
+                                                "fp32": "topk_cosine_kernel"}[args.retrieval_kernel],
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                     "mma_tflops_issued": 3 * achieved if tensor else None,
+                     "mma_tflops_issued": mma_per_product * achieved if tensor else None,
                      "peak_kind": peak_kind,
                      "flops_per_launch": flops / Ksteps, "kernel_ms_per_launch": kernel_ms / Ksteps, "traffic": None},
     }
@@ -574,7 +579,8 @@ def main():
     ap.add_argument("--ref-words", type=int, default=20_000, help="word tokens per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--queries", type=int, default=8192, help="query rows per call of --mode topk")
-    ap.add_argument("--retrieval-kernel", choices=["fp32", "tensor"], default="tensor")
+    ap.add_argument("--retrieval-kernel", choices=["fp32", "tensor", "screen"], default="screen")
+    ap.add_argument("--tau", type=float, default=0.65, help="similarity threshold of --mode topk (-2 keeps everything)")
     ap.add_argument("--mode", choices=["hogwild", "snapshot", "sharded", "topk"], default="hogwild",
                     help="update mode of the timed steps (the headline number is hogwild); sharded = the "
                          "paper's column partition, --shards slices of one model on one GPU")

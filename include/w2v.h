@@ -314,12 +314,18 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
 /*
  * Which kernel w2v_topk_cosine runs (the paper has no say in this):
  *   0  fp32 multiply-adds on the CUDA cores: cosines within about 1e-6 of exact;
- *   1  the tensor cores (the default): every value is split into a TF32 head and a TF32 tail and
+ *   1  the tensor cores: every value is split into a TF32 head and a TF32 tail and
  *      each product is formed as head*head + head*tail + tail*head in fp32 accumulators that the
  *      hardware updates 3 d/8 times with rounding toward zero: cosines within about
  *      2e-6 + 3 (d/8) 2^-24 of exact (9e-6 at d = 300; 2e-6 typical), at three times the speed.
- *      A block of this kernel that waits too long on its own pipeline gives up; w2v_sync then
- *      returns W2V_ERR_CUDA.
+ *   2  the tensor cores as a screen (the default): one TF32 product per pair of values gives every
+ *      cosine to about 1.5e-3, which decides for all but a few candidates that they cannot reach
+ *      the query's current K-th best (or tau); the few within 2e-3 of it are recomputed as fp32
+ *      dot products of the two rows, and only those values are ranked and returned: cosines within
+ *      about 1e-6 of exact, as with kind 0.  Rows of more than 320 columns do not fit this
+ *      kernel's shared-memory plan and are handled as kind 1.
+ *   A block of kind 1 or 2 that waits too long on its own pipeline gives up; w2v_sync then
+ *   returns W2V_ERR_CUDA.
  */
 int32_t w2v_set_retrieval_kernel(w2v_handle *h, uint32_t kind);
 

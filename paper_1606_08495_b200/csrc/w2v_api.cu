@@ -24,7 +24,7 @@ struct w2v_handle {
     uint64_t l_cap_pairs = 0, l_cap_negs = 0;
     float *inv_norm = nullptr; uint64_t inv_norm_cap = 0;                      // retrieval scratch
     float *part_cos = nullptr; long long *part_ids = nullptr; uint64_t part_cap = 0;
-    uint32_t retrieval_kernel = 1;       // 0: fp32 on the CUDA cores, 1: tensor cores (3 x TF32)
+    uint32_t retrieval_kernel = 2;       // 0: fp32 on the CUDA cores, 1: tensor cores (3 x TF32), 2: tensor-core screen + exact fp32
     int *tc_error = nullptr;             // device word raised by a tensor-core block whose wait ran out
     unsigned char *qsplit = nullptr; uint64_t qsplit_cap = 0;   // query rows split into TF32 head and tail
     uint32_t pend_window = 0, pend_negatives = 0;
@@ -738,7 +738,7 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
         h->inv_norm_cap = nc;
     }
     // few query blocks: split the candidates over several blocks per query block, merge afterwards
-    const bool tc = h->retrieval_kernel == 1;
+    const bool tc = h->retrieval_kernel >= 1;
     const uint64_t splits = tc ? topk_splits(m, nc, h->sms, 128, 256) : topk_splits(m, nc, h->sms);
     const uint64_t need = (splits > 1 || tc) ? splits * m * K : 0;
     if (tc && topk_tc_qsplit_bytes(m, h->d) > h->qsplit_cap) {
@@ -768,7 +768,7 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
     if (tc) {
         k2 = launch_topk_tc(table, h->d, h->ld, h->vocab, reinterpret_cast<const long long *>(queries), m, cand_lo,
                             cand_hi, K, tau, h->inv_norm, h->qsplit, h->part_cos, h->part_ids, (uint32_t)splits,
-                            h->tc_error, h->stream);
+                            h->tc_error, h->retrieval_kernel == 2, h->stream);
         if (k2 >= 0) {
             const int k3 = launch_topk_merge(h->part_cos, h->part_ids, m, K, (uint32_t)splits, out_cos,
                                              reinterpret_cast<long long *>(out_ids), h->sms, h->stream);
@@ -845,7 +845,7 @@ int32_t w2v_sync(w2v_handle *h)
 int32_t w2v_set_retrieval_kernel(w2v_handle *h, uint32_t kind)
 {
     if (!h) return W2V_ERR_ARG;
-    if (kind > 1) return fail(h, W2V_ERR_ARG, "kind must be 0 (fp32 CUDA cores) or 1 (tensor cores)");
+    if (kind > 2) return fail(h, W2V_ERR_ARG, "kind must be 0 (fp32 CUDA cores), 1 (tensor cores) or 2 (tensor-core screen)");
     h->retrieval_kernel = kind;
     return W2V_OK;
 }

@@ -148,7 +148,9 @@ size_t topk_tc_qsplit_bytes(uint64_t m, uint32_t d);
 int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, const long long *queries, uint64_t m,
                    uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, const float *inv_norm,
                    unsigned char *qsplit, float *part_cos, long long *part_ids, uint32_t splits, int *error,
-                   cudaStream_t s);
+                   bool screen, cudaStream_t s);
+// whether the screening variant (query block resident in shared memory) can take rows of d columns
+bool topk_screen_fits(uint32_t d);
 int launch_inv_norms(const float *table, uint32_t d, uint32_t ld, uint64_t lo, uint64_t count, float *inv_norm,
                      int sms, cudaStream_t s);
 // Returns launches made, -1 on a launch error, -2 if the shape does not fit shared memory.
