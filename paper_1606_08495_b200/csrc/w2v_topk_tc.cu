@@ -534,20 +534,20 @@ topk_cosine_screen_kernel(TcParams p)
                     const uint32_t j = __shfl_sync(kFullMask, (uint32_t)__ffs((int)maybe) - 1u, src);
                     const long long qr = qrow[warp * 32u + src];
                     const uint64_t c = c0 + cc + j;
-                    const float dot = warp_row_dot(T4, (size_t)qr, (size_t)(p.cand_lo + c), p.d4, p.ld4, lane);
-                    const float cs = dot * __shfl_sync(kFullMask, qinv, src) * __shfl_sync(kFullMask, icv, j);
                     const long long cid = (long long)(p.cand_lo + c);
                     const uint32_t hv = __shfl_sync(kFullMask, have, src);
                     const float th = __shfl_sync(kFullMask, thr, src);
                     if (lane == src) maybe &= maybe - 1u;
-                    if (!(cs > p.tau) || cid == qr || (hv == p.K && cs < th)) continue;     // same for every lane
-                    // sorted insertion into query src's list by the whole warp: lane l holds entries l and l + 32
+                    // query src's sorted list, lane l holding entries l and l + 32 (read while the rows are fetched)
                     float *wl = p.part_cos + ((size_t)blockIdx.y * p.m + (q0 + warp * 32u + src)) * p.K;
                     long long *wi = p.part_ids + ((size_t)blockIdx.y * p.m + (q0 + warp * 32u + src)) * p.K;
                     float e0 = 0.f, e1 = 0.f;
                     long long i0 = -1, i1 = -1;
                     if (lane < hv) { e0 = __ldcg(wl + lane); i0 = __ldcg(wi + lane); }
                     if (lane + 32u < hv) { e1 = __ldcg(wl + lane + 32u); i1 = __ldcg(wi + lane + 32u); }
+                    const float dot = warp_row_dot(T4, (size_t)qr, (size_t)(p.cand_lo + c), p.d4, p.ld4, lane);
+                    const float cs = dot * __shfl_sync(kFullMask, qinv, src) * __shfl_sync(kFullMask, icv, j);
+                    if (!(cs > p.tau) || cid == qr || (hv == p.K && cs < th)) continue;     // same for every lane
                     const bool a0 = lane < hv && !ranks_ahead_tc(cs, cid, e0, i0);         // entries that stay ahead: a prefix
                     const bool a1 = lane + 32u < hv && !ranks_ahead_tc(cs, cid, e1, i1);
                     const uint32_t pos = (uint32_t)__popc(__ballot_sync(kFullMask, a0)) + (uint32_t)__popc(__ballot_sync(kFullMask, a1));
