@@ -131,9 +131,7 @@ cbow_snap_adjust_v_kernel(StepParams p)
     const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
     const uint32_t nk = (uint32_t)p.st->n_kept;
-    float4 *V4 = reinterpret_cast<float4 *>(p.V);
     const uint32_t n1p = p.negatives + 1u;
-    const bool wide = p.negatives > 32u;
     uint32_t draws = 0, redraws = 0;    // regenerated draws are not counted twice
     for (uint32_t q = warp; q < nk; q += nwarps) {
         const uint32_t w = p.win[q];
@@ -145,13 +143,7 @@ cbow_snap_adjust_v_kernel(StepParams p)
         context_mean<VPL, TB>(p, q, left, cw, lane, h, inv);
         uint32_t n0, n1;
         draw_pair_negatives(p, p.cidx[q], p.window, wq, lane, n0, n1, draws, redraws);
-        const size_t gi = (size_t)q * n1p;
-        for (uint32_t t = 0; t <= p.negatives; ++t) {
-            const uint32_t tgt = pair_target(t, wq, n0, n1, wide);
-            const float g = __ldcg(p.G + gi + t);
-            if (tgt < p.hot_rows) row_add_scaled_f64(p.DV + (size_t)tgt * (4u * p.d4), g, h, p.d4, lane);
-            else row_red_scaled(V4 + (size_t)tgt * p.ld4, g, h, p.d4, lane);
-        }
+        adjust_targets<VPL>(p, h, wq, n0, n1, (unsigned long long)q * n1p, lane);
     }
 }
 

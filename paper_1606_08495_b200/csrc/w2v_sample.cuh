@@ -135,6 +135,45 @@ __device__ __forceinline__ void for_each_target_touched(const StepParams &p, con
         target_batch<VPL, TB>(p, u, w_out, n0, n1, lane, t0, off, onTarget);
 }
 
+// Algorithm 2 for the output rows of one pair (or one CBOW example): v(t) += G[gi + t] * r for
+// t = 0..N.  An addition that has to fetch its line costs the memory system more than one that
+// finds it in L2, so the rows of a batch of targets are touched first (one word per DRAM burst,
+// see row_touch) and the additions' addresses wait for the touches.  The most-hit rows collect
+// in double precision (DV) instead.
+constexpr int kTouchBatch = 12;
+
+template <int VPL>
+__device__ __forceinline__ void adjust_targets(const StepParams &p, const Row<VPL> &r, uint32_t w_out, uint32_t n0,
+                                               uint32_t n1, unsigned long long gi, uint32_t lane)
+{
+    constexpr int NCH = (VPL + 3) / 4;
+    float4 *V4 = reinterpret_cast<float4 *>(p.V);
+    const uint32_t n1p = p.negatives + 1u;
+    const bool wide = p.negatives > 32u;
+    for (uint32_t t0 = 0; t0 < n1p; t0 += kTouchBatch) {
+        const uint32_t nb = n1p - t0 < (uint32_t)kTouchBatch ? n1p - t0 : (uint32_t)kTouchBatch;
+        const float gl = lane < nb ? __ldcg(p.G + gi + t0 + lane) : 0.f;   // lane b: coefficient of target t0 + b
+        uint32_t tgt[kTouchBatch], x[kTouchBatch][NCH];
+#pragma unroll
+        for (int b = 0; b < kTouchBatch; ++b) {
+            tgt[b] = pair_target(t0 + b, w_out, n0, n1, wide);
+            if ((uint32_t)b < nb && tgt[b] >= p.hot_rows) row_touch<NCH>(x[b], V4 + (size_t)tgt[b] * p.ld4, p.d4, lane);
+            else {
+#pragma unroll
+                for (int k = 0; k < NCH; ++k) x[b][k] = 0u;
+            }
+        }
+#pragma unroll
+        for (int b = 0; b < kTouchBatch; ++b) {
+            const float g = __shfl_sync(kFullMask, gl, b);
+            if ((uint32_t)b < nb) {
+                if (tgt[b] < p.hot_rows) row_add_scaled_f64(p.DV + (size_t)tgt[b] * (4u * p.d4), g, r, p.d4, lane);
+                else row_red_scaled(V4 + (size_t)tgt[b] * p.ld4 + touch_fence<NCH>(x[b], p.zero), g, r, p.d4, lane);
+            }
+        }
+    }
+}
+
 __device__ __forceinline__ void flush_draw_counts(DevState *st, uint32_t draws, uint32_t redraws)
 {
     const uint32_t d = warp_sum(draws), r = warp_sum(redraws);

@@ -102,25 +102,17 @@ sgns_snap_dots_kernel(StepParams p)
 }
 
 // ---- snapshot mode, pass 2 (Algorithm 2, output rows): v(target) += G u(c) ------------------
-// U is still untouched, so u(c) is the start-of-step vector; V is only added to.  An addition
-// that has to fetch its line costs the memory system far more than one that finds it in L2, so
-// the rows of a batch of targets are touched first (one word per DRAM burst, see row_touch) and
-// the additions are issued when the touches have landed.
-constexpr int kTouchBatch = 12;
-
+// U is still untouched, so u(c) is the start-of-step vector; V is only added to (adjust_targets).
 template <int VPL>
 __global__ void __launch_bounds__(kBlock)
 sgns_snap_adjust_v_kernel(StepParams p)
 {
-    constexpr int NCH = (VPL + 3) / 4;
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
     const uint32_t nk = (uint32_t)p.st->n_kept;
     const float4 *U4 = reinterpret_cast<const float4 *>(p.U);
-    float4 *V4 = reinterpret_cast<float4 *>(p.V);
     const uint32_t n1p = p.negatives + 1u;
-    const bool wide = p.negatives > 32u;
     uint32_t draws = 0, redraws = 0;   // regenerated draws are not counted twice
     for (uint32_t q = warp; q < nk; q += nwarps) {
         const uint32_t w = p.win[q];
@@ -136,28 +128,7 @@ sgns_snap_adjust_v_kernel(StepParams p)
             const uint32_t w_out = (uint32_t)p.ctok[pp];
             uint32_t n0, n1;
             draw_pair_negatives(p, i, pp + p.window - q, w_out, lane, n0, n1, draws, redraws);
-            for (uint32_t t0 = 0; t0 < n1p; t0 += kTouchBatch) {
-                const uint32_t nb = n1p - t0 < (uint32_t)kTouchBatch ? n1p - t0 : (uint32_t)kTouchBatch;
-                const float gl = lane < nb ? __ldcg(p.G + gi + t0 + lane) : 0.f;   // lane b: coefficient of target t0+b
-                uint32_t tgt[kTouchBatch], x[kTouchBatch][NCH];
-#pragma unroll
-                for (int b = 0; b < kTouchBatch; ++b) {
-                    tgt[b] = pair_target(t0 + b, w_out, n0, n1, wide);
-                    if ((uint32_t)b < nb && tgt[b] >= p.hot_rows) row_touch<NCH>(x[b], V4 + (size_t)tgt[b] * p.ld4, p.d4, lane);
-                    else {
-#pragma unroll
-                        for (int k = 0; k < NCH; ++k) x[b][k] = 0u;
-                    }
-                }
-#pragma unroll
-                for (int b = 0; b < kTouchBatch; ++b) {
-                    const float g = __shfl_sync(kFullMask, gl, b);
-                    if ((uint32_t)b < nb) {
-                        if (tgt[b] < p.hot_rows) row_add_scaled_f64(p.DV + (size_t)tgt[b] * (4u * p.d4), g, u, p.d4, lane);
-                        else row_red_scaled(V4 + (size_t)tgt[b] * p.ld4 + touch_fence<NCH>(x[b], p.zero), g, u, p.d4, lane);
-                    }
-                }
-            }
+            adjust_targets<VPL>(p, u, w_out, n0, n1, gi, lane);
             gi += n1p;
         }
     }
