@@ -531,10 +531,14 @@ def run_topk(args):
                 bf16, kind = float(json.load(f)["bf16_tflops_sustained"]), "measured sustained bf16 x 1.1/2.25"
         except Exception:
             bf16, kind = 1400.0, "fallback sustained bf16 x 1.1/2.25"
-        peak, bound = bf16 * 1.1 / 2.25, "tensor"
+        bound = "tensor"
         mma_per_product = 3 if args.retrieval_kernel == "tensor" else 1
-        peak_kind = kind + (" (tf32); the kernel issues 3 MMA flops per useful flop" if mma_per_product == 3 else
-                            " (tf32); one MMA flop per useful flop, plus fp32 dot products for the candidates near the cut")
+        if mma_per_product == 3:
+            peak = bf16 * 1.1 / 2.25
+            peak_kind = kind + " (tf32); the kernel issues 3 MMA flops per useful flop"
+        else:
+            peak = bf16        # the screen's MMAs are bf16 x bf16 -> fp32
+            peak_kind = kind.replace(" x 1.1/2.25", "") + "; one bf16 MMA flop per useful flop, plus fp32 dot products for the candidates near the cut"
     else:
         peak, bound = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12, "alu"     # fp32 FMA lanes x 2 flop x clock, TFLOP/s
         peak_kind = "148 SMs x 128 fp32 FMA lanes x 2 flop x max SM clock"
@@ -545,7 +549,7 @@ def run_topk(args):
         "config": {"workload": name + " (retrieval)", "vocab": V, "d": d, "queries_per_step": m,
                    "candidates": hi - lo, "K": K, "tau": tau, "row_stride_floats": model.row_stride,
                    "kernel": {"tensor": "tcgen05 tf32, head/tail split (3 MMAs per product)",
-                              "screen": "tcgen05 tf32 screen (1 MMA per product) + exact fp32 cosines near the cut",
+                              "screen": "tcgen05 bf16 screen (1 MMA per product) + exact fp32 cosines near the cut",
                               "fp32": "fp32 CUDA cores"}[args.retrieval_kernel],
                    "l2": "3 M candidate rows (3.8 GB) streamed per call, far larger than L2"},
         "clocks": clocks,

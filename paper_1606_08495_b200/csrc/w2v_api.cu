@@ -27,6 +27,7 @@ struct w2v_handle {
     uint32_t retrieval_kernel = 2;       // 0: fp32 on the CUDA cores, 1: tensor cores (3 x TF32), 2: tensor-core screen + exact fp32
     int *tc_error = nullptr;             // device word raised by a tensor-core block whose wait ran out
     unsigned char *qsplit = nullptr; uint64_t qsplit_cap = 0;   // query rows split into TF32 head and tail
+    unsigned char *ctiles = nullptr; uint64_t ctiles_cap = 0;   // candidate rows packed as bf16 operand blocks (screening kernel)
     uint32_t pend_window = 0, pend_negatives = 0;
     uint64_t pend_n = 0, pend_pairs = 0;
     uint64_t seed = 0;
@@ -408,7 +409,7 @@ int32_t w2v_destroy(w2v_handle *h)
     if (h->st_host) cudaFreeHost(h->st_host);
     cudaFree(h->G); cudaFree(h->DU); cudaFree(h->DV); cudaFree(h->tok_stage);
     cudaFree(h->l_centre); cudaFree(h->l_context); cudaFree(h->l_negs);
-    cudaFree(h->inv_norm); cudaFree(h->part_cos); cudaFree(h->part_ids); cudaFree(h->tc_error); cudaFree(h->qsplit);
+    cudaFree(h->inv_norm); cudaFree(h->part_cos); cudaFree(h->part_ids); cudaFree(h->tc_error); cudaFree(h->qsplit); cudaFree(h->ctiles);
     for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
     cudaGetLastError();
     delete h;
@@ -739,8 +740,20 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
     }
     // few query blocks: split the candidates over several blocks per query block, merge afterwards
     const bool tc = h->retrieval_kernel >= 1;
-    const uint64_t splits = tc ? topk_splits(m, nc, h->sms, 128, 256) : topk_splits(m, nc, h->sms);
-    const uint64_t need = (splits > 1 || tc) ? splits * m * K : 0;
+    const bool screen = h->retrieval_kernel == 2 && topk_screen_fits(h->d);
+    // the screening kernel takes the candidates in chunks, each with its own set of partial lists
+    const uint64_t chunk = screen ? topk_screen_chunk(nc) : nc;
+    const uint64_t chunks = chunk ? (nc + chunk - 1) / chunk : 0;
+    const uint64_t splits = tc ? topk_splits(m, chunk, h->sms, 128, 256) : topk_splits(m, nc, h->sms);
+    const uint64_t lists = screen ? chunks * splits : splits;
+    const uint64_t need = (splits > 1 || tc) ? lists * m * K : 0;
+    if (screen && topk_screen_ctiles_bytes(nc, h->d) > h->ctiles_cap) {
+        W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+        cudaFree(h->ctiles); h->ctiles = nullptr; h->ctiles_cap = 0;
+        const uint64_t bytes = topk_screen_ctiles_bytes(nc, h->d);
+        W2V_CUDA(h, dev_alloc(&h->ctiles, bytes));
+        h->ctiles_cap = bytes;
+    }
     if (tc && topk_tc_qsplit_bytes(m, h->d) > h->qsplit_cap) {
         W2V_CUDA(h, cudaStreamSynchronize(h->stream));
         cudaFree(h->qsplit); h->qsplit = nullptr; h->qsplit_cap = 0;
@@ -767,10 +780,10 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
     int k2;
     if (tc) {
         k2 = launch_topk_tc(table, h->d, h->ld, h->vocab, reinterpret_cast<const long long *>(queries), m, cand_lo,
-                            cand_hi, K, tau, h->inv_norm, h->qsplit, h->part_cos, h->part_ids, (uint32_t)splits,
-                            h->tc_error, h->retrieval_kernel == 2, h->stream);
+                            cand_hi, K, tau, h->inv_norm, h->qsplit, h->ctiles, h->part_cos, h->part_ids, (uint32_t)splits,
+                            h->tc_error, screen, h->sms, h->stream);
         if (k2 >= 0) {
-            const int k3 = launch_topk_merge(h->part_cos, h->part_ids, m, K, (uint32_t)splits, out_cos,
+            const int k3 = launch_topk_merge(h->part_cos, h->part_ids, m, K, (uint32_t)lists, out_cos,
                                              reinterpret_cast<long long *>(out_ids), h->sms, h->stream);
             k2 = k3 < 0 ? -1 : k2 + k3;
         }

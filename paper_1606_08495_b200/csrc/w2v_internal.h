@@ -147,9 +147,13 @@ int launch_topk_merge(const float *part_cos, const long long *part_ids, uint64_t
 size_t topk_tc_qsplit_bytes(uint64_t m, uint32_t d);
 int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, const long long *queries, uint64_t m,
                    uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, const float *inv_norm,
-                   unsigned char *qsplit, float *part_cos, long long *part_ids, uint32_t splits, int *error,
-                   bool screen, cudaStream_t s);
-// whether the screening variant (query block resident in shared memory) can take rows of d columns
+                   unsigned char *qsplit, unsigned char *ctiles, float *part_cos, long long *part_ids, uint32_t splits,
+                   int *error, bool screen, int sms, cudaStream_t s);
+// The screening variant: whether it can take rows of d columns; how many candidates it handles per
+// launch (a range is cut into chunks of that size, each with its own partial lists); bytes of the
+// packed bf16 copy of one chunk.
+uint64_t topk_screen_chunk(uint64_t n_candidates);
+size_t topk_screen_ctiles_bytes(uint64_t n_candidates, uint32_t d);
 bool topk_screen_fits(uint32_t d);
 int launch_inv_norms(const float *table, uint32_t d, uint32_t ld, uint64_t lo, uint64_t count, float *inv_norm,
                      int sms, cudaStream_t s);

@@ -112,6 +112,7 @@ struct TcParams {
     const long long *queries;
     const float *inv_norm;
     const unsigned char *qsplit;  // [query blocks][K-blocks][hi, lo] operand blocks, laid out as in shared memory
+    const unsigned char *ctiles;  // screening kernel: candidate operand blocks (topk_pack_candidates_kernel)
     float *part_cos;              // [splits][m][K]
     long long *part_ids;
     int *error;                   // device word: set to 1 if a wait ran out
@@ -371,44 +372,85 @@ topk_cosine_tc_kernel(TcParams p)
 }
 
 // =================================================================================================
-// Screening variant.  One TF32 MMA per product instead of three: the accumulator then holds the dot
-// product to about 1e-3 of |a||b| only (the query side is rounded to TF32 by a pre-pass, the
-// candidate side is read by the tensor core as it lies in memory, i.e. truncated: relative errors
-// of at most 2^-11 and 2^-10 per factor, so by Cauchy-Schwarz the cosine is off by less than
-// 2^-11 + 2^-10 + 2^-20 = 1.47e-3; the fp32 accumulation adds some 1e-5).  That is enough to
-// decide that a candidate cannot reach a query's current cut.  Only a candidate whose approximate
-// cosine comes within kScreenEps of the cut is looked at again: its warp computes the fp32 dot
-// product of the two rows from the table, and that exact cosine goes to the sorted list.  With a
-// list of K the number of such candidates is about K ln(n / K) per query, against n screened.
+// Screening variant.  One low-precision MMA per product instead of three TF32 ones: both sides are
+// rounded to bf16 (relative error at most 2^-9 per value), so each product is off by at most
+// (2^-8 + 2^-18) |a_i b_i| and, by Cauchy-Schwarz, the cosine by less than 3.92e-3; the fp32
+// accumulation adds some 1e-5.  That is enough to decide that a candidate cannot reach a query's
+// current cut.  Only a candidate whose approximate cosine comes within kScreenEps of the cut is
+// looked at again: its warp computes the fp32 dot product of the two rows from the table, and that
+// exact cosine goes to the sorted list.  With a list of K the number of such candidates is about
+// K ln(n / K) per query, against n screened.
 //
-// The query block stays in shared memory for the whole kernel (d <= 320: 160 KB), so only candidate
-// rows stream: 128 query rows x 256 candidates per tile, two 32-column stages of candidates.
-constexpr float kScreenEps = 2e-3f;
-constexpr int kScMaxKB = 10;                                     // K-blocks of 32 columns that fit: d <= 320
-constexpr int kScAChunk = kTcM * 16;                             // query operand: no padding (filled by bulk copies)
-constexpr int kScABlock = 8 * kScAChunk;                         // bytes of one K-block of the query operand
-constexpr int kScStageBytes = kTcOperandC;                       // one stage = one candidate operand block
-constexpr int kScGroups = 3;                                     // loader groups: 96 KB of candidate rows in flight in registers
-constexpr int kScThreads = 5 * 32 + kScGroups * kTcLoaders;
+// Both sides are converted by pre-passes into global scratch that has exactly the layout of the
+// shared-memory operands ([K-block][16-byte chunk][row][8 bf16]), so the main kernel moves them
+// with bulk copies only and has no loader warps.  The query block stays in shared memory for the
+// whole kernel (d <= 320: 80 KB); candidates stream through eight 16 KB stages (one K-block of 32
+// columns of a 256-candidate tile: two MMAs of K = 16), each filled by one `cp.async.bulk` that a
+// single producer lane issues as soon as the stage's previous MMAs have committed.  The bf16 copy
+// halves what every query block pulls through L2, which is what bounds this kernel.
+constexpr float kScreenEps = 4.5e-3f;
+constexpr int kScKB = 32;                                        // columns per stage
+constexpr int kScCh = kScKB / 8;                                 // 16-byte chunks (8 bf16) per row and stage
+constexpr int kScMaxKB = 10;                                     // stages per row that fit: d <= 320
+constexpr int kScStages = 8;
+constexpr int kScAChunk = kTcM * 16;                             // query operand, one 16-byte chunk of all rows
+constexpr int kScABlock = kScCh * kScAChunk;                     // bytes of one K-block of the query operand
+constexpr int kScBChunk = kTcN * 16;                             // candidate operand
+constexpr int kScStageBytes = kScCh * kScBChunk;                 // one stage = one K-block of one candidate tile = one bulk copy
+constexpr int kScThreads = 6 * 32;                               // 4 epilogue warps, the MMA warp, the producer warp
 
-// Query rows of one block, rounded to TF32, in the layout of the shared-memory operand
-// ([K-block][16-byte chunk][row][16 B]).  One block per (query block, K-block).
+// two floats -> two bf16 (round to nearest even), first in the low half
+__device__ __forceinline__ uint32_t bf16x2(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// Query rows of one block as bf16 in the layout of the shared-memory operand
+// ([K-block][16-byte chunk][row][8 bf16]).  One block per (query block, K-block).
 __global__ void __launch_bounds__(256)
 topk_round_queries_kernel(const float *__restrict__ table, const long long *__restrict__ queries, uint64_t m,
-                          uint64_t vocab, uint32_t d4, uint32_t ld4, uint32_t nkb, unsigned char *__restrict__ qtf32)
+                          uint64_t vocab, uint32_t d4, uint32_t ld4, uint32_t nkb, unsigned char *__restrict__ qb16)
 {
     const uint32_t qb = blockIdx.x / nkb, kb = blockIdx.x % nkb;
-    unsigned char *dst = qtf32 + ((size_t)qb * nkb + kb) * kScABlock;
+    unsigned char *dst = qb16 + ((size_t)qb * nkb + kb) * kScABlock;
     const float4 *T4 = reinterpret_cast<const float4 *>(table);
-    for (uint32_t e = threadIdx.x; e < (uint32_t)kTcM * 8; e += blockDim.x) {
-        const uint32_t r = e >> 3, ch = e & 7;
+    for (uint32_t e = threadIdx.x; e < (uint32_t)(kTcM * kScCh); e += blockDim.x) {
+        const uint32_t r = e / kScCh, ch = e % kScCh;
         const uint64_t qi = (uint64_t)qb * kTcM + r;
         long long row = qi < m ? queries[qi] : -1;
         if (row < 0 || (unsigned long long)row >= vocab) row = -1;
-        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (row >= 0 && kb * 8 + ch < d4) x = __ldcg(T4 + (size_t)row * ld4 + (kb * 8 + ch));
-        *reinterpret_cast<float4 *>(dst + ch * kScAChunk + r * 16) =
-            make_float4(tf32_round(x.x), tf32_round(x.y), tf32_round(x.z), tf32_round(x.w));
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f), y = x;
+        const uint32_t c4 = kb * (kScKB / 4) + 2 * ch;                      // first of the two float4 of this chunk
+        if (row >= 0 && c4 < d4) x = __ldcg(T4 + (size_t)row * ld4 + c4);
+        if (row >= 0 && c4 + 1 < d4) y = __ldcg(T4 + (size_t)row * ld4 + c4 + 1);
+        *reinterpret_cast<uint4 *>(dst + ch * kScAChunk + r * 16) =
+            make_uint4(bf16x2(x.x, x.y), bf16x2(x.z, x.w), bf16x2(y.x, y.y), bf16x2(y.z, y.w));
+    }
+}
+
+// Candidate rows cand_lo + [0, nc), scaled to unit length (inv_norm[c] = 1/|row|), as bf16 operand blocks: [tile of 256 rows][K-block][chunk][row][8 bf16],
+// zeros past the end of the range and of the row.  One thread per (row, chunk).
+__global__ void __launch_bounds__(256)
+topk_pack_candidates_kernel(const float *__restrict__ table, const float *__restrict__ inv_norm, uint32_t d4, uint32_t ld4,
+                            uint64_t cand_lo, uint64_t nc, uint32_t nkb, unsigned char *__restrict__ out)
+{
+    const uint64_t tiles = (nc + kTcN - 1) / kTcN;
+    const uint64_t total = tiles * kTcN * (uint64_t)(nkb * kScCh);
+    const float4 *T4 = reinterpret_cast<const float4 *>(table);
+    for (uint64_t e = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (uint64_t)gridDim.x * blockDim.x) {
+        const uint32_t chr = (uint32_t)(e % (nkb * kScCh));          // chunk of the row: 8 columns
+        const uint64_t c = e / (nkb * kScCh);                        // candidate (padded to whole tiles)
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f), y = x;
+        if (c < nc && 2 * chr < d4) x = __ldcg(T4 + (size_t)(cand_lo + c) * ld4 + 2 * chr);
+        if (c < nc && 2 * chr + 1 < d4) y = __ldcg(T4 + (size_t)(cand_lo + c) * ld4 + 2 * chr + 1);
+        const float ic = c < nc ? __ldg(inv_norm + c) : 0.f;         // unit rows: an accumulator column times 1/|query| is a cosine
+        x.x *= ic; x.y *= ic; x.z *= ic; x.w *= ic; y.x *= ic; y.y *= ic; y.z *= ic; y.w *= ic;
+        const uint64_t tile = c / kTcN;
+        const uint32_t r = (uint32_t)(c % kTcN), kb = chr / kScCh, ch = chr % kScCh;
+        *reinterpret_cast<uint4 *>(out + ((tile * nkb + kb) * kScCh + ch) * (size_t)kScBChunk + r * 16) =
+            make_uint4(bf16x2(x.x, x.y), bf16x2(x.z, x.w), bf16x2(y.x, y.y), bf16x2(y.z, y.w));
     }
 }
 
@@ -426,32 +468,53 @@ __device__ __forceinline__ float warp_row_dot(const float4 *__restrict__ T4, siz
     return s;
 }
 
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}\n"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0), "r"(0), "r"(0), "r"(0) : "memory");
+}
+
+// 32 consecutive fp32 columns of this thread's accumulator row (lane of tensor memory); asynchronous
+// until tcgen05.wait::ld
+__device__ __forceinline__ void tmem_ld32(uint32_t (&v)[32], uint32_t taddr)
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                   "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                   "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                 : "r"(taddr));
+}
+
 __global__ void __launch_bounds__(kScThreads, 1)
 topk_cosine_screen_kernel(TcParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char *a_op = smem;                                              // [kScMaxKB] query K-blocks
-    unsigned char *b_op = smem + kScMaxKB * kScABlock;                       // [kTcStages] candidate stages
-    uint64_t *full = reinterpret_cast<uint64_t *>(b_op + kTcStages * kScStageBytes);
-    uint64_t *empty = full + kTcStages;
-    uint64_t *tfull = empty + kTcStages;
+    unsigned char *b_op = smem + kScMaxKB * kScABlock;                       // [kScStages] candidate stages
+    uint64_t *full = reinterpret_cast<uint64_t *>(b_op + kScStages * kScStageBytes);
+    uint64_t *empty = full + kScStages;
+    uint64_t *tfull = empty + kScStages;
     uint64_t *tempty = tfull + 2;
     uint64_t *afull = tempty + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(afull + 1);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
-    volatile uint32_t *consumed = reinterpret_cast<volatile uint32_t *>(tmem_slot + 2);   // [kTcStages] uses of a stage the MMAs are done with
-    long long *qrow = reinterpret_cast<long long *>(tmem_slot + 4);          // [128]
+    long long *qrow = reinterpret_cast<long long *>(tmem_slot + 2);          // [128]
 
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint64_t q0 = (uint64_t)blockIdx.x * kTcM;
     const uint64_t nc = p.cand_hi - p.cand_lo;
     const uint64_t tiles = (nc + kTcN - 1) / kTcN;
     const uint64_t t_lo = tiles * blockIdx.y / p.splits, t_hi = tiles * (blockIdx.y + 1) / p.splits;
-    const uint32_t nkb = (4u * p.d4 + kTcKB - 1) / kTcKB;
+    const uint32_t nkb = (4u * p.d4 + kScKB - 1) / kScKB;
     const uint64_t n_tiles = t_hi - t_lo;
 
     if (tid == 0) {
-        for (int s = 0; s < kTcStages; ++s) { mbar_init(full + s, kTcLoaders); mbar_init(empty + s, 1); consumed[s] = 0u; }
+        for (int s = 0; s < kScStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(tfull + b, 1); mbar_init(tempty + b, kTcM); }
         mbar_init(afull, 1);
         *abort_flag = 0;
@@ -493,77 +556,81 @@ topk_cosine_screen_kernel(TcParams p)
         const bool mine = my_q >= 0 && live;
         uint32_t have = 0;
         float thr = p.tau;
+        // one chunk of 32 columns of the current tile (first candidate c0 + cc)
+        uint64_t c0 = 0;
+        auto screen_chunk = [&](const uint32_t (&v)[32], uint32_t cc) {
+            __syncwarp();
+            const float cut = (have < p.K ? p.tau : fmaxf(p.tau, thr)) - kScreenEps;
+            float top = __uint_as_float(v[0]);
+#pragma unroll
+            for (int j = 1; j < 32; ++j) top = fmaxf(top, __uint_as_float(v[j]));
+            uint32_t maybe = 0u;
+            if (mine && c0 + cc < nc && top * qinv >= cut) {              // rare: which of them?
+#pragma unroll
+                for (int j = 0; j < 32; ++j) maybe |= (__uint_as_float(v[j]) * qinv >= cut ? 1u : 0u) << j;
+                const uint64_t left = nc - (c0 + cc);                      // candidates of the range from column cc on
+                if (left < 32) maybe &= (1u << (uint32_t)left) - 1u;
+            }
+            // exact pass, one (query, candidate) at a time, the whole warp on one dot product
+            for (;;) {
+                const uint32_t owners = __ballot_sync(kFullMask, maybe != 0u);
+                if (!owners) break;
+                const uint32_t src = (uint32_t)__ffs((int)owners) - 1u;
+                const uint32_t j = __shfl_sync(kFullMask, (uint32_t)__ffs((int)maybe) - 1u, src);
+                const long long qr = qrow[warp * 32u + src];
+                const uint64_t c = c0 + cc + j;
+                const long long cid = (long long)(p.cand_lo + c);
+                const uint32_t hv = __shfl_sync(kFullMask, have, src);
+                const float th = __shfl_sync(kFullMask, thr, src);
+                if (lane == src) maybe &= maybe - 1u;
+                // query src's sorted list, lane l holding entries l and l + 32 (read while the rows are fetched)
+                float *wl = p.part_cos + ((size_t)blockIdx.y * p.m + (q0 + warp * 32u + src)) * p.K;
+                long long *wi = p.part_ids + ((size_t)blockIdx.y * p.m + (q0 + warp * 32u + src)) * p.K;
+                float e0 = 0.f, e1 = 0.f;
+                long long i0 = -1, i1 = -1;
+                if (lane < hv) { e0 = __ldcg(wl + lane); i0 = __ldcg(wi + lane); }
+                if (lane + 32u < hv) { e1 = __ldcg(wl + lane + 32u); i1 = __ldcg(wi + lane + 32u); }
+                const float dot = warp_row_dot(T4, (size_t)qr, (size_t)(p.cand_lo + c), p.d4, p.ld4, lane);
+                const float cs = dot * __shfl_sync(kFullMask, qinv, src) * __ldg(p.inv_norm + c);
+                if (!(cs > p.tau) || cid == qr || (hv == p.K && cs < th)) continue;     // same for every lane
+                const bool a0 = lane < hv && !ranks_ahead_tc(cs, cid, e0, i0);         // entries that stay ahead: a prefix
+                const bool a1 = lane + 32u < hv && !ranks_ahead_tc(cs, cid, e1, i1);
+                const uint32_t pos = (uint32_t)__popc(__ballot_sync(kFullMask, a0)) + (uint32_t)__popc(__ballot_sync(kFullMask, a1));
+                const uint32_t km2 = p.K >= 2u ? p.K - 2u : 0u;
+                const float e_km2 = km2 < 32u ? __shfl_sync(kFullMask, e0, km2) : __shfl_sync(kFullMask, e1, km2 - 32u);
+                if (pos < p.K) {
+                    if (lane < hv && !a0 && lane + 1u < p.K) { wl[lane + 1u] = e0; wi[lane + 1u] = i0; }
+                    if (lane + 32u < hv && !a1 && lane + 33u < p.K) { wl[lane + 33u] = e1; wi[lane + 33u] = i1; }
+                    if (lane == 0) { wl[pos] = cs; wi[pos] = cid; }
+                    if (lane == src) {
+                        have = hv < p.K ? hv + 1u : p.K;
+                        thr = have == p.K ? (pos == p.K - 1u ? cs : e_km2) : p.tau;
+                    }
+                }
+                __syncwarp();
+            }
+        };
         for (uint64_t i = 0; i < n_tiles; ++i) {
             const uint32_t b = (uint32_t)(i & 1);
-            const uint64_t c0 = (t_lo + i) * kTcN;
+            c0 = (t_lo + i) * kTcN;
             // the tensor-memory loads below are warp-wide: the whole warp goes on or gives up together
             if (!__all_sync(kFullMask, mbar_wait(tfull + b, (uint32_t)((i >> 1) & 1), abort_flag))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            // Two chunks of 32 accumulator columns are in flight: the load of chunk k + 1 is issued before
+            // chunk k is looked at.  The candidate rows were packed as unit vectors, so a column times
+            // 1/|query| is the screened cosine; the largest of the 32 decides whether the chunk needs a
+            // closer look at all.
+            uint32_t va[32], vb[32];
+            tmem_ld32(va, tmem_base + ((warp * 32u) << 16) + b * kTcN);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll 1
-            for (uint32_t cc = 0; cc < (uint32_t)kTcN; cc += 32) {
-                uint32_t v[32];
-                __syncwarp();
-                // lane l: 1/|x| of candidate cc + l of the tile (0 past the end of the range)
-                const float icv = c0 + cc + lane < nc ? __ldg(p.inv_norm + c0 + cc + lane) : 0.f;
-                const uint32_t ta = tmem_base + ((warp * 32u) << 16) + b * kTcN + cc;
-                asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                             "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                             "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                             : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                               "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-                               "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-                               "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                             : "r"(ta));
+            for (uint32_t cc = 0; cc < (uint32_t)kTcN; cc += 64) {
+                tmem_ld32(vb, tmem_base + ((warp * 32u) << 16) + b * kTcN + cc + 32u);
+                screen_chunk(va, cc);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                // screen: bit j = candidate cc + j may reach this query's cut
-                const float cut = (have < p.K ? p.tau : fmaxf(p.tau, thr)) - kScreenEps;
-                uint32_t maybe = 0u;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const float ic = __shfl_sync(kFullMask, icv, j);
-                    maybe |= (__uint_as_float(v[j]) * qinv * ic >= cut ? 1u : 0u) << j;
-                }
-                const uint64_t left = nc - (c0 + cc);                  // candidates of the range from column cc on
-                if (!mine || c0 + cc >= nc) maybe = 0u;
-                else if (left < 32) maybe &= (1u << (uint32_t)left) - 1u;
-                // exact pass, one (query, candidate) at a time, the whole warp on one dot product
-                for (;;) {
-                    const uint32_t owners = __ballot_sync(kFullMask, maybe != 0u);
-                    if (!owners) break;
-                    const uint32_t src = (uint32_t)__ffs((int)owners) - 1u;
-                    const uint32_t j = __shfl_sync(kFullMask, (uint32_t)__ffs((int)maybe) - 1u, src);
-                    const long long qr = qrow[warp * 32u + src];
-                    const uint64_t c = c0 + cc + j;
-                    const long long cid = (long long)(p.cand_lo + c);
-                    const uint32_t hv = __shfl_sync(kFullMask, have, src);
-                    const float th = __shfl_sync(kFullMask, thr, src);
-                    if (lane == src) maybe &= maybe - 1u;
-                    // query src's sorted list, lane l holding entries l and l + 32 (read while the rows are fetched)
-                    float *wl = p.part_cos + ((size_t)blockIdx.y * p.m + (q0 + warp * 32u + src)) * p.K;
-                    long long *wi = p.part_ids + ((size_t)blockIdx.y * p.m + (q0 + warp * 32u + src)) * p.K;
-                    float e0 = 0.f, e1 = 0.f;
-                    long long i0 = -1, i1 = -1;
-                    if (lane < hv) { e0 = __ldcg(wl + lane); i0 = __ldcg(wi + lane); }
-                    if (lane + 32u < hv) { e1 = __ldcg(wl + lane + 32u); i1 = __ldcg(wi + lane + 32u); }
-                    const float dot = warp_row_dot(T4, (size_t)qr, (size_t)(p.cand_lo + c), p.d4, p.ld4, lane);
-                    const float cs = dot * __shfl_sync(kFullMask, qinv, src) * __shfl_sync(kFullMask, icv, j);
-                    if (!(cs > p.tau) || cid == qr || (hv == p.K && cs < th)) continue;     // same for every lane
-                    const bool a0 = lane < hv && !ranks_ahead_tc(cs, cid, e0, i0);         // entries that stay ahead: a prefix
-                    const bool a1 = lane + 32u < hv && !ranks_ahead_tc(cs, cid, e1, i1);
-                    const uint32_t pos = (uint32_t)__popc(__ballot_sync(kFullMask, a0)) + (uint32_t)__popc(__ballot_sync(kFullMask, a1));
-                    const uint32_t km2 = p.K >= 2u ? p.K - 2u : 0u;
-                    const float e_km2 = km2 < 32u ? __shfl_sync(kFullMask, e0, km2) : __shfl_sync(kFullMask, e1, km2 - 32u);
-                    if (pos < p.K) {
-                        if (lane < hv && !a0 && lane + 1u < p.K) { wl[lane + 1u] = e0; wi[lane + 1u] = i0; }
-                        if (lane + 32u < hv && !a1 && lane + 33u < p.K) { wl[lane + 33u] = e1; wi[lane + 33u] = i1; }
-                        if (lane == 0) { wl[pos] = cs; wi[pos] = cid; }
-                        if (lane == src) {
-                            have = hv < p.K ? hv + 1u : p.K;
-                            thr = have == p.K ? (pos == p.K - 1u ? cs : e_km2) : p.tau;
-                        }
-                    }
-                    __syncwarp();
-                }
+                if (cc + 64u < (uint32_t)kTcN) tmem_ld32(va, tmem_base + ((warp * 32u) << 16) + b * kTcN + cc + 64u);
+                screen_chunk(vb, cc + 32u);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             mbar_arrive(tempty + b);                              // this accumulator buffer may be overwritten
@@ -571,7 +638,8 @@ topk_cosine_screen_kernel(TcParams p)
     } else if (warp == 4) {
         // ================= MMA issue: one lane =================
         if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTcN >> 3) << 17) | ((uint32_t)(kTcM >> 4) << 24);
+            // bf16 x bf16 -> fp32, both operands K-major, N = 256, M = 128
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcN >> 3) << 17) | ((uint32_t)(kTcM >> 4) << 24);
             // the query block: one bulk copy per K-block, all on one barrier
             asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
                          ::"r"(smem_addr(afull)), "r"(nkb * (uint32_t)kScABlock) : "memory");
@@ -586,65 +654,45 @@ topk_cosine_screen_kernel(TcParams p)
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t dst = tmem_base + b * kTcN;
                 for (uint32_t kb = 0; kb < nkb && ok; ++kb, ++g) {
-                    const uint32_t s = (uint32_t)(g % kTcStages);
-                    ok = mbar_wait(full + s, (uint32_t)((g / kTcStages) & 1), abort_flag);
+                    const uint32_t s = (uint32_t)(g % kScStages);
+                    ok = mbar_wait(full + s, (uint32_t)((g / kScStages) & 1), abort_flag);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t abase = smem_addr(a_op + (size_t)kb * kScABlock);
                     const uint32_t bbase = smem_addr(b_op + (size_t)s * kScStageBytes);
-                    const uint32_t chunks = p.d4 - kb * 8u < 8u ? p.d4 - kb * 8u : 8u;   // 16-byte chunks with data
-                    const uint32_t nk = (chunks + 1u) / 2u;                              // MMAs of K = 8 columns
+                    const uint32_t cols = 4u * p.d4 - kb * kScKB < (uint32_t)kScKB ? 4u * p.d4 - kb * kScKB : (uint32_t)kScKB;
+                    const uint32_t nk = (cols + 15u) / 16u;                              // MMAs of K = 16 columns with data
                     for (uint32_t kk = 0; kk < nk; ++kk) {
                         const uint64_t qa = umma_desc(abase + 2 * kk * kScAChunk, kScAChunk, 128);
-                        const uint64_t cb = umma_desc(bbase + 2 * kk * kTcChunkStrideC, kTcChunkStrideC, 128);
-                        umma_tf32(dst, qa, cb, idesc, (kb | kk) ? 1u : 0u);
+                        const uint64_t cb = umma_desc(bbase + 2 * kk * kScBChunk, kScBChunk, 128);
+                        umma_bf16(dst, qa, cb, idesc, (kb | kk) ? 1u : 0u);
                     }
                     umma_commit(empty + s);                       // the stage is free once these MMAs have read it
                 }
                 if (ok) umma_commit(tfull + b);                   // the tile's accumulator is complete
             }
-        } else if (lane == 1) {
-            // Relay.  More loader groups than stages take turns on a stage, and a parity wait cannot
-            // tell "free again" from "free two uses ago"; this lane waits for every release in order
-            // and publishes the count, which the loaders poll.
-            const uint64_t total_g = n_tiles * nkb;
-            for (uint64_t g = 0; g < total_g; ++g) {
-                const uint32_t s = (uint32_t)(g % kTcStages);
-                const uint64_t use = g / kTcStages;
-                if (!mbar_wait(empty + s, (uint32_t)(use & 1), abort_flag)) break;
-                __threadfence_block();
-                consumed[s] = (uint32_t)(use + 1);
-            }
         }
     } else {
-        // ================= loaders: candidate rows as they are =================
-        const uint32_t group = (tid - 5 * 32) / kTcLoaders, ltid = (tid - 5 * 32) % kTcLoaders;
-        const uint64_t total_g = n_tiles * nkb;
-        float4 x[kTcPer];
-        uint64_t g = group;
-        if (g < total_g) candidates_issue(p, x, (uint32_t)(g % nkb) * kTcKB, ltid, (t_lo + g / nkb) * kTcN, nc);
-        while (g < total_g) {
-            const uint32_t s = (uint32_t)(g % kTcStages);
-            {   // the stage's previous use must have been read by the MMAs
-                const uint32_t need = (uint32_t)(g / kTcStages);
-                bool ok = false;
-                for (uint32_t spin = 0; spin < kTcSpinLimit * 16u; ++spin) {
-                    if (consumed[s] >= need) { ok = true; break; }
-                    if ((spin & 1023u) == 1023u && *abort_flag) break;
-                }
-                if (!ok) { *abort_flag = 1; break; }
-                __threadfence_block();
+        // ================= producer: one lane =================
+        // one bulk copy per stage, issued when the MMAs that read the stage's previous contents have
+        // committed; its bytes complete the stage's "full" barrier
+        if (lane == 0) {
+            const uint64_t total_g = n_tiles * nkb;
+            uint64_t g = 0;
+            for (; g < total_g; ++g) {
+                const uint32_t s = (uint32_t)(g % kScStages);
+                if (!mbar_wait(empty + s, (uint32_t)(((g / kScStages) & 1) ^ 1), abort_flag)) break;
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                             ::"r"(smem_addr(full + s)), "r"((uint32_t)kScStageBytes) : "memory");
+                bulk_to_smem(b_op + (size_t)s * kScStageBytes,
+                             p.ctiles + ((t_lo + g / nkb) * nkb + g % nkb) * (size_t)kScStageBytes, (uint32_t)kScStageBytes, full + s);
             }
-            unsigned char *st = b_op + (size_t)s * kScStageBytes;
-#pragma unroll
-            for (int it = 0; it < kTcPer; ++it) {
-                const uint32_t e = ltid + it * kTcLoaders;
-                *reinterpret_cast<float4 *>(st + (e & 7) * kTcChunkStrideC + (e >> 3) * 16) = x[it];
+            if (*abort_flag) {
+                // the block is giving up: let the copies still in flight land before shared memory is released
+                for (uint64_t j = g > (uint64_t)kScStages ? g - kScStages : 0; j < g; ++j)
+                    for (uint32_t spin = 0; spin < kTcSpinLimit; ++spin)
+                        if (mbar_try(full + j % kScStages, (uint32_t)((j / kScStages) & 1))) break;
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");         // stores -> tensor-core reads
-            mbar_arrive(full + s);
-            g += kScGroups;
-            if (g < total_g) candidates_issue(p, x, (uint32_t)(g % nkb) * kTcKB, ltid, (t_lo + g / nkb) * kTcN, nc);
         }
     }
     // ================= common exit =================
@@ -659,54 +707,83 @@ topk_cosine_screen_kernel(TcParams p)
 
 static size_t topk_screen_smem_bytes()
 {
-    return (size_t)kScMaxKB * kScABlock + (size_t)kTcStages * kScStageBytes + (2 * kTcStages + 5) * 8 + 16 + kTcM * 8 + 128;
+    return (size_t)kScMaxKB * kScABlock + (size_t)kScStages * kScStageBytes + (2 * kScStages + 5) * 8 + 8 + kTcM * 8 + 128;
 }
 
-bool topk_screen_fits(uint32_t d) { return (d + kTcKB - 1) / kTcKB <= (uint32_t)kScMaxKB; }
+bool topk_screen_fits(uint32_t d) { return (d + kScKB - 1) / kScKB <= (uint32_t)kScMaxKB; }
 
 size_t topk_tc_smem_bytes()
 {
     return (size_t)kTcStages * kTcStageBytes + (2 * kTcStages + 4) * 8 + 16 + kTcM * 8 + 8 * kTcN * 4 + 128;
 }
 
-// Returns the launches made, or -1 on a launch error.  Results go to part_* ([splits][m][K]); the caller merges.
 size_t topk_tc_qsplit_bytes(uint64_t m, uint32_t d)
 {
     const uint64_t qblocks = (m + kTcM - 1) / kTcM, nkb = (d + kTcKB - 1) / kTcKB;
     return (size_t)(qblocks * nkb * 2 * kTcOperand);          // the screening layout needs less (kScABlock per K-block)
 }
 
+// Screening kernel: candidates are handled in chunks of at most kScChunk rows (the packed bf16 copy of
+// one chunk is the scratch `ctiles`); every chunk has its own `splits` partial lists.
+constexpr uint64_t kScChunk = 1ull << 22;
+
+uint64_t topk_screen_chunk(uint64_t nc) { return nc < kScChunk ? nc : kScChunk; }
+
+size_t topk_screen_ctiles_bytes(uint64_t nc, uint32_t d)
+{
+    const uint64_t chunk = topk_screen_chunk(nc), tiles = (chunk + kTcN - 1) / kTcN, nkb = (d + kScKB - 1) / kScKB;
+    return (size_t)(tiles * nkb * kScStageBytes);
+}
+
+// Returns the launches made, or -1 on a launch error.  Results go to part_* ([lists][m][K], lists = splits, or
+// chunks x splits for the screening kernel); the caller merges.
 int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, const long long *queries, uint64_t m,
                    uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, const float *inv_norm,
-                   unsigned char *qsplit, float *part_cos, long long *part_ids, uint32_t splits, int *error,
-                   bool screen, cudaStream_t s)
+                   unsigned char *qsplit, unsigned char *ctiles, float *part_cos, long long *part_ids, uint32_t splits,
+                   int *error, bool screen, int sms, cudaStream_t s)
 {
     if (m == 0) return 0;
-    const uint32_t nkb = (d + kTcKB - 1) / kTcKB;
     const unsigned qblocks = (unsigned)((m + kTcM - 1) / kTcM);
     screen = screen && topk_screen_fits(d);
-    if (screen) topk_round_queries_kernel<<<qblocks * nkb, 256, 0, s>>>(table, queries, m, vocab, d / 4, ld / 4, nkb, qsplit);
-    else topk_split_queries_kernel<<<qblocks * nkb, 256, 0, s>>>(table, queries, m, vocab, d / 4, ld / 4, nkb, qsplit);
-    if (cudaGetLastError() != cudaSuccess) return -1;
     TcParams p;
-    p.qsplit = qsplit;
+    p.qsplit = qsplit; p.ctiles = ctiles;
     p.table = table; p.queries = queries; p.inv_norm = inv_norm; p.part_cos = part_cos; p.part_ids = part_ids;
     p.error = error; p.m = m; p.vocab = vocab; p.cand_lo = cand_lo; p.cand_hi = cand_hi;
     p.d4 = d / 4; p.ld4 = ld / 4; p.K = K; p.splits = splits; p.tau = tau;
-    dim3 grid((unsigned)((m + kTcM - 1) / kTcM), splits);
-    if (screen) {
-        const size_t sm = topk_screen_smem_bytes();
-        if (cudaFuncSetAttribute(topk_cosine_screen_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess)
-            return -1;
-        topk_cosine_screen_kernel<<<grid, kScThreads, sm, s>>>(p);
-    } else {
+    dim3 grid(qblocks, splits);
+    if (!screen) {
+        const uint32_t nkb = (d + kTcKB - 1) / kTcKB;
+        topk_split_queries_kernel<<<qblocks * nkb, 256, 0, s>>>(table, queries, m, vocab, d / 4, ld / 4, nkb, qsplit);
+        if (cudaGetLastError() != cudaSuccess) return -1;
         const size_t sm = topk_tc_smem_bytes();
         if (cudaFuncSetAttribute(topk_cosine_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess)
             return -1;
         topk_cosine_tc_kernel<<<grid, kTcThreads, sm, s>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return -1;
+        return 2;
     }
+    const uint32_t nkb = (d + kScKB - 1) / kScKB;
+    topk_round_queries_kernel<<<qblocks * nkb, 256, 0, s>>>(table, queries, m, vocab, d / 4, ld / 4, nkb, qsplit);
     if (cudaGetLastError() != cudaSuccess) return -1;
-    return 2;
+    const size_t sm = topk_screen_smem_bytes();
+    if (cudaFuncSetAttribute(topk_cosine_screen_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess)
+        return -1;
+    int launched = 1;
+    const uint64_t nc = cand_hi - cand_lo, chunk = topk_screen_chunk(nc);
+    uint64_t list = 0;
+    for (uint64_t c0 = 0; c0 < nc; c0 += chunk, ++list) {
+        const uint64_t n = nc - c0 < chunk ? nc - c0 : chunk;
+        topk_pack_candidates_kernel<<<sms * 8, 256, 0, s>>>(table, inv_norm + c0, d / 4, ld / 4, cand_lo + c0, n, nkb, ctiles);
+        if (cudaGetLastError() != cudaSuccess) return -1;
+        p.cand_lo = cand_lo + c0; p.cand_hi = cand_lo + c0 + n;
+        p.inv_norm = inv_norm + c0;
+        p.part_cos = part_cos + list * splits * m * K;
+        p.part_ids = part_ids + list * splits * m * K;
+        topk_cosine_screen_kernel<<<grid, kScThreads, sm, s>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return -1;
+        launched += 2;
+    }
+    return launched;
 }
 
 }  // namespace w2v

@@ -121,3 +121,14 @@ def test_topk_zero_rows_and_exact_ties(kernel):
     assert np.array_equal(gi, wi)                         # ties go to the smaller row number
     assert np.allclose(gc, wc, atol=tolerance(kernel, 8))
     gpu.close()
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_topk_candidate_range_longer_than_one_chunk(kernel):
+    # the screening kernel takes the candidates in chunks of 2^22 rows, each with its own partial lists
+    V, d = (1 << 22) + 70_001, 8
+    gpu, cpu, X = pair(V, d, seed=11, kernel=kernel)
+    q = np.array([0, 5, (1 << 22) - 1, 1 << 22, V - 1, 123_456])
+    check(gpu, cpu, X, 0, q, 0, V, 20, -2.0, tolerance(kernel, d))
+    check(gpu, cpu, X, 0, q, 3, V - 5, 7, 0.9, tolerance(kernel, d))
+    gpu.close()
