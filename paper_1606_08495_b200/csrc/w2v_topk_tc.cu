@@ -397,6 +397,7 @@ constexpr int kScAChunk = kTcM * 16;                             // query operan
 constexpr int kScABlock = kScCh * kScAChunk;                     // bytes of one K-block of the query operand
 constexpr int kScBChunk = kTcN * 16;                             // candidate operand
 constexpr int kScStageBytes = kScCh * kScBChunk;                 // one stage = one K-block of one candidate tile = one bulk copy
+constexpr int kExact = 4;                                        // (query, candidate) pairs whose exact cosines are computed together
 constexpr int kScThreads = 6 * 32;                               // 4 epilogue warps, the MMA warp, the producer warp
 
 // two floats -> two bf16 (round to nearest even), first in the low half
@@ -571,40 +572,75 @@ topk_cosine_screen_kernel(TcParams p)
                 const uint64_t left = nc - (c0 + cc);                      // candidates of the range from column cc on
                 if (left < 32) maybe &= (1u << (uint32_t)left) - 1u;
             }
-            // exact pass, one (query, candidate) at a time, the whole warp on one dot product
+            // Exact pass: the set bits of all lanes, up to kExact queries (lanes) at a time.  The whole warp
+            // works on each (query, candidate): 32 lanes on the fp32 dot product of the two table rows
+            // (the loads of all kExact pairs are issued before the first sum is reduced), then on the
+            // insertion into that query's sorted list, lane l holding entries l and l + 32.
             for (;;) {
-                const uint32_t owners = __ballot_sync(kFullMask, maybe != 0u);
+                uint32_t owners = __ballot_sync(kFullMask, maybe != 0u);
                 if (!owners) break;
-                const uint32_t src = (uint32_t)__ffs((int)owners) - 1u;
-                const uint32_t j = __shfl_sync(kFullMask, (uint32_t)__ffs((int)maybe) - 1u, src);
-                const long long qr = qrow[warp * 32u + src];
-                const uint64_t c = c0 + cc + j;
-                const long long cid = (long long)(p.cand_lo + c);
-                const uint32_t hv = __shfl_sync(kFullMask, have, src);
-                const float th = __shfl_sync(kFullMask, thr, src);
-                if (lane == src) maybe &= maybe - 1u;
-                // query src's sorted list, lane l holding entries l and l + 32 (read while the rows are fetched)
-                float *wl = p.part_cos + ((size_t)blockIdx.y * p.m + (q0 + warp * 32u + src)) * p.K;
-                long long *wi = p.part_ids + ((size_t)blockIdx.y * p.m + (q0 + warp * 32u + src)) * p.K;
-                float e0 = 0.f, e1 = 0.f;
-                long long i0 = -1, i1 = -1;
-                if (lane < hv) { e0 = __ldcg(wl + lane); i0 = __ldcg(wi + lane); }
-                if (lane + 32u < hv) { e1 = __ldcg(wl + lane + 32u); i1 = __ldcg(wi + lane + 32u); }
-                const float dot = warp_row_dot(T4, (size_t)qr, (size_t)(p.cand_lo + c), p.d4, p.ld4, lane);
-                const float cs = dot * __shfl_sync(kFullMask, qinv, src) * __ldg(p.inv_norm + c);
-                if (!(cs > p.tau) || cid == qr || (hv == p.K && cs < th)) continue;     // same for every lane
-                const bool a0 = lane < hv && !ranks_ahead_tc(cs, cid, e0, i0);         // entries that stay ahead: a prefix
-                const bool a1 = lane + 32u < hv && !ranks_ahead_tc(cs, cid, e1, i1);
-                const uint32_t pos = (uint32_t)__popc(__ballot_sync(kFullMask, a0)) + (uint32_t)__popc(__ballot_sync(kFullMask, a1));
-                const uint32_t km2 = p.K >= 2u ? p.K - 2u : 0u;
-                const float e_km2 = km2 < 32u ? __shfl_sync(kFullMask, e0, km2) : __shfl_sync(kFullMask, e1, km2 - 32u);
-                if (pos < p.K) {
-                    if (lane < hv && !a0 && lane + 1u < p.K) { wl[lane + 1u] = e0; wi[lane + 1u] = i0; }
-                    if (lane + 32u < hv && !a1 && lane + 33u < p.K) { wl[lane + 33u] = e1; wi[lane + 33u] = i1; }
-                    if (lane == 0) { wl[pos] = cs; wi[pos] = cid; }
-                    if (lane == src) {
-                        have = hv < p.K ? hv + 1u : p.K;
-                        thr = have == p.K ? (pos == p.K - 1u ? cs : e_km2) : p.tau;
+                bool on[kExact];
+                uint32_t src[kExact], hv[kExact];
+                float th[kExact], qi[kExact], dot[kExact], e0[kExact], e1[kExact];
+                long long i0[kExact], i1[kExact], qr[kExact];
+                uint64_t cnd[kExact];
+#pragma unroll
+                for (int e = 0; e < kExact; ++e) {
+                    on[e] = owners != 0u;
+                    src[e] = on[e] ? (uint32_t)__ffs((int)owners) - 1u : 0u;
+                    owners &= owners - 1u;
+                    const uint32_t j = __shfl_sync(kFullMask, (uint32_t)__ffs((int)maybe) - 1u, src[e]);
+                    cnd[e] = c0 + cc + j;
+                    qr[e] = qrow[warp * 32u + src[e]];
+                    hv[e] = __shfl_sync(kFullMask, have, src[e]);
+                    th[e] = __shfl_sync(kFullMask, thr, src[e]);
+                    qi[e] = __shfl_sync(kFullMask, qinv, src[e]);
+                    if (on[e] && lane == src[e]) maybe &= maybe - 1u;
+                    e0[e] = 0.f; e1[e] = 0.f; i0[e] = -1; i1[e] = -1; dot[e] = 0.f;
+                    if (on[e]) {
+                        const size_t lb = ((size_t)blockIdx.y * p.m + (q0 + warp * 32u + src[e])) * p.K;
+                        if (lane < hv[e]) { e0[e] = __ldcg(p.part_cos + lb + lane); i0[e] = __ldcg(p.part_ids + lb + lane); }
+                        if (lane + 32u < hv[e]) { e1[e] = __ldcg(p.part_cos + lb + lane + 32u); i1[e] = __ldcg(p.part_ids + lb + lane + 32u); }
+                    }
+                }
+                for (uint32_t idx = lane; idx < p.d4; idx += 32) {
+#pragma unroll
+                    for (int e = 0; e < kExact; ++e) {
+                        if (on[e]) {
+                            const float4 x = __ldcg(T4 + (size_t)qr[e] * p.ld4 + idx);
+                            const float4 y = __ldcg(T4 + (size_t)(p.cand_lo + cnd[e]) * p.ld4 + idx);
+                            dot[e] = fmaf(x.x, y.x, dot[e]); dot[e] = fmaf(x.y, y.y, dot[e]);
+                            dot[e] = fmaf(x.z, y.z, dot[e]); dot[e] = fmaf(x.w, y.w, dot[e]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                    for (int e = 0; e < kExact; ++e) dot[e] += __shfl_xor_sync(kFullMask, dot[e], o);
+                }
+#pragma unroll
+                for (int e = 0; e < kExact; ++e) {
+                    if (!on[e]) continue;                                                   // same for every lane
+                    const float cs = dot[e] * qi[e] * __ldg(p.inv_norm + cnd[e]);
+                    const long long cid = (long long)(p.cand_lo + cnd[e]);
+                    if (!(cs > p.tau) || cid == qr[e] || (hv[e] == p.K && cs < th[e])) continue;
+                    const size_t lb = ((size_t)blockIdx.y * p.m + (q0 + warp * 32u + src[e])) * p.K;
+                    float *wl = p.part_cos + lb;
+                    long long *wi = p.part_ids + lb;
+                    const bool a0 = lane < hv[e] && !ranks_ahead_tc(cs, cid, e0[e], i0[e]);         // entries that stay ahead: a prefix
+                    const bool a1 = lane + 32u < hv[e] && !ranks_ahead_tc(cs, cid, e1[e], i1[e]);
+                    const uint32_t pos = (uint32_t)__popc(__ballot_sync(kFullMask, a0)) + (uint32_t)__popc(__ballot_sync(kFullMask, a1));
+                    const uint32_t km2 = p.K >= 2u ? p.K - 2u : 0u;
+                    const float e_km2 = km2 < 32u ? __shfl_sync(kFullMask, e0[e], km2) : __shfl_sync(kFullMask, e1[e], km2 - 32u);
+                    if (pos < p.K) {
+                        if (lane < hv[e] && !a0 && lane + 1u < p.K) { wl[lane + 1u] = e0[e]; wi[lane + 1u] = i0[e]; }
+                        if (lane + 32u < hv[e] && !a1 && lane + 33u < p.K) { wl[lane + 33u] = e1[e]; wi[lane + 33u] = i1[e]; }
+                        if (lane == 0) { wl[pos] = cs; wi[pos] = cid; }
+                        if (lane == src[e]) {
+                            have = hv[e] < p.K ? hv[e] + 1u : p.K;
+                            thr = have == p.K ? (pos == p.K - 1u ? cs : e_km2) : p.tau;
+                        }
                     }
                 }
                 __syncwarp();
