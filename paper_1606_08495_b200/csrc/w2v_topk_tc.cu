@@ -431,27 +431,33 @@ topk_round_queries_kernel(const float *__restrict__ table, const long long *__re
     }
 }
 
-// Candidate rows cand_lo + [0, nc), scaled to unit length (inv_norm[c] = 1/|row|), as bf16 operand blocks: [tile of 256 rows][K-block][chunk][row][8 bf16],
-// zeros past the end of the range and of the row.  One thread per (row, chunk).
-__global__ void __launch_bounds__(256)
+// Candidate rows cand_lo + [0, nc), scaled to unit length (inv_norm[c] = 1/|row|), as bf16 operand blocks:
+// [tile of 256 rows][K-block][chunk][row][8 bf16], zeros past the end of the range and of the row.
+// One block per tile, one thread per row: a thread reads its row 128 bytes (one K-block) at a time
+// through L1, and the 256 threads' 16-byte stores of one chunk are contiguous.
+__global__ void __launch_bounds__(kTcN)
 topk_pack_candidates_kernel(const float *__restrict__ table, const float *__restrict__ inv_norm, uint32_t d4, uint32_t ld4,
                             uint64_t cand_lo, uint64_t nc, uint32_t nkb, unsigned char *__restrict__ out)
 {
     const uint64_t tiles = (nc + kTcN - 1) / kTcN;
-    const uint64_t total = tiles * kTcN * (uint64_t)(nkb * kScCh);
-    const float4 *T4 = reinterpret_cast<const float4 *>(table);
-    for (uint64_t e = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (uint64_t)gridDim.x * blockDim.x) {
-        const uint32_t chr = (uint32_t)(e % (nkb * kScCh));          // chunk of the row: 8 columns
-        const uint64_t c = e / (nkb * kScCh);                        // candidate (padded to whole tiles)
-        float4 x = make_float4(0.f, 0.f, 0.f, 0.f), y = x;
-        if (c < nc && 2 * chr < d4) x = __ldcg(T4 + (size_t)(cand_lo + c) * ld4 + 2 * chr);
-        if (c < nc && 2 * chr + 1 < d4) y = __ldcg(T4 + (size_t)(cand_lo + c) * ld4 + 2 * chr + 1);
-        const float ic = c < nc ? __ldg(inv_norm + c) : 0.f;         // unit rows: an accumulator column times 1/|query| is a cosine
-        x.x *= ic; x.y *= ic; x.z *= ic; x.w *= ic; y.x *= ic; y.y *= ic; y.z *= ic; y.w *= ic;
-        const uint64_t tile = c / kTcN;
-        const uint32_t r = (uint32_t)(c % kTcN), kb = chr / kScCh, ch = chr % kScCh;
-        *reinterpret_cast<uint4 *>(out + ((tile * nkb + kb) * kScCh + ch) * (size_t)kScBChunk + r * 16) =
-            make_uint4(bf16x2(x.x, x.y), bf16x2(x.z, x.w), bf16x2(y.x, y.y), bf16x2(y.z, y.w));
+    const uint32_t r = threadIdx.x;
+    for (uint64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+        const uint64_t c = tile * kTcN + r;
+        const bool valid = c < nc;
+        const float ic = valid ? __ldg(inv_norm + c) : 0.f;       // unit rows: an accumulator column times 1/|query| is a cosine
+        const float4 *row = reinterpret_cast<const float4 *>(table) + (size_t)(cand_lo + (valid ? c : 0)) * ld4;
+        for (uint32_t kb = 0; kb < nkb; ++kb) {
+            unsigned char *dst = out + (tile * nkb + kb) * (size_t)kScStageBytes + r * 16;
+#pragma unroll
+            for (int ch = 0; ch < kScCh; ++ch) {
+                const uint32_t c4 = kb * (kScKB / 4) + 2 * ch;
+                float4 x = make_float4(0.f, 0.f, 0.f, 0.f), y = x;
+                if (valid && c4 < d4) x = __ldg(row + c4);
+                if (valid && c4 + 1 < d4) y = __ldg(row + c4 + 1);
+                *reinterpret_cast<uint4 *>(dst + ch * kScBChunk) =
+                    make_uint4(bf16x2(x.x * ic, x.y * ic), bf16x2(x.z * ic, x.w * ic), bf16x2(y.x * ic, y.y * ic), bf16x2(y.z * ic, y.w * ic));
+            }
+        }
     }
 }
 
@@ -809,7 +815,7 @@ int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, 
     uint64_t list = 0;
     for (uint64_t c0 = 0; c0 < nc; c0 += chunk, ++list) {
         const uint64_t n = nc - c0 < chunk ? nc - c0 : chunk;
-        topk_pack_candidates_kernel<<<sms * 8, 256, 0, s>>>(table, inv_norm + c0, d / 4, ld / 4, cand_lo + c0, n, nkb, ctiles);
+        topk_pack_candidates_kernel<<<sms * 16, kTcN, 0, s>>>(table, inv_norm + c0, d / 4, ld / 4, cand_lo + c0, n, nkb, ctiles);
         if (cudaGetLastError() != cudaSuccess) return -1;
         p.cand_lo = cand_lo + c0; p.cand_hi = cand_lo + c0 + n;
         p.inv_norm = inv_norm + c0;
