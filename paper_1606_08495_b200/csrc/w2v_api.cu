@@ -775,7 +775,7 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
     const float *table = which ? h->V : h->U;
     int32_t rc;
     if ((rc = profile_mark(h)) != W2V_OK) return rc;
-    int k = launch_inv_norms(table, h->d, h->ld, cand_lo, nc, h->inv_norm, h->sms, h->stream);
+    int k = screen ? 0 : launch_inv_norms(table, h->d, h->ld, cand_lo, nc, h->inv_norm, h->sms, h->stream);
     if (k < 0) return fail(h, W2V_ERR_CUDA, "norm launch", cudaGetLastError());
     int k2;
     if (tc) {

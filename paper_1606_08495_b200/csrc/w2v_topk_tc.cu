@@ -431,12 +431,14 @@ topk_round_queries_kernel(const float *__restrict__ table, const long long *__re
     }
 }
 
-// Candidate rows cand_lo + [0, nc), scaled to unit length (inv_norm[c] = 1/|row|), as bf16 operand blocks:
-// [tile of 256 rows][K-block][chunk][row][8 bf16], zeros past the end of the range and of the row.
-// One block per tile, one thread per row: a thread reads its row 128 bytes (one K-block) at a time
-// through L1, and the 256 threads' 16-byte stores of one chunk are contiguous.
+// Candidate rows cand_lo + [0, nc), scaled to unit length, as bf16 operand blocks:
+// [tile of 256 rows][K-block][chunk][row][8 bf16], zeros past the end of the range and of the row;
+// inv_norm[c] = 1/|row c| (0 for a zero row) is written on the way, for the exact cosines.
+// One block per tile, one thread per row: a thread reads its row once for the norm and once more,
+// 128 bytes (one K-block) at a time through L1 and L2, for the operand; the 256 threads' 16-byte
+// stores of one chunk are contiguous.
 __global__ void __launch_bounds__(kTcN)
-topk_pack_candidates_kernel(const float *__restrict__ table, const float *__restrict__ inv_norm, uint32_t d4, uint32_t ld4,
+topk_pack_candidates_kernel(const float *__restrict__ table, float *__restrict__ inv_norm, uint32_t d4, uint32_t ld4,
                             uint64_t cand_lo, uint64_t nc, uint32_t nkb, unsigned char *__restrict__ out)
 {
     const uint64_t tiles = (nc + kTcN - 1) / kTcN;
@@ -444,8 +446,17 @@ topk_pack_candidates_kernel(const float *__restrict__ table, const float *__rest
     for (uint64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
         const uint64_t c = tile * kTcN + r;
         const bool valid = c < nc;
-        const float ic = valid ? __ldg(inv_norm + c) : 0.f;       // unit rows: an accumulator column times 1/|query| is a cosine
         const float4 *row = reinterpret_cast<const float4 *>(table) + (size_t)(cand_lo + (valid ? c : 0)) * ld4;
+        float ic = 0.f;                                            // unit rows: an accumulator column times 1/|query| is a cosine
+        if (valid) {
+            float q = 0.f;
+            for (uint32_t j = 0; j < d4; ++j) {
+                const float4 x = __ldg(row + j);
+                q = fmaf(x.x, x.x, q); q = fmaf(x.y, x.y, q); q = fmaf(x.z, x.z, q); q = fmaf(x.w, x.w, q);
+            }
+            ic = q > 0.f ? 1.0f / sqrtf(q) : 0.f;
+            inv_norm[c] = ic;
+        }
         for (uint32_t kb = 0; kb < nkb; ++kb) {
             unsigned char *dst = out + (tile * nkb + kb) * (size_t)kScStageBytes + r * 16;
 #pragma unroll
@@ -780,7 +791,7 @@ size_t topk_screen_ctiles_bytes(uint64_t nc, uint32_t d)
 // Returns the launches made, or -1 on a launch error.  Results go to part_* ([lists][m][K], lists = splits, or
 // chunks x splits for the screening kernel); the caller merges.
 int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, const long long *queries, uint64_t m,
-                   uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, const float *inv_norm,
+                   uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, float *inv_norm,
                    unsigned char *qsplit, unsigned char *ctiles, float *part_cos, long long *part_ids, uint32_t splits,
                    int *error, bool screen, int sms, cudaStream_t s)
 {
