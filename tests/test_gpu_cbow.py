@@ -82,6 +82,12 @@ def test_cbow_snapshot_steps_small_and_medium_shapes():
                                       minibatch=32_768), steps=2, words=8_000, row_stride=320)
 
 
+@pytest.mark.parametrize("N", [1, 13, 33, 64])
+def test_cbow_snapshot_other_negative_counts(N):
+    cfg = corpus.scaled(TINY, vocab=3000, d=100, negatives=N, minibatch=600, corpus_tokens=60_000)
+    check_cbow_snapshot(cfg, steps=2)
+
+
 @pytest.mark.parametrize("d", [4, 64, 132, 512, 1024])
 def test_cbow_snapshot_other_dimensions(d):
     check_cbow_snapshot(corpus.scaled(TINY, vocab=3000, d=d, minibatch=1500, corpus_tokens=100_000), steps=2)

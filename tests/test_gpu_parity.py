@@ -222,6 +222,13 @@ def test_snapshot_other_dimensions(d):
     check_snapshot_steps(cfg, steps=2)
 
 
+@pytest.mark.parametrize("N,W", [(1, 3), (13, 2), (33, 2), (64, 1)])
+def test_snapshot_other_negative_counts(N, W):
+    # more targets per pair than one batch of row touches (12), than one register of draws per lane (32)
+    cfg = corpus.scaled(TINY, vocab=3000, d=100, negatives=N, window=W, minibatch=400, corpus_tokens=60_000)
+    check_snapshot_steps(cfg, steps=2)
+
+
 @pytest.mark.parametrize("d,row_stride", [(300, 320), (300, 304), (100, 128), (8, 16), (132, 2048)])
 def test_snapshot_padded_rows(d, row_stride):
     # rows on 64-byte boundaries: same vectors, same step, only the addresses differ
