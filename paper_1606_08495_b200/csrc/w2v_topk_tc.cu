@@ -16,7 +16,7 @@
 //              (the query side is split once by a pre-pass and arrives by cp.async.bulk), K-major core-matrix layout without
 //              swizzle ([16-byte column chunk][row][16 B], chunk stride 2064 B: conflict-free stores).
 // Shared-memory stages and the two accumulator buffers are handed over with mbarriers; every wait
-// has an iteration limit, after which the block raises the error flag and leaves through the common
+// has a time limit, after which the block raises the error flag and leaves through the common
 // exit that frees the tensor memory.
 #include "w2v_device.cuh"
 #include "w2v_internal.h"
@@ -55,12 +55,25 @@ __device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity)
     return done != 0;
 }
 // Bounded wait.  Returns false (and raises the block's abort flag) when the limit is reached or
-// another thread has already given up.
+// another thread has already given up.  The limit is a time, not a count: how long a partner may
+// legitimately take depends on the data (an epilogue warp computes an exact cosine for every pair
+// that passes the screen, which for rows that are all alike is every pair).
+constexpr unsigned long long kTcWaitNs = 4000000000ull;           // 4 s
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
-    for (uint32_t spin = 0; spin < kTcSpinLimit; ++spin) {
+    const unsigned long long t0 = global_ns();
+    for (uint32_t spin = 0; spin < (1u << 30); ++spin) {
         if (mbar_try(bar, parity)) return true;
-        if ((spin & 1023u) == 1023u && *abort_flag) return false;
+        if ((spin & 1023u) == 1023u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > kTcWaitNs) break;
+        }
     }
     *abort_flag = 1;
     return false;

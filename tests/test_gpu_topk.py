@@ -132,3 +132,18 @@ def test_topk_candidate_range_longer_than_one_chunk(kernel):
     check(gpu, cpu, X, 0, q, 0, V, 20, -2.0, tolerance(kernel, d))
     check(gpu, cpu, X, 0, q, 3, V - 5, 7, 0.9, tolerance(kernel, d))
     gpu.close()
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_topk_rows_that_are_all_alike(kernel):
+    # every candidate is (almost) the same direction as every query: nothing can be dismissed early, every
+    # pair gets an exact cosine, and the order is decided in the last bits
+    rng = np.random.default_rng(17)
+    V, d = 4000, 64
+    v = rng.normal(size=d)
+    rows = (rng.uniform(0.5, 2.0, size=(V, 1)) * v + 1e-4 * rng.normal(size=(V, d))).astype(np.float32)
+    gpu, cpu, X = pair(V, d, 0, rows=rows, kernel=kernel)
+    q = rng.integers(0, V, 96)
+    check(gpu, cpu, X, 0, q, 0, V, 10, -2.0, tolerance(kernel, d))
+    check(gpu, cpu, X, 0, q, 100, 3000, 30, 0.999, tolerance(kernel, d))
+    gpu.close()
