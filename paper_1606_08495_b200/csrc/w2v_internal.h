@@ -66,6 +66,7 @@ struct StepParams {
     double *DV;                 // [hot_rows * d] fp64 sums of G u(c) for the most-hit output rows
     uint32_t hot_rows;          // output rows [0, hot_rows) accumulate in DV (snapshot mode)
     uint32_t zero;              // always 0; ANDed with a loaded word it ties a later address to that load's arrival
+    uint32_t keep_negs;         // snapshot mode: pass 1 writes the negatives of every pair to l_negs, pass 2 reads them back
 };
 
 // F arrays of all shards (this one included) that receive a shard's partial dot products.

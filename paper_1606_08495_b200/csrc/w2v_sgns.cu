@@ -77,12 +77,17 @@ sgns_snap_dots_kernel(StepParams p)
         Row<VPL> u, du;
         row_load(u, U4 + (size_t)c * p.ld4, p.d4, lane);
         row_zero(du);
-        unsigned long long gi = p.pair_off[q] * n1p;
+        unsigned long long pair = p.pair_off[q], gi = pair * n1p;
         for (uint32_t pp = q - left; pp <= q + right; ++pp) {
             if (pp == q) continue;
             const uint32_t w_out = (uint32_t)p.ctok[pp];
             uint32_t n0, n1;
             draw_pair_negatives(p, i, pp + p.window - q, w_out, lane, n0, n1, draws, redraws);
+            if (p.keep_negs) {
+                int32_t *dst = const_cast<int32_t *>(p.l_negs) + pair * p.negatives;     // this launch is the list's writer
+                if (lane < p.negatives) dst[lane] = (int32_t)n0;
+                if (lane + 32u < p.negatives) dst[lane + 32u] = (int32_t)n1;
+            }
             for_each_target_touched<VPL, TB>(p, u, w_out, n0, n1, lane,
                 [&](uint32_t t, uint32_t, const Row<VPL> &v, float f) {
                     const float s = sigmoidf_exact(f);
@@ -91,6 +96,7 @@ sgns_snap_dots_kernel(StepParams p)
                     row_axpy(du, g, v);
                 });
             gi += n1p;
+            ++pair;
         }
 #pragma unroll
         for (int v = 0; v < VPL; ++v) {
@@ -103,6 +109,8 @@ sgns_snap_dots_kernel(StepParams p)
 
 // ---- snapshot mode, pass 2 (Algorithm 2, output rows): v(target) += G u(c) ------------------
 // U is still untouched, so u(c) is the start-of-step vector; V is only added to (adjust_targets).
+// The negatives are read back from pass 1's list when there is one (a draw costs a random read of the
+// alias table), else regenerated from the seed as the paper's adjust call does (column shards).
 template <int VPL>
 __global__ void __launch_bounds__(kBlock)
 sgns_snap_adjust_v_kernel(StepParams p)
@@ -122,14 +130,21 @@ sgns_snap_adjust_v_kernel(StepParams p)
         const uint32_t i = p.cidx[q];
         Row<VPL> u;
         row_load(u, U4 + (size_t)c * p.ld4, p.d4, lane);
-        unsigned long long gi = p.pair_off[q] * n1p;
+        unsigned long long pair = p.pair_off[q], gi = pair * n1p;
         for (uint32_t pp = q - left; pp <= q + right; ++pp) {
             if (pp == q) continue;
             const uint32_t w_out = (uint32_t)p.ctok[pp];
-            uint32_t n0, n1;
-            draw_pair_negatives(p, i, pp + p.window - q, w_out, lane, n0, n1, draws, redraws);
+            uint32_t n0 = 0, n1 = 0;
+            if (p.keep_negs) {
+                const int32_t *src = p.l_negs + pair * p.negatives;
+                if (lane < p.negatives) n0 = (uint32_t)__ldcg(src + lane);
+                if (lane + 32u < p.negatives) n1 = (uint32_t)__ldcg(src + lane + 32u);
+            } else {
+                draw_pair_negatives(p, i, pp + p.window - q, w_out, lane, n0, n1, draws, redraws);
+            }
             adjust_targets<VPL>(p, u, w_out, n0, n1, gi, lane);
             gi += n1p;
+            ++pair;
         }
     }
 }
