@@ -324,8 +324,8 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
  *      few within 4.5e-3 of it are recomputed as fp32 dot products of the two rows, and only those
  *      values are ranked and returned: cosines within about 1e-6 of exact, as with kind 0.  Needs
  *      scratch for the bf16 copy of the candidates (2 d bytes per candidate, at most 2^22
- *      candidates at a time: longer ranges are handled in pieces).  Rows of more than 320 columns
- *      do not fit this kernel's shared-memory plan and are handled as kind 1.
+ *      candidates and 2.7 GB at a time: longer ranges are handled in pieces).  Up to 320 columns
+ *      the query block stays in shared memory; wider rows stream it beside the candidates.
  *   A block of kind 1 or 2 that waits too long on its own pipeline gives up; w2v_sync then
  *   returns W2V_ERR_CUDA.
  */

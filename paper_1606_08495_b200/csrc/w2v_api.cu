@@ -749,9 +749,9 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
     }
     // few query blocks: split the candidates over several blocks per query block, merge afterwards
     const bool tc = h->retrieval_kernel >= 1;
-    const bool screen = h->retrieval_kernel == 2 && topk_screen_fits(h->d);
+    const bool screen = h->retrieval_kernel == 2;
     // the screening kernel takes the candidates in chunks, each with its own set of partial lists
-    const uint64_t chunk = screen ? topk_screen_chunk(nc) : nc;
+    const uint64_t chunk = screen ? topk_screen_chunk(nc, h->d) : nc;
     const uint64_t chunks = chunk ? (nc + chunk - 1) / chunk : 0;
     const uint64_t splits = tc ? topk_splits(m, chunk, h->sms, 128, 256) : topk_splits(m, nc, h->sms);
     const uint64_t lists = screen ? chunks * splits : splits;

@@ -152,12 +152,10 @@ int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, 
                    int *error, bool screen, int sms, cudaStream_t s);
 // inv_norm: 1/|row| of the candidates, an input for the three-MMA kernel (launch_inv_norms); the screening
 // variant computes it itself while it packs the candidates.
-// The screening variant: whether it can take rows of d columns; how many candidates it handles per
-// launch (a range is cut into chunks of that size, each with its own partial lists); bytes of the
-// packed bf16 copy of one chunk.
-uint64_t topk_screen_chunk(uint64_t n_candidates);
+// The screening variant: how many candidates it handles per launch (a range is cut into chunks of that
+// size, each with its own partial lists); bytes of the packed bf16 copy of one chunk.
+uint64_t topk_screen_chunk(uint64_t n_candidates, uint32_t d);
 size_t topk_screen_ctiles_bytes(uint64_t n_candidates, uint32_t d);
-bool topk_screen_fits(uint32_t d);
 int launch_inv_norms(const float *table, uint32_t d, uint32_t ld, uint64_t lo, uint64_t count, float *inv_norm,
                      int sms, cudaStream_t s);
 // Returns launches made, -1 on a launch error, -2 if the shape does not fit shared memory.

@@ -404,7 +404,7 @@ topk_cosine_tc_kernel(TcParams p)
 constexpr float kScreenEps = 4.5e-3f;
 constexpr int kScKB = 32;                                        // columns per stage
 constexpr int kScCh = kScKB / 8;                                 // 16-byte chunks (8 bf16) per row and stage
-constexpr int kScMaxKB = 10;                                     // stages per row that fit: d <= 320
+constexpr int kScMaxKB = 10;                                     // K-blocks of a query block that can stay in shared memory: d <= 320
 constexpr int kScStages = 8;
 constexpr int kScAChunk = kTcM * 16;                             // query operand, one 16-byte chunk of all rows
 constexpr int kScABlock = kScCh * kScAChunk;                     // bytes of one K-block of the query operand
@@ -521,13 +521,18 @@ __device__ __forceinline__ void tmem_ld32(uint32_t (&v)[32], uint32_t taddr)
                  : "r"(taddr));
 }
 
+// RES: the query block is resident in shared memory (d <= 320); otherwise its K-blocks stream through
+// the stages beside the candidates' (8 KB + 16 KB per stage).
+template <bool RES>
 __global__ void __launch_bounds__(kScThreads, 1)
 topk_cosine_screen_kernel(TcParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char *a_op = smem;                                              // [kScMaxKB] query K-blocks
-    unsigned char *b_op = smem + kScMaxKB * kScABlock;                       // [kScStages] candidate stages
-    uint64_t *full = reinterpret_cast<uint64_t *>(b_op + kScStages * kScStageBytes);
+    // RES: [kScMaxKB query K-blocks][kScStages candidate stages]; else [kScStages stages of (query K-block, candidate K-block)]
+    constexpr int kStage = RES ? kScStageBytes : kScABlock + kScStageBytes;
+    unsigned char *a_op = smem;
+    unsigned char *b_op = smem + (RES ? kScMaxKB * kScABlock : kScABlock);
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + (RES ? kScMaxKB * kScABlock : 0) + kScStages * kStage);
     uint64_t *empty = full + kScStages;
     uint64_t *tfull = empty + kScStages;
     uint64_t *tempty = tfull + 2;
@@ -706,13 +711,16 @@ topk_cosine_screen_kernel(TcParams p)
         if (lane == 0) {
             // bf16 x bf16 -> fp32, both operands K-major, N = 256, M = 128
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcN >> 3) << 17) | ((uint32_t)(kTcM >> 4) << 24);
-            // the query block: one bulk copy per K-block, all on one barrier
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
-                         ::"r"(smem_addr(afull)), "r"(nkb * (uint32_t)kScABlock) : "memory");
-            for (uint32_t kb = 0; kb < nkb; ++kb)
-                bulk_to_smem(a_op + (size_t)kb * kScABlock, p.qsplit + ((size_t)blockIdx.x * nkb + kb) * kScABlock,
-                             (uint32_t)kScABlock, afull);
-            bool ok = mbar_wait(afull, 0u, abort_flag);
+            bool ok = true;
+            if (RES) {
+                // the query block: one bulk copy per K-block, all on one barrier
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                             ::"r"(smem_addr(afull)), "r"(nkb * (uint32_t)kScABlock) : "memory");
+                for (uint32_t kb = 0; kb < nkb; ++kb)
+                    bulk_to_smem(a_op + (size_t)kb * kScABlock, p.qsplit + ((size_t)blockIdx.x * nkb + kb) * kScABlock,
+                                 (uint32_t)kScABlock, afull);
+                ok = mbar_wait(afull, 0u, abort_flag);
+            }
             uint64_t g = 0;
             for (uint64_t i = 0; i < n_tiles && ok; ++i) {
                 const uint32_t b = (uint32_t)(i & 1);
@@ -724,8 +732,8 @@ topk_cosine_screen_kernel(TcParams p)
                     ok = mbar_wait(full + s, (uint32_t)((g / kScStages) & 1), abort_flag);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t abase = smem_addr(a_op + (size_t)kb * kScABlock);
-                    const uint32_t bbase = smem_addr(b_op + (size_t)s * kScStageBytes);
+                    const uint32_t abase = smem_addr(a_op + (RES ? (size_t)kb * kScABlock : (size_t)s * kStage));
+                    const uint32_t bbase = smem_addr(b_op + (size_t)s * kStage);
                     const uint32_t cols = 4u * p.d4 - kb * kScKB < (uint32_t)kScKB ? 4u * p.d4 - kb * kScKB : (uint32_t)kScKB;
                     const uint32_t nk = (cols + 15u) / 16u;                              // MMAs of K = 16 columns with data
                     for (uint32_t kk = 0; kk < nk; ++kk) {
@@ -749,8 +757,11 @@ topk_cosine_screen_kernel(TcParams p)
                 const uint32_t s = (uint32_t)(g % kScStages);
                 if (!mbar_wait(empty + s, (uint32_t)(((g / kScStages) & 1) ^ 1), abort_flag)) break;
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
-                             ::"r"(smem_addr(full + s)), "r"((uint32_t)kScStageBytes) : "memory");
-                bulk_to_smem(b_op + (size_t)s * kScStageBytes,
+                             ::"r"(smem_addr(full + s)), "r"((uint32_t)kStage) : "memory");
+                if (!RES)
+                    bulk_to_smem(a_op + (size_t)s * kStage, p.qsplit + ((size_t)blockIdx.x * nkb + g % nkb) * kScABlock,
+                                 (uint32_t)kScABlock, full + s);
+                bulk_to_smem(b_op + (size_t)s * kStage,
                              p.ctiles + ((t_lo + g / nkb) * nkb + g % nkb) * (size_t)kScStageBytes, (uint32_t)kScStageBytes, full + s);
             }
             if (*abort_flag) {
@@ -771,12 +782,15 @@ topk_cosine_screen_kernel(TcParams p)
     }
 }
 
-static size_t topk_screen_smem_bytes()
+static size_t topk_screen_smem_bytes(bool resident)
 {
-    return (size_t)kScMaxKB * kScABlock + (size_t)kScStages * kScStageBytes + (2 * kScStages + 5) * 8 + 8 + kTcM * 8 + 128;
+    const size_t operands = resident ? (size_t)kScMaxKB * kScABlock + (size_t)kScStages * kScStageBytes
+                                     : (size_t)kScStages * (kScABlock + kScStageBytes);
+    return operands + (2 * kScStages + 5) * 8 + 8 + kTcM * 8 + 128;
 }
 
-bool topk_screen_fits(uint32_t d) { return (d + kScKB - 1) / kScKB <= (uint32_t)kScMaxKB; }
+// whether the query block of rows of d columns can stay in shared memory
+static bool topk_screen_resident(uint32_t d) { return (d + kScKB - 1) / kScKB <= (uint32_t)kScMaxKB; }
 
 size_t topk_tc_smem_bytes()
 {
@@ -789,15 +803,23 @@ size_t topk_tc_qsplit_bytes(uint64_t m, uint32_t d)
     return (size_t)(qblocks * nkb * 2 * kTcOperand);          // the screening layout needs less (kScABlock per K-block)
 }
 
-// Screening kernel: candidates are handled in chunks of at most kScChunk rows (the packed bf16 copy of
-// one chunk is the scratch `ctiles`); every chunk has its own `splits` partial lists.
+// Screening kernel: candidates are handled in chunks of at most kScChunk rows and at most kScScratch
+// bytes of packed bf16 copy (the scratch `ctiles`); every chunk has its own `splits` partial lists.
 constexpr uint64_t kScChunk = 1ull << 22;
+constexpr uint64_t kScScratch = 2752512000ull;                  // 2^22 rows of 320 columns, plus a little
 
-uint64_t topk_screen_chunk(uint64_t nc) { return nc < kScChunk ? nc : kScChunk; }
+uint64_t topk_screen_chunk(uint64_t nc, uint32_t d)
+{
+    const uint64_t nkb = (d + kScKB - 1) / kScKB;
+    uint64_t chunk = kScScratch / (nkb * kScStageBytes) * kTcN;     // whole tiles
+    if (chunk > kScChunk) chunk = kScChunk;
+    if (chunk < (uint64_t)kTcN) chunk = kTcN;
+    return nc < chunk ? nc : chunk;
+}
 
 size_t topk_screen_ctiles_bytes(uint64_t nc, uint32_t d)
 {
-    const uint64_t chunk = topk_screen_chunk(nc), tiles = (chunk + kTcN - 1) / kTcN, nkb = (d + kScKB - 1) / kScKB;
+    const uint64_t chunk = topk_screen_chunk(nc, d), tiles = (chunk + kTcN - 1) / kTcN, nkb = (d + kScKB - 1) / kScKB;
     return (size_t)(tiles * nkb * kScStageBytes);
 }
 
@@ -810,7 +832,6 @@ int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, 
 {
     if (m == 0) return 0;
     const unsigned qblocks = (unsigned)((m + kTcM - 1) / kTcM);
-    screen = screen && topk_screen_fits(d);
     TcParams p;
     p.qsplit = qsplit; p.ctiles = ctiles;
     p.table = table; p.queries = queries; p.inv_norm = inv_norm; p.part_cos = part_cos; p.part_ids = part_ids;
@@ -831,11 +852,13 @@ int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, 
     const uint32_t nkb = (d + kScKB - 1) / kScKB;
     topk_round_queries_kernel<<<qblocks * nkb, 256, 0, s>>>(table, queries, m, vocab, d / 4, ld / 4, nkb, qsplit);
     if (cudaGetLastError() != cudaSuccess) return -1;
-    const size_t sm = topk_screen_smem_bytes();
-    if (cudaFuncSetAttribute(topk_cosine_screen_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess)
+    const bool resident = topk_screen_resident(d);
+    const size_t sm = topk_screen_smem_bytes(resident);
+    if (cudaFuncSetAttribute(resident ? topk_cosine_screen_kernel<true> : topk_cosine_screen_kernel<false>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess)
         return -1;
     int launched = 1;
-    const uint64_t nc = cand_hi - cand_lo, chunk = topk_screen_chunk(nc);
+    const uint64_t nc = cand_hi - cand_lo, chunk = topk_screen_chunk(nc, d);
     uint64_t list = 0;
     for (uint64_t c0 = 0; c0 < nc; c0 += chunk, ++list) {
         const uint64_t n = nc - c0 < chunk ? nc - c0 : chunk;
@@ -845,7 +868,8 @@ int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, 
         p.inv_norm = inv_norm + c0;
         p.part_cos = part_cos + list * splits * m * K;
         p.part_ids = part_ids + list * splits * m * K;
-        topk_cosine_screen_kernel<<<grid, kScThreads, sm, s>>>(p);
+        if (resident) topk_cosine_screen_kernel<true><<<grid, kScThreads, sm, s>>>(p);
+        else topk_cosine_screen_kernel<false><<<grid, kScThreads, sm, s>>>(p);
         if (cudaGetLastError() != cudaSuccess) return -1;
         launched += 2;
     }

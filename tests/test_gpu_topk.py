@@ -21,7 +21,7 @@ def tolerance(kernel, d):
     the head/tail split leaves ~2^-21 per product, but the accumulator in tensor memory is updated
     3 * d/8 times (three MMAs per 8 columns) with rounding toward zero, each time up to 2^-24 of the
     running sum (|cos| <= 1): a bias of up to 3 (d/8) 2^-24 on top."""
-    if kernel == 0 or (kernel == 2 and d <= 320):      # the screen ranks and returns fp32 dot products (d <= 320; else kernel 1 runs)
+    if kernel in (0, 2):                               # the screen ranks and returns fp32 dot products
         return TOL
     return TOL + 3 * ((d + 7) // 8) * 2.0 ** -24
 
