@@ -304,8 +304,9 @@ int32_t w2v_write_rows(w2v_handle *h, uint32_t which, const int64_t *ids, uint64
  * Accuracy of the cosines: see w2v_set_retrieval_kernel.  Asynchronous except when scratch
  * (1/|x| per candidate, partial lists) has to grow.  Errors: W2V_ERR_ARG, W2V_ERR_NOMEM,
  * W2V_ERR_CUDA.  Reads the table as it is: call it between steps, not during one.  Scratch grows
- * with m (about 2.6 KB per query at d = 300 for the split query rows, plus 12 K bytes per query and
- * candidate split for the partial lists): hand large query sets over in batches of some 10^4-10^5.
+ * with m (about 2.6 KB per query at d = 300 for the converted query rows, plus 12 K bytes per query
+ * and candidate split for the partial lists): hand large query sets over in batches of some
+ * 10^4-10^5.  The default kernel also keeps a bf16 copy of up to 2^22 candidates (at most 2.7 GB).
  */
 int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, uint64_t m,
                         uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, int64_t *out_ids,
