@@ -332,8 +332,17 @@ int32_t cbow_step_impl(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_
             W2V_CUDA(h, cudaMemsetAsync(h->DV, 0, need_dv * sizeof(double), h->stream));
             h->DV_cap = need_dv;
         }
+        // the negatives of every example: drawn in pass 1, read back in pass 2 (indexed by kept position)
+        const uint64_t need_negs = h->st_host->n_kept * (uint64_t)negatives;
+        if (need_negs > h->l_cap_negs) {
+            cudaFree(h->l_negs); h->l_negs = nullptr; h->l_cap_negs = 0;
+            const uint64_t cap = need_negs + need_negs / 4 + 1024;
+            W2V_CUDA(h, dev_alloc(&h->l_negs, cap));
+            h->l_cap_negs = cap;
+        }
         if (h->st_host->pairs > 0) {
             StepParams p = make_params(h, window, negatives, lr);
+            p.keep_negs = 1u;
             if ((rc = profile_mark(h)) != W2V_OK) return rc;
             int k = launch_cbow_snapshot(p, h->blocks_per_sm, h->sms, h->stream);
             if (k < 0) return fail(h, W2V_ERR_CUDA, "update kernel launch", cudaGetLastError());

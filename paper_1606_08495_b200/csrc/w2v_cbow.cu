@@ -103,9 +103,14 @@ cbow_snap_dots_kernel(StepParams p)
         context_mean<VPL, TB>(p, q, left, cw, lane, h, inv);
         uint32_t n0, n1;
         draw_pair_negatives(p, p.cidx[q], p.window, wq, lane, n0, n1, draws, redraws);
+        if (p.keep_negs) {
+            int32_t *dst = const_cast<int32_t *>(p.l_negs) + (size_t)q * p.negatives;     // this launch is the list's writer
+            if (lane < p.negatives) dst[lane] = (int32_t)n0;
+            if (lane + 32u < p.negatives) dst[lane + 32u] = (int32_t)n1;
+        }
         row_zero(e);
         const size_t gi = (size_t)q * n1p;
-        for_each_target<VPL, TB>(p, h, wq, n0, n1, lane,
+        for_each_target_touched<VPL, TB>(p, h, wq, n0, n1, lane,
             [&](uint32_t t, uint32_t, const Row<VPL> &v, float f) {
                 const float s = sigmoidf_exact(f);
                 const float g = t == 0 ? p.lr * (1.0f - s) : -p.lr * s;
@@ -141,8 +146,14 @@ cbow_snap_adjust_v_kernel(StepParams p)
         Row<VPL> h;
         float inv;
         context_mean<VPL, TB>(p, q, left, cw, lane, h, inv);
-        uint32_t n0, n1;
-        draw_pair_negatives(p, p.cidx[q], p.window, wq, lane, n0, n1, draws, redraws);
+        uint32_t n0 = 0, n1 = 0;
+        if (p.keep_negs) {
+            const int32_t *src = p.l_negs + (size_t)q * p.negatives;
+            if (lane < p.negatives) n0 = (uint32_t)__ldcg(src + lane);
+            if (lane + 32u < p.negatives) n1 = (uint32_t)__ldcg(src + lane + 32u);
+        } else {
+            draw_pair_negatives(p, p.cidx[q], p.window, wq, lane, n0, n1, draws, redraws);
+        }
         adjust_targets<VPL>(p, h, wq, n0, n1, (unsigned long long)q * n1p, lane);
     }
 }
