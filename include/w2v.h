@@ -320,9 +320,9 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
  *      hardware updates 3 d/8 times with rounding toward zero: cosines within about
  *      2e-6 + 3 (d/8) 2^-24 of exact (9e-6 at d = 300; 2e-6 typical), at three times the speed.
  *   2  the tensor cores as a screen (the default): queries and unit-length candidates are rounded
- *      to bf16 and one MMA per pair of values gives every cosine to about 4e-3, which decides for
+ *      to bf16 and one MMA per pair of values gives every cosine to within 8e-3, which decides for
  *      all but a few candidates that they cannot reach the query's current K-th best (or tau); the
- *      few within 4.5e-3 of it are recomputed as fp32 dot products of the two rows, and only those
+ *      few within 8.5e-3 of it are recomputed as fp32 dot products of the two rows, and only those
  *      values are ranked and returned: cosines within about 1e-6 of exact, as with kind 0.  Needs
  *      scratch for the bf16 copy of the candidates (2 d bytes per candidate, at most 2^22
  *      candidates and 2.7 GB at a time: longer ranges are handled in pieces).  Up to 320 columns

@@ -386,10 +386,11 @@ topk_cosine_tc_kernel(TcParams p)
 
 // =================================================================================================
 // Screening variant.  One low-precision MMA per product instead of three TF32 ones: both sides are
-// rounded to bf16 (relative error at most 2^-9 per value), so each product is off by at most
-// (2^-8 + 2^-18) |a_i b_i| and, by Cauchy-Schwarz, the cosine by less than 3.92e-3; the fp32
-// accumulation adds some 1e-5.  That is enough to decide that a candidate cannot reach a query's
-// current cut.  Only a candidate whose approximate cosine comes within kScreenEps of the cut is
+// rounded to bf16 (8 significant bits: relative error at most 2^-8 per value), so each product is off
+// by at most (2^-7 + 2^-16) |a_i b_i| and, by Cauchy-Schwarz, the cosine by less than 7.83e-3; the fp32
+// accumulation adds some 1e-5.  (Rows of a few hundred columns come nowhere near: 6e-4 is typical at
+// d = 300; rows of 4 columns reach 5e-3.)  That is enough to decide that a candidate cannot reach a
+// query's current cut.  Only a candidate whose approximate cosine comes within kScreenEps of the cut is
 // looked at again: its warp computes the fp32 dot product of the two rows from the table, and that
 // exact cosine goes to the sorted list.  With a list of K the number of such candidates is about
 // K ln(n / K) per query, against n screened.
@@ -401,7 +402,7 @@ topk_cosine_tc_kernel(TcParams p)
 // columns of a 256-candidate tile: two MMAs of K = 16), each filled by one `cp.async.bulk` that a
 // single producer lane issues as soon as the stage's previous MMAs have committed.  The bf16 copy
 // halves what every query block pulls through L2, which is what bounds this kernel.
-constexpr float kScreenEps = 4.5e-3f;
+constexpr float kScreenEps = 8.5e-3f;
 constexpr int kScKB = 32;                                        // columns per stage
 constexpr int kScCh = kScKB / 8;                                 // 16-byte chunks (8 bf16) per row and stage
 constexpr int kScMaxKB = 10;                                     // K-blocks of a query block that can stay in shared memory: d <= 320
