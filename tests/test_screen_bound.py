@@ -7,6 +7,9 @@ bits (bf16: 7 stored, one implied) changes a value by at most 2^-8 of itself, so
 (2^-7 + 2^-16) of itself, and by Cauchy-Schwarz the cosine by at most 2^-7 + 2^-16 = 7.83e-3.  Checked
 here on random rows and on rows built so that every rounding error has the same sign and nearly the
 largest size."""
+import os
+import re
+
 import numpy as np
 
 BOUND = 2.0 ** -7 + 2.0 ** -16
@@ -71,3 +74,11 @@ def test_margin_covers_bound_and_fp32_accumulation():
     # fp32 accumulation of d = 1024 products of magnitude <= 1 and the two scalings add at most about
     # (d/16 + 4) 2^-24 to the bound (one rounding per 16-column MMA step plus the scalings)
     assert BOUND + (1024 / 16 + 4) * 2.0 ** -24 < MARGIN
+
+
+def test_margin_is_the_kernels():
+    src = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "paper_1606_08495_b200", "csrc",
+                       "w2v_topk_tc.cu")
+    with open(src) as f:
+        m = re.search(r"constexpr float kScreenEps = ([0-9.eE+-]+)f;", f.read())
+    assert m and float(m.group(1)) == MARGIN
