@@ -1,5 +1,7 @@
 // Cosine retrieval on the tensor cores (tcgen05, TMEM accumulators), same contract as the fp32
-// kernel in w2v_topk.cu.
+// kernel in w2v_topk.cu.  Two kernels: first the one that forms every cosine to full accuracy on the
+// tensor cores (three TF32 MMAs per product), then, further down, the default: a bf16 screen followed
+// by exact fp32 cosines for the few candidates that the screen cannot dismiss.
 //
 // The dot products of 128 query rows with 256 candidate rows are one M128 x N256 accumulator tile in
 // tensor memory.  The tensor cores read fp32 operands as TF32 (the 13 low mantissa bits are
