@@ -28,6 +28,7 @@ struct w2v_handle {
     int *tc_error = nullptr;             // device word raised by a tensor-core block whose wait ran out
     unsigned char *qsplit = nullptr; uint64_t qsplit_cap = 0;   // query rows split into TF32 head and tail
     unsigned char *ctiles = nullptr; uint64_t ctiles_cap = 0;   // candidate rows packed as bf16 operand blocks (screening kernel)
+    unsigned int *floor_q = nullptr; uint64_t floor_cap = 0;    // per query: best K-th cosine reached by any block (screening kernel)
     uint32_t pend_window = 0, pend_negatives = 0;
     uint64_t pend_n = 0, pend_pairs = 0;
     uint64_t seed = 0;
@@ -427,7 +428,7 @@ int32_t w2v_destroy(w2v_handle *h)
     if (h->st_host) cudaFreeHost(h->st_host);
     cudaFree(h->G); cudaFree(h->DU); cudaFree(h->DV); cudaFree(h->tok_stage);
     cudaFree(h->l_centre); cudaFree(h->l_context); cudaFree(h->l_negs);
-    cudaFree(h->inv_norm); cudaFree(h->part_cos); cudaFree(h->part_ids); cudaFree(h->tc_error); cudaFree(h->qsplit); cudaFree(h->ctiles);
+    cudaFree(h->inv_norm); cudaFree(h->part_cos); cudaFree(h->part_ids); cudaFree(h->tc_error); cudaFree(h->qsplit); cudaFree(h->ctiles); cudaFree(h->floor_q);
     for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
     cudaGetLastError();
     delete h;
@@ -765,6 +766,12 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
     const uint64_t splits = tc ? topk_splits(m, chunk, h->sms, 128, 256) : topk_splits(m, nc, h->sms);
     const uint64_t lists = screen ? chunks * splits : splits;
     const uint64_t need = (splits > 1 || tc) ? lists * m * K : 0;
+    if (screen && m > h->floor_cap) {
+        W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+        cudaFree(h->floor_q); h->floor_q = nullptr; h->floor_cap = 0;
+        W2V_CUDA(h, dev_alloc(&h->floor_q, m));
+        h->floor_cap = m;
+    }
     if (screen && topk_screen_ctiles_bytes(nc, h->d) > h->ctiles_cap) {
         W2V_CUDA(h, cudaStreamSynchronize(h->stream));
         cudaFree(h->ctiles); h->ctiles = nullptr; h->ctiles_cap = 0;
@@ -798,7 +805,7 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
     int k2;
     if (tc) {
         k2 = launch_topk_tc(table, h->d, h->ld, h->vocab, reinterpret_cast<const long long *>(queries), m, cand_lo,
-                            cand_hi, K, tau, h->inv_norm, h->qsplit, h->ctiles, h->part_cos, h->part_ids, (uint32_t)splits,
+                            cand_hi, K, tau, h->inv_norm, h->qsplit, h->ctiles, h->floor_q, h->part_cos, h->part_ids, (uint32_t)splits,
                             h->tc_error, screen, h->sms, h->stream);
         if (k2 >= 0) {
             const int k3 = launch_topk_merge(h->part_cos, h->part_ids, m, K, (uint32_t)lists, out_cos,

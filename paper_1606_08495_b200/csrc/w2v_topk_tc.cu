@@ -128,6 +128,7 @@ struct TcParams {
     const float *inv_norm;
     const unsigned char *qsplit;  // [query blocks][K-blocks][hi, lo] operand blocks, laid out as in shared memory
     const unsigned char *ctiles;  // screening kernel: candidate operand blocks (topk_pack_candidates_kernel)
+    unsigned int *floor_q;        // screening kernel: [m] best K-th cosine any block has reached for the query (ordered encoding, 0 = none)
     float *part_cos;              // [splits][m][K]
     long long *part_ids;
     int *error;                   // device word: set to 1 if a wait ran out
@@ -524,6 +525,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t (&v)[32], uint32_t taddr)
                  : "r"(taddr));
 }
 
+// Floats as unsigned integers in the same order (0 is below every float): for atomicMax.
+__device__ __forceinline__ unsigned int ordered_bits(float f)
+{
+    const unsigned int u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float ordered_float(unsigned int o)
+{
+    return __uint_as_float((o & 0x80000000u) ? (o & 0x7FFFFFFFu) : ~o);
+}
+
 // RES: the query block is resident in shared memory (d <= 320); otherwise its K-blocks stream through
 // the stages beside the candidates' (8 KB + 16 KB per stage).
 template <bool RES>
@@ -595,11 +607,15 @@ topk_cosine_screen_kernel(TcParams p)
         const bool mine = my_q >= 0 && live;
         uint32_t have = 0;
         float thr = p.tau;
+        // The blocks that work on other candidates of the same queries publish the K-th best cosine they
+        // have reached (floor_q, raised by atomicMax); K candidates at or above it exist, so whatever is
+        // below it cannot be among the query's final K, in any block.  Read once per tile.
+        float flo = -INFINITY;
         // one chunk of 32 columns of the current tile (first candidate c0 + cc)
         uint64_t c0 = 0;
         auto screen_chunk = [&](const uint32_t (&v)[32], uint32_t cc) {
             __syncwarp();
-            const float cut = (have < p.K ? p.tau : fmaxf(p.tau, thr)) - kScreenEps;
+            const float cut = fmaxf(have < p.K ? p.tau : fmaxf(p.tau, thr), flo) - kScreenEps;
             float top = __uint_as_float(v[0]);
 #pragma unroll
             for (int j = 1; j < 32; ++j) top = fmaxf(top, __uint_as_float(v[j]));
@@ -619,7 +635,7 @@ topk_cosine_screen_kernel(TcParams p)
                 if (!owners) break;
                 bool on[kExact];
                 uint32_t src[kExact], hv[kExact];
-                float th[kExact], qi[kExact], dot[kExact], e0[kExact], e1[kExact];
+                float th[kExact], fl[kExact], qi[kExact], dot[kExact], e0[kExact], e1[kExact];
                 long long i0[kExact], i1[kExact], qr[kExact];
                 uint64_t cnd[kExact];
 #pragma unroll
@@ -632,6 +648,7 @@ topk_cosine_screen_kernel(TcParams p)
                     qr[e] = qrow[warp * 32u + src[e]];
                     hv[e] = __shfl_sync(kFullMask, have, src[e]);
                     th[e] = __shfl_sync(kFullMask, thr, src[e]);
+                    fl[e] = __shfl_sync(kFullMask, flo, src[e]);
                     qi[e] = __shfl_sync(kFullMask, qinv, src[e]);
                     if (on[e] && lane == src[e]) maybe &= maybe - 1u;
                     e0[e] = 0.f; e1[e] = 0.f; i0[e] = -1; i1[e] = -1; dot[e] = 0.f;
@@ -662,7 +679,7 @@ topk_cosine_screen_kernel(TcParams p)
                     if (!on[e]) continue;                                                   // same for every lane
                     const float cs = dot[e] * qi[e] * __ldg(p.inv_norm + cnd[e]);
                     const long long cid = (long long)(p.cand_lo + cnd[e]);
-                    if (!(cs > p.tau) || cid == qr[e] || (hv[e] == p.K && cs < th[e])) continue;
+                    if (!(cs > p.tau) || cid == qr[e] || (hv[e] == p.K && cs < th[e]) || cs < fl[e]) continue;
                     const size_t lb = ((size_t)blockIdx.y * p.m + (q0 + warp * 32u + src[e])) * p.K;
                     float *wl = p.part_cos + lb;
                     long long *wi = p.part_ids + lb;
@@ -678,6 +695,7 @@ topk_cosine_screen_kernel(TcParams p)
                         if (lane == src[e]) {
                             have = hv[e] < p.K ? hv[e] + 1u : p.K;
                             thr = have == p.K ? (pos == p.K - 1u ? cs : e_km2) : p.tau;
+                            if (have == p.K) atomicMax(p.floor_q + (q0 + warp * 32u + src[e]), ordered_bits(thr));
                         }
                     }
                 }
@@ -687,6 +705,7 @@ topk_cosine_screen_kernel(TcParams p)
         for (uint64_t i = 0; i < n_tiles; ++i) {
             const uint32_t b = (uint32_t)(i & 1);
             c0 = (t_lo + i) * kTcN;
+            if (mine) { const unsigned int o = __ldcg(p.floor_q + (q0 + r)); if (o) flo = ordered_float(o); }
             // the tensor-memory loads below are warp-wide: the whole warp goes on or gives up together
             if (!__all_sync(kFullMask, mbar_wait(tfull + b, (uint32_t)((i >> 1) & 1), abort_flag))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -830,13 +849,13 @@ size_t topk_screen_ctiles_bytes(uint64_t nc, uint32_t d)
 // chunks x splits for the screening kernel); the caller merges.
 int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, const long long *queries, uint64_t m,
                    uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, float *inv_norm,
-                   unsigned char *qsplit, unsigned char *ctiles, float *part_cos, long long *part_ids, uint32_t splits,
-                   int *error, bool screen, int sms, cudaStream_t s)
+                   unsigned char *qsplit, unsigned char *ctiles, unsigned int *floor_q, float *part_cos, long long *part_ids,
+                   uint32_t splits, int *error, bool screen, int sms, cudaStream_t s)
 {
     if (m == 0) return 0;
     const unsigned qblocks = (unsigned)((m + kTcM - 1) / kTcM);
     TcParams p;
-    p.qsplit = qsplit; p.ctiles = ctiles;
+    p.qsplit = qsplit; p.ctiles = ctiles; p.floor_q = floor_q;
     p.table = table; p.queries = queries; p.inv_norm = inv_norm; p.part_cos = part_cos; p.part_ids = part_ids;
     p.error = error; p.m = m; p.vocab = vocab; p.cand_lo = cand_lo; p.cand_hi = cand_hi;
     p.d4 = d / 4; p.ld4 = ld / 4; p.K = K; p.splits = splits; p.tau = tau;
@@ -855,6 +874,7 @@ int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, 
     const uint32_t nkb = (d + kScKB - 1) / kScKB;
     topk_round_queries_kernel<<<qblocks * nkb, 256, 0, s>>>(table, queries, m, vocab, d / 4, ld / 4, nkb, qsplit);
     if (cudaGetLastError() != cudaSuccess) return -1;
+    if (cudaMemsetAsync(floor_q, 0, m * sizeof(unsigned int), s) != cudaSuccess) return -1;   // 0 = no floor yet
     const bool resident = topk_screen_resident(d);
     const size_t sm = topk_screen_smem_bytes(resident);
     if (cudaFuncSetAttribute(resident ? topk_cosine_screen_kernel<true> : topk_cosine_screen_kernel<false>,
