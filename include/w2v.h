@@ -268,6 +268,30 @@ int32_t w2v_shard_dots(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_
 int32_t w2v_shard_adjust(w2v_handle *h, const float *F, float lr);
 
 /*
+ * The barrier between w2v_shard_dots and w2v_shard_adjust when the shards add their partial dot
+ * products straight into one another's arrays (the sum of Algorithm 3 done over peer pointers):
+ * one small kernel on the handle's stream that announces "shard `rank` has finished epoch `epoch`"
+ * to every shard and waits until every shard has announced it.  Stream order does the rest: the
+ * additions of this shard's w2v_shard_dots precede the announcement, and the w2v_shard_adjust
+ * enqueued after the barrier runs only once all announcements have arrived.
+ *   flags_peers  host array of n_peers (1..16) device pointers; flags_peers[r] is shard r's array
+ *                of n_peers uint32 epoch words (peer-to-peer pointers for r != rank), zeroed once
+ *                before the first step and never reset.
+ *   rank         which shard this handle is.
+ *   epoch        a counter the shards advance together, one per barrier, starting at 1 (compared
+ *                modulo 2^32, so it may wrap).
+ *   timeout_ms   1..600000.  A shard that never arrives (its process failed before the launch)
+ *                must not hang the others' GPUs: when the limit passes the kernel gives up, and
+ *                the next w2v_sync on this handle returns W2V_ERR_CUDA once (the step that ran
+ *                after the barrier used incomplete sums; the tables are to be restored from a
+ *                saved copy).  Nothing traps and the device stays usable.
+ * Kernels of different shards wait for one another here, so every shard must be on a GPU of its own
+ * (or, for one shard, n_peers == 1).  Asynchronous.
+ */
+int32_t w2v_peer_barrier(w2v_handle *h, uint32_t *const *flags_peers, uint32_t n_peers, uint32_t rank,
+                         uint32_t epoch, uint32_t timeout_ms);
+
+/*
  * Partial dot products of one column slice, the body of Algorithm 1 on shard s:
  * out[i] = sum_{j = col_lo}^{col_hi - 1} U[pairs[2i]][j] * V[pairs[2i+1]][j].
  * Summing the results over any partition of [0, d) gives the full dot products

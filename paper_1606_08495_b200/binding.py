@@ -18,6 +18,7 @@ W2V_ERR_ARG, W2V_ERR_STATE, W2V_ERR_NOMEM, W2V_ERR_CUDA = -1, -2, -3, -4
 W2V_ERR_TOKEN_RANGE, W2V_ERR_CAPACITY = -5, -6
 MODE_SNAPSHOT, MODE_HOGWILD = 0, 1
 TABLE_U, TABLE_V = 0, 1
+MAX_SHARDS = 16                  # most column shards (and epoch words per barrier array)
 
 EXPORTS = (
     "w2v_create", "w2v_create_strided", "w2v_create_shard", "w2v_shard_dots", "w2v_shard_adjust",
@@ -26,7 +27,7 @@ EXPORTS = (
     "w2v_sgns_step_host", "w2v_sample_pairs", "w2v_partial_dots", "w2v_read_rows", "w2v_write_rows",
     "w2v_set_step", "w2v_get_step", "w2v_get_table_ptrs", "w2v_sync", "w2v_profile_enable",
     "w2v_profile_read", "w2v_get_launch_count", "w2v_set_tuning", "w2v_last_error",
-    "w2v_sample_pairs_noalloc",
+    "w2v_sample_pairs_noalloc", "w2v_peer_barrier",
 )
 
 
@@ -71,6 +72,7 @@ def load():
         "w2v_create_shard": [u64, u32, u32, u32, u32, u64, vp, vp, vp, C.POINTER(vp)],
         "w2v_shard_dots": [vp, vp, u64, u32, u32, C.POINTER(vp), u32, u64, C.POINTER(StepStats)],
         "w2v_shard_adjust": [vp, vp, C.c_float],
+        "w2v_peer_barrier": [vp, C.POINTER(vp), u32, u32, u32, u32],
         "w2v_destroy": [vp],
         "w2v_build_alias": [vp, vp, C.c_double],
         "w2v_get_tables": [vp, vp, vp, vp],
@@ -161,6 +163,12 @@ def w2v_shard_dots(h, tokens, n, window, negatives, F_peers, cap, stats=None, al
 
 def w2v_shard_adjust(h, F, lr):
     return _check(h, load().w2v_shard_adjust(h, _ptr(F), float(lr)))
+
+
+def w2v_peer_barrier(h, flags_peers, rank, epoch, timeout_ms):
+    """flags_peers: device pointers (ints or tensors), one array of len(flags_peers) uint32 per shard."""
+    ptrs = (C.c_void_p * len(flags_peers))(*[_ptr(f) for f in flags_peers])
+    return _check(h, load().w2v_peer_barrier(h, ptrs, len(flags_peers), int(rank), int(epoch), int(timeout_ms)))
 
 
 def w2v_get_row_stride(h):

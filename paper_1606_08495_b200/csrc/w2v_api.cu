@@ -127,6 +127,62 @@ int32_t ensure_scratch(w2v_handle *h, uint64_t n)
     return W2V_OK;
 }
 
+// Makes *p hold at least `need` elements.  When it does not, the stream is drained (it may still
+// use the old array), the array is freed and a new one allocated; with `slack`, a quarter more than
+// asked for, so that chunks of slightly different sizes do not re-allocate every time.
+template <typename T>
+int32_t grow(w2v_handle *h, T **p, uint64_t *cap, uint64_t need, bool slack)
+{
+    if (need <= *cap) return W2V_OK;
+    W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+    cudaFree(*p); *p = nullptr; *cap = 0;
+    const uint64_t want = slack ? need + need / 4 + 1024 : need;
+    W2V_CUDA(h, dev_alloc(p, want));
+    *cap = want;
+    return W2V_OK;
+}
+
+// Scratch of the deferred-update passes (Algorithm 2's "not updated until the end of the call"):
+// coefficients G for `targets` targets, per-centre sums DU for every token the chunk scratch holds,
+// fp64 sums DV of the most-hit output rows (zero between steps).
+int32_t ensure_update_scratch(w2v_handle *h, uint64_t targets, bool slack)
+{
+    int32_t rc;
+    if ((rc = grow(h, &h->G, &h->G_cap, targets, slack)) != W2V_OK) return rc;
+    if ((rc = grow(h, &h->DU, &h->DU_cap, h->sc.n_cap * (uint64_t)h->d, false)) != W2V_OK) return rc;
+    const uint64_t need_dv = (uint64_t)h->hot_rows * h->d;
+    if (need_dv > h->DV_cap) {
+        if ((rc = grow(h, &h->DV, &h->DV_cap, need_dv, false)) != W2V_OK) return rc;
+        W2V_CUDA(h, cudaMemsetAsync(h->DV, 0, h->DV_cap * sizeof(double), h->stream));
+    }
+    return W2V_OK;
+}
+
+// Copies a chunk that lives in host memory into the handle's staging array (stream-ordered).
+int32_t stage_tokens(w2v_handle *h, const int32_t *tokens_host, uint64_t n)
+{
+    int32_t rc = grow(h, &h->tok_stage, &h->tok_stage_cap, n, false);
+    if (rc != W2V_OK) return rc;
+    if (n)
+        W2V_CUDA(h, cudaMemcpyAsync(h->tok_stage, tokens_host, n * sizeof(int32_t), cudaMemcpyHostToDevice, h->stream));
+    return W2V_OK;
+}
+
+// The device word that kernels with bounded waits raise when a wait runs out (read by w2v_sync).
+int32_t ensure_error_word(w2v_handle *h)
+{
+    if (h->tc_error) return W2V_OK;
+    W2V_CUDA(h, dev_alloc(&h->tc_error, 1));
+    W2V_CUDA(h, cudaMemsetAsync(h->tc_error, 0, sizeof(int), h->stream));
+    return W2V_OK;
+}
+
+// Snapshot mode sizes its per-target arrays from the bound "every token is an input word with a
+// full window" when they then stay within this many bytes: the steady-state step neither waits for
+// the pair count nor re-allocates.  Larger bounds (wide windows on long chunks) fall back to
+// reading the pair count.
+constexpr uint64_t kSnapshotBoundBudget = 1ull << 30;
+
 int32_t check_step_args(w2v_handle *h, const void *tokens, uint64_t n, uint32_t window, uint32_t negatives)
 {
     if (!h) return W2V_ERR_ARG;
@@ -245,37 +301,18 @@ int32_t step_impl(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t win
         int k = launch_pair_offsets(n, h->sc, h->st, h->stream);
         if (k < 0) return fail(h, W2V_ERR_CUDA, "pair offset launch", cudaGetLastError());
         h->launches += (uint64_t)k;
-        // the coefficient array is sized by the pair count, which only the device knows
-        if ((rc = read_state(h, n, nullptr)) != W2V_OK) return rc;
-        const uint64_t need_g = h->st_host->pairs * (uint64_t)(negatives + 1);
-        if (need_g > h->G_cap) {
-            cudaFree(h->G); h->G = nullptr; h->G_cap = 0;
-            const uint64_t cap = need_g + need_g / 4 + 1024;
-            W2V_CUDA(h, dev_alloc(&h->G, cap));
-            h->G_cap = cap;
+        // G and the list of negatives (drawn in pass 1, read back instead of drawn again in pass 2) hold
+        // one entry per target / per negative: sized from the bound when that is affordable, else
+        // from the pair count, which only the device knows
+        uint64_t pairs_cap = n * 2ull * window;
+        const bool bounded = pairs_cap * (2ull * negatives + 1ull) * sizeof(float) <= kSnapshotBoundBudget;
+        if (!bounded) {
+            if ((rc = read_state(h, n, nullptr)) != W2V_OK) return rc;
+            pairs_cap = h->st_host->pairs;
         }
-        const uint64_t need_du = h->sc.n_cap * (uint64_t)h->d;
-        if (need_du > h->DU_cap) {
-            cudaFree(h->DU); h->DU = nullptr; h->DU_cap = 0;
-            W2V_CUDA(h, dev_alloc(&h->DU, need_du));
-            h->DU_cap = need_du;
-        }
-        const uint64_t need_dv = (uint64_t)h->hot_rows * h->d;
-        if (need_dv > h->DV_cap) {
-            cudaFree(h->DV); h->DV = nullptr; h->DV_cap = 0;
-            W2V_CUDA(h, dev_alloc(&h->DV, need_dv));
-            W2V_CUDA(h, cudaMemsetAsync(h->DV, 0, need_dv * sizeof(double), h->stream));
-            h->DV_cap = need_dv;
-        }
-        // the negatives of every pair: drawn in pass 1, read back (instead of drawn again) in pass 2
-        const uint64_t need_negs = h->st_host->pairs * (uint64_t)negatives;
-        if (need_negs > h->l_cap_negs) {
-            cudaFree(h->l_negs); h->l_negs = nullptr; h->l_cap_negs = 0;
-            const uint64_t cap = need_negs + need_negs / 4 + 1024;
-            W2V_CUDA(h, dev_alloc(&h->l_negs, cap));
-            h->l_cap_negs = cap;
-        }
-        if (h->st_host->pairs > 0) {
+        if ((rc = ensure_update_scratch(h, pairs_cap * (uint64_t)(negatives + 1), !bounded)) != W2V_OK) return rc;
+        if ((rc = grow(h, &h->l_negs, &h->l_cap_negs, pairs_cap * (uint64_t)negatives, !bounded)) != W2V_OK) return rc;
+        if (pairs_cap > 0) {
             StepParams p = make_params(h, window, negatives, lr);
             p.keep_negs = 1u;
             if ((rc = profile_mark(h)) != W2V_OK) return rc;
@@ -311,37 +348,10 @@ int32_t cbow_step_impl(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_
         if (h->profiling) h->prof_launches += (uint64_t)k;
         if ((rc = profile_mark(h)) != W2V_OK) return rc;
     } else {
-        // coefficients are indexed by kept position, so the kept count sizes their array
-        if ((rc = read_state(h, n, nullptr)) != W2V_OK) return rc;
-        const uint64_t need_g = h->st_host->n_kept * (uint64_t)(negatives + 1);
-        if (need_g > h->G_cap) {
-            cudaFree(h->G); h->G = nullptr; h->G_cap = 0;
-            const uint64_t cap = need_g + need_g / 4 + 1024;
-            W2V_CUDA(h, dev_alloc(&h->G, cap));
-            h->G_cap = cap;
-        }
-        const uint64_t need_du = h->sc.n_cap * (uint64_t)h->d;
-        if (need_du > h->DU_cap) {
-            cudaFree(h->DU); h->DU = nullptr; h->DU_cap = 0;
-            W2V_CUDA(h, dev_alloc(&h->DU, need_du));
-            h->DU_cap = need_du;
-        }
-        const uint64_t need_dv = (uint64_t)h->hot_rows * h->d;
-        if (need_dv > h->DV_cap) {
-            cudaFree(h->DV); h->DV = nullptr; h->DV_cap = 0;
-            W2V_CUDA(h, dev_alloc(&h->DV, need_dv));
-            W2V_CUDA(h, cudaMemsetAsync(h->DV, 0, need_dv * sizeof(double), h->stream));
-            h->DV_cap = need_dv;
-        }
-        // the negatives of every example: drawn in pass 1, read back in pass 2 (indexed by kept position)
-        const uint64_t need_negs = h->st_host->n_kept * (uint64_t)negatives;
-        if (need_negs > h->l_cap_negs) {
-            cudaFree(h->l_negs); h->l_negs = nullptr; h->l_cap_negs = 0;
-            const uint64_t cap = need_negs + need_negs / 4 + 1024;
-            W2V_CUDA(h, dev_alloc(&h->l_negs, cap));
-            h->l_cap_negs = cap;
-        }
-        if (h->st_host->pairs > 0) {
+        // coefficients and kept negatives are indexed by kept position: at most one example per token
+        if ((rc = ensure_update_scratch(h, n * (uint64_t)(negatives + 1), false)) != W2V_OK) return rc;
+        if ((rc = grow(h, &h->l_negs, &h->l_cap_negs, n * (uint64_t)negatives, false)) != W2V_OK) return rc;
+        if (n > 0) {
             StepParams p = make_params(h, window, negatives, lr);
             p.keep_negs = 1u;
             if ((rc = profile_mark(h)) != W2V_OK) return rc;
@@ -499,14 +509,7 @@ int32_t w2v_sgns_step_host(w2v_handle *h, const int32_t *tokens_host, uint64_t n
     int32_t rc = check_step_args(h, tokens_host, n, window, negatives);
     if (rc != W2V_OK) return rc;
     DeviceGuard g(h->device);
-    if (n > h->tok_stage_cap) {
-        W2V_CUDA(h, cudaStreamSynchronize(h->stream));
-        cudaFree(h->tok_stage); h->tok_stage = nullptr; h->tok_stage_cap = 0;
-        W2V_CUDA(h, dev_alloc(&h->tok_stage, n));
-        h->tok_stage_cap = n;
-    }
-    if (n)
-        W2V_CUDA(h, cudaMemcpyAsync(h->tok_stage, tokens_host, n * sizeof(int32_t), cudaMemcpyHostToDevice, h->stream));
+    if ((rc = stage_tokens(h, tokens_host, n)) != W2V_OK) return rc;
     return step_impl(h, h->tok_stage, n, window, negatives, lr, mode, stats);
 }
 
@@ -553,14 +556,7 @@ int32_t w2v_cbow_step_host(w2v_handle *h, const int32_t *tokens_host, uint64_t n
     int32_t rc = check_step_args(h, tokens_host, n, window, negatives);
     if (rc != W2V_OK) return rc;
     DeviceGuard g(h->device);
-    if (n > h->tok_stage_cap) {
-        W2V_CUDA(h, cudaStreamSynchronize(h->stream));
-        cudaFree(h->tok_stage); h->tok_stage = nullptr; h->tok_stage_cap = 0;
-        W2V_CUDA(h, dev_alloc(&h->tok_stage, n));
-        h->tok_stage_cap = n;
-    }
-    if (n)
-        W2V_CUDA(h, cudaMemcpyAsync(h->tok_stage, tokens_host, n * sizeof(int32_t), cudaMemcpyHostToDevice, h->stream));
+    if ((rc = stage_tokens(h, tokens_host, n)) != W2V_OK) return rc;
     return cbow_step_impl(h, h->tok_stage, n, window, negatives, lr, mode, stats);
 }
 
@@ -616,19 +612,10 @@ int32_t w2v_shard_dots(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_
         return fail(h, W2V_ERR_CAPACITY, "more targets than the arrays for the partial dot products hold");
     if (pairs > 0 && h->d / 4 <= kNarrowD4) {
         // narrow slice: write the index sets once, the three passes stream over them
-        if (pairs > h->l_cap_pairs) {
-            cudaFree(h->l_centre); cudaFree(h->l_context); h->l_centre = h->l_context = nullptr; h->l_cap_pairs = 0;
-            const uint64_t cap_p = pairs + pairs / 4 + 1024;
-            W2V_CUDA(h, dev_alloc(&h->l_centre, cap_p));
-            W2V_CUDA(h, dev_alloc(&h->l_context, cap_p));
-            h->l_cap_pairs = cap_p;
-        }
-        if (pairs * negatives > h->l_cap_negs) {
-            cudaFree(h->l_negs); h->l_negs = nullptr; h->l_cap_negs = 0;
-            const uint64_t cap_n = pairs * negatives + pairs * negatives / 4 + 1024;
-            W2V_CUDA(h, dev_alloc(&h->l_negs, cap_n));
-            h->l_cap_negs = cap_n;
-        }
+        uint64_t cap_ctx = h->l_cap_pairs;                  // centre and context lists grow together
+        if ((rc = grow(h, &h->l_centre, &h->l_cap_pairs, pairs, true)) != W2V_OK) return rc;
+        if ((rc = grow(h, &h->l_context, &cap_ctx, pairs, true)) != W2V_OK) return rc;
+        if ((rc = grow(h, &h->l_negs, &h->l_cap_negs, pairs * (uint64_t)negatives, true)) != W2V_OK) return rc;
         StepParams pl = make_params(h, window, negatives, 0.f);
         if ((rc = profile_mark(h)) != W2V_OK) return rc;
         k = launch_emit_pairs(pl, h->l_centre, h->l_context, h->l_negs, pairs, h->sms * 8, h->stream);
@@ -663,28 +650,7 @@ int32_t w2v_shard_adjust(w2v_handle *h, const float *F, float lr)
     if (targets && !F) return fail(h, W2V_ERR_ARG, "F is NULL");
     DeviceGuard g(h->device);
     int32_t rc;
-    if (targets > h->G_cap) {
-        W2V_CUDA(h, cudaStreamSynchronize(h->stream));
-        cudaFree(h->G); h->G = nullptr; h->G_cap = 0;
-        const uint64_t cap = targets + targets / 4 + 1024;
-        W2V_CUDA(h, dev_alloc(&h->G, cap));
-        h->G_cap = cap;
-    }
-    const uint64_t need_du = h->sc.n_cap * (uint64_t)h->d;
-    if (need_du > h->DU_cap) {
-        W2V_CUDA(h, cudaStreamSynchronize(h->stream));
-        cudaFree(h->DU); h->DU = nullptr; h->DU_cap = 0;
-        W2V_CUDA(h, dev_alloc(&h->DU, need_du));
-        h->DU_cap = need_du;
-    }
-    const uint64_t need_dv = (uint64_t)h->hot_rows * h->d;
-    if (need_dv > h->DV_cap) {
-        W2V_CUDA(h, cudaStreamSynchronize(h->stream));
-        cudaFree(h->DV); h->DV = nullptr; h->DV_cap = 0;
-        W2V_CUDA(h, dev_alloc(&h->DV, need_dv));
-        W2V_CUDA(h, cudaMemsetAsync(h->DV, 0, need_dv * sizeof(double), h->stream));
-        h->DV_cap = need_dv;
-    }
+    if ((rc = ensure_update_scratch(h, targets, true)) != W2V_OK) return rc;
     if (targets) {
         StepParams p = make_params(h, h->pend_window, h->pend_negatives, lr);
         if ((rc = profile_mark(h)) != W2V_OK) return rc;
@@ -698,6 +664,30 @@ int32_t w2v_shard_adjust(w2v_handle *h, const float *F, float lr)
     }
     h->shard_pending = false;
     h->step_id += 1;
+    return W2V_OK;
+}
+
+int32_t w2v_peer_barrier(w2v_handle *h, uint32_t *const *flags_peers, uint32_t n_peers, uint32_t rank,
+                         uint32_t epoch, uint32_t timeout_ms)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (!flags_peers || n_peers < 1 || n_peers > (uint32_t)kMaxShards || rank >= n_peers)
+        return fail(h, W2V_ERR_ARG, "need between 1 and 16 epoch arrays and rank < n_peers");
+    if (timeout_ms < 1 || timeout_ms > 600000u) return fail(h, W2V_ERR_ARG, "timeout_ms must be in 1..600000");
+    PeerFlags flags;
+    std::memset(&flags, 0, sizeof(flags));
+    for (uint32_t r = 0; r < n_peers; ++r) {
+        if (!flags_peers[r] || (reinterpret_cast<uintptr_t>(flags_peers[r]) & 3u))
+            return fail(h, W2V_ERR_ARG, "an epoch array is NULL or not 4-byte aligned");
+        flags.p[r] = flags_peers[r];
+    }
+    flags.n = n_peers;
+    DeviceGuard g(h->device);
+    int32_t rc;
+    if ((rc = ensure_error_word(h)) != W2V_OK) return rc;
+    const int k = launch_peer_barrier(flags, rank, epoch, timeout_ms, h->tc_error, h->stream);
+    if (k < 0) return fail(h, W2V_ERR_CUDA, "barrier launch", cudaGetLastError());
+    h->launches += (uint64_t)k;
     return W2V_OK;
 }
 
@@ -750,6 +740,7 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
     if (m >= (1ull << 31)) return fail(h, W2V_ERR_ARG, "m must be below 2^31");
     if (m == 0) return W2V_OK;
     DeviceGuard g(h->device);
+    int32_t rc;
     const uint64_t nc = cand_hi - cand_lo;
     if (nc > h->inv_norm_cap) {
         W2V_CUDA(h, cudaStreamSynchronize(h->stream));
@@ -786,10 +777,7 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
         W2V_CUDA(h, dev_alloc(&h->qsplit, bytes));
         h->qsplit_cap = bytes;
     }
-    if (tc && !h->tc_error) {
-        W2V_CUDA(h, dev_alloc(&h->tc_error, 1));
-        W2V_CUDA(h, cudaMemsetAsync(h->tc_error, 0, sizeof(int), h->stream));
-    }
+    if (tc && (rc = ensure_error_word(h)) != W2V_OK) return rc;
     if (need > h->part_cap) {
         W2V_CUDA(h, cudaStreamSynchronize(h->stream));
         cudaFree(h->part_cos); cudaFree(h->part_ids); h->part_cos = nullptr; h->part_ids = nullptr; h->part_cap = 0;
@@ -798,7 +786,6 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
         h->part_cap = need;
     }
     const float *table = which ? h->V : h->U;
-    int32_t rc;
     if ((rc = profile_mark(h)) != W2V_OK) return rc;
     int k = screen ? 0 : launch_inv_norms(table, h->d, h->ld, cand_lo, nc, h->inv_norm, h->sms, h->stream);
     if (k < 0) return fail(h, W2V_ERR_CUDA, "norm launch", cudaGetLastError());
@@ -874,6 +861,9 @@ int32_t w2v_sync(w2v_handle *h)
         W2V_CUDA(h, cudaMemcpy(&flag, h->tc_error, sizeof(int), cudaMemcpyDeviceToHost));
         if (flag) {
             W2V_CUDA(h, cudaMemset(h->tc_error, 0, sizeof(int)));
+            if (flag & 2)
+                return fail(h, W2V_ERR_CUDA, "a peer barrier gave up waiting for another shard; the step that followed it "
+                                             "used incomplete dot products");
             return fail(h, W2V_ERR_CUDA, "a tensor-core retrieval block gave up waiting; its results are incomplete");
         }
     }

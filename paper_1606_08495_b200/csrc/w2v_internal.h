@@ -77,6 +77,12 @@ struct ShardPeers {
     uint32_t n;
 };
 
+// Epoch words of all shards (this one included) for the barrier of a peer-to-peer exchange.
+struct PeerFlags {
+    uint32_t *p[kMaxShards];
+    uint32_t n;
+};
+
 struct Scratch {
     uint64_t n_cap = 0;
     uint8_t *flags = nullptr;
@@ -133,6 +139,9 @@ int launch_shard_dots(const StepParams &p, const ShardPeers &peers, int sms, cud
 int launch_shard_coefficients(const float *F, float *G, unsigned long long total, uint32_t n1p, float lr,
                               int sms, cudaStream_t s);
 int launch_shard_du(const StepParams &p, int sms, cudaStream_t s);
+// one launch; a wait that runs out sets bit 1 of *error
+int launch_peer_barrier(const PeerFlags &flags, uint32_t rank, uint32_t epoch, uint32_t timeout_ms, int *error,
+                        cudaStream_t s);
 
 int launch_partial_dots(const float *U, const float *V, uint32_t vocab, uint32_t ld,
                         const int32_t *pairs, uint64_t m, uint32_t col_lo, uint32_t col_hi,

@@ -314,6 +314,49 @@ shard_adjust_v_list_kernel(StepParams p)
     }
 }
 
+// ---- barrier between the shards of a peer-to-peer exchange -----------------------------------
+// Every shard keeps an array of n epoch words (one per shard) that its peers can write.  Shard
+// `rank` announces epoch e by storing e into word `rank` of every shard's array, then waits until
+// every word of its own array has reached e.  The stores follow a system-scope fence, so the
+// additions that earlier kernels of this stream made into the peers' F arrays are visible before
+// the announcement; the waits are acquire loads, so the kernels that follow see the peers'
+// additions.  Epochs only grow, so nothing is ever reset, and a word already beyond e (a peer one
+// step ahead) also ends the wait.  The wait has a time limit: a peer that never arrives (it
+// failed on the host before its launch) makes this kernel set bit 1 of the error word and return;
+// nothing traps and the context stays usable.
+__global__ void __launch_bounds__(32)
+peer_barrier_kernel(PeerFlags flags, uint32_t rank, uint32_t epoch, unsigned long long limit_ns, int *error)
+{
+    const uint32_t r = threadIdx.x;
+    if (r >= flags.n) return;
+    __threadfence_system();
+    asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(flags.p[r] + rank), "r"(epoch) : "memory");
+    unsigned long long t0;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    const uint32_t *mine = flags.p[rank] + r;
+    for (uint32_t polls = 1;; ++polls) {
+        uint32_t seen;
+        asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(seen) : "l"(mine) : "memory");
+        if ((int32_t)(seen - epoch) >= 0) break;
+        if ((polls & 63u) == 0) {
+            unsigned long long now;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+            if (now - t0 > limit_ns || polls > (1u << 30)) {
+                atomicOr(error, 2);
+                break;
+            }
+        }
+        __nanosleep(200);
+    }
+}
+
+int launch_peer_barrier(const PeerFlags &flags, uint32_t rank, uint32_t epoch, uint32_t timeout_ms, int *error,
+                        cudaStream_t s)
+{
+    peer_barrier_kernel<<<1, 32, 0, s>>>(flags, rank, epoch, (unsigned long long)timeout_ms * 1000000ull, error);
+    return cudaGetLastError() != cudaSuccess ? -1 : 1;
+}
+
 // ---- launchers --------------------------------------------------------------------------------
 template <typename K>
 static int shard_grid(K kernel, int sms)

@@ -15,7 +15,8 @@ LocalShards       all shards in one process on one GPU: each shard's kernel adds
 DistributedShard  one shard per rank of a torch.distributed group (one process per GPU).
                   exchange="allreduce": partials into a local array, then one NCCL all-reduce.
                   exchange="p2p": the arrays live in symmetric memory and the dots kernel adds
-                  into every peer's array directly over NVLink; one device barrier per step.
+                  into every peer's array directly over NVLink; one time-limited device barrier
+                  (w2v_peer_barrier) per step.
 """
 from __future__ import annotations
 
@@ -135,7 +136,10 @@ class DistributedShard:
     """
 
     def __init__(self, vocab, d, seed, device, group=None, exchange="allreduce", aligned_rows=True,
-                 max_tokens=1 << 20, window=5, negatives=5):
+                 max_tokens=1 << 20, window=5, negatives=5, barrier_timeout_ms=5000):
+        """barrier_timeout_ms (exchange="p2p"): how long a rank's barrier kernel waits for the other
+        ranks before it gives up; the next sync() of that rank then raises, and no GPU hangs on a
+        rank that failed."""
         import torch.distributed as dist
 
         if exchange not in ("allreduce", "p2p"):
@@ -158,10 +162,13 @@ class DistributedShard:
             # barrier per step orders both "all partials added" and "array of step k-2 zeroed"
             import torch.distributed._symmetric_memory as symm_mem
 
-            self.buf = symm_mem.empty(2 * self.cap, dtype=torch.float32, device=self.device)
+            # and, behind them, one epoch word per rank for the library's time-limited barrier
+            self.barrier_timeout_ms = int(barrier_timeout_ms)
+            self.buf = symm_mem.empty(2 * self.cap + binding.MAX_SHARDS, dtype=torch.float32, device=self.device)
             self.buf.zero_()
             self.symm = symm_mem.rendezvous(self.buf, group if group is not None else dist.group.WORLD)
             self.peer_ptrs = [int(p) for p in self.symm.buffer_ptrs]
+            self.flag_ptrs = [p + 4 * 2 * self.cap for p in self.peer_ptrs]
             torch.cuda.synchronize(self.device)
             dist.barrier(group)
 
@@ -188,12 +195,23 @@ class DistributedShard:
             half = (self.steps & 1) * self.cap
             peers = [p + 4 * half for p in self.peer_ptrs]
             binding.w2v_shard_dots(m.h, t, n, window, negatives, peers, self.cap, st)
-            self.symm.barrier()                                   # every rank's additions have landed
+            # every rank's additions have landed once every rank has announced this step
+            binding.w2v_peer_barrier(m.h, self.flag_ptrs, self.rank, self.steps + 1, self.barrier_timeout_ms)
             mine = self.buf[half: half + self.cap]
             binding.w2v_shard_adjust(m.h, mine, lr)
             mine.zero_()                                          # ready for step k + 2
         self.steps += 1
         return st.as_dict()
+
+    def set_step(self, s):
+        self.model.set_step(s)
+
+    def set_interleave(self, phase, stride):
+        self.model.set_interleave(phase, stride)
+
+    def sync(self):
+        """Waits for this rank's stream; raises if one of its barriers gave up waiting for a peer."""
+        self.model.sync()
 
     def read_rows(self, which, ids):
         """This rank's columns of the rows."""

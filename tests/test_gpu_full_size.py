@@ -195,3 +195,50 @@ def test_large_snapshot_step_on_sampled_rows(large):
           "row-relative error U %.2e V %.2e" % (len(cm), len(c), len(S_u), len(S_v), cnt_v.max(), eu, ev))
     assert eu <= SNAPSHOT_TOL and ev <= SNAPSHOT_TOL, (eu, ev)
     assert row_rel_err(gpu.read_rows(1, [hot]), cpu.read_rows(1, [hot])) <= SNAPSHOT_TOL
+
+
+def test_large_hogwild_step_from_nonzero_rows(large):
+    # A Hogwild step at full size whose dot products are far from zero, judged by the acceptance rule
+    # of that mode: the loss of the pairs of sampled centre words after the step, evaluated by the
+    # checker on the vectors read back, against the sequential checker's.  The sampled centres and
+    # all their target rows start from seeded vectors of ordinary trained size on both sides; every
+    # other input row is still of initial size (|u| ~ 0.03), so what the rest of the chunk adds to
+    # the shared target rows moves these pairs' dot products by ~1e-3 while their own updates move
+    # them by ~0.1: the checker can run the sampled centres' pairs alone.
+    cfg, gpu, cpu, cp = large["cfg"], large["gpu"], large["cpu"], large["cp"]
+    W, N, lr, d = cfg["window"], cfg["negatives"], cfg["lr"], cfg["d"]
+    toks = cp.chunk(1)
+    step = gpu.get_step() + 5
+    gpu.set_step(step); cpu.set_step(step)
+    c, x, n = cpu.sample_pairs(toks, W, N)
+    rng = np.random.default_rng(6)
+    run_start = np.ones(len(c), dtype=bool)
+    run_start[1:] = c[1:] != c[:-1]
+    cw, runs = np.unique(c[run_start], return_counts=True)
+    S_u = rng.choice(cw[runs == 1], 400, replace=False)              # centre words that occur once in the chunk
+    mask = np.isin(c, S_u)
+    cm, xm, nm = c[mask], x[mask], n[mask]
+    assert len(cm) > 1500
+    R_v = np.unique(np.concatenate([xm, nm.ravel()]))
+    Uv = rng.normal(scale=0.05, size=(len(S_u), d)).astype(np.float32)
+    Vv = rng.normal(scale=0.15, size=(len(R_v), d)).astype(np.float32)
+    S_u = np.sort(S_u)
+    for m in (gpu, cpu):
+        m.write_rows(0, S_u, Uv)
+        m.write_rows(1, R_v, Vv)
+    before = cpu.loss_pairs(cm, xm, nm) / len(cm)
+    st = gpu.sgns_step(toks, W, N, lr, binding.MODE_HOGWILD)
+    assert st["pairs"] == len(c)
+    cpu.step_pairs(cm, xm, nm, lr, 1)
+    want = cpu.loss_pairs(cm, xm, nm) / len(cm)
+    ev = Oracle(cfg["vocab"], d, SEED, sparse=True)
+    ev.write_rows(0, S_u, gpu.read_rows(0, S_u))
+    ev.write_rows(1, R_v, gpu.read_rows(1, R_v))
+    got = ev.loss_pairs(cm, xm, nm) / len(cm)
+    eu = row_rel_err(gpu.read_rows(0, S_u), cpu.read_rows(0, S_u))
+    ev.close()
+    print("full-size hogwild step from non-zero rows: %d pairs of %d centres, loss per pair %.6f -> checker %.6f, "
+          "gpu %.6f; worst centre row differs by %.2e" % (len(cm), len(S_u), before, want, got, eu))
+    assert before - want > 0.01 * before                  # the step moved the loss by more than the tolerance
+    assert abs(got - want) <= 0.01 * want
+    assert abs((before - got) - (before - want)) <= 0.05 * (before - want)
