@@ -30,11 +30,11 @@ from paper_1606_08495_b200 import corpus  # noqa: E402
 METRIC = "sgns_positive_pairs_per_sec"
 UNIT = "pairs/s"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes moved per algorithmic byte by the Hogwild update kernel on the large workload, from
-# the one-pass ncu capture summarised in profiles/sgns_update_kernels_large.md
-# ((dram__bytes_read.sum + dram__bytes_write.sum) / model bytes of the captured launch: 126.42 / 121.9 GB,
-# rows on 128-byte boundaries).  Applies to the large workload in Hogwild mode with the default row
-# stride and launch shape only; anything else reports null.
+# DRAM bytes moved per algorithmic byte by the Hogwild update kernel on the large workload, from one
+# one-pass ncu capture of that kernel ((dram__bytes_read.sum + dram__bytes_write.sum) / model bytes of the
+# captured launch: 126.42 / 121.9 GB, rows on 128-byte boundaries).  It is a constant taken once, not a
+# counter read during this run (the JSON line says so in "traffic_kind"), and applies to the large workload
+# in Hogwild mode with the default row stride and launch shape only; anything else reports null.
 TRAFFIC_PER_ALGORITHMIC_BYTE = 1.037
 
 
@@ -209,6 +209,128 @@ def reduce_over_ranks(ms, e2e_ms, pairs, e2e_pairs, launches, world, device):
     return float(mx[0]), float(mx[1]), float(sm[2]), float(sm[3]), int(sm[4])
 
 
+def measured_tensor_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured sustained bf16"
+    except Exception:
+        return 1400.0, "fallback sustained bf16"
+
+
+def fill_clustered(table, rows, d, lo, hi, seed, cluster_size=50, noise=0.55, loose=0.2):
+    """Writes the recipe of corpus.clustered_rows into rows [lo, hi) of a device table (torch's
+    generator on the device instead of numpy's: same distribution, other numbers).  Input data."""
+    import torch
+
+    dev = table.device
+    g = torch.Generator(device=dev); g.manual_seed(seed)
+    view = table.view(rows, -1)
+    n_clusters = max(1, (hi - lo) // cluster_size)
+    centres = torch.randn(n_clusters, d, generator=g, device=dev)
+    for a in range(lo, hi, 1 << 20):
+        b = min(hi, a + (1 << 20))
+        which = torch.randint(0, n_clusters, (b - a,), generator=g, device=dev)
+        is_loose = torch.rand(b - a, generator=g, device=dev) < loose
+        x = noise * torch.randn(b - a, d, generator=g, device=dev)
+        x += torch.where(is_loose[:, None], torch.zeros((), device=dev), centres[which])
+        x[is_loose] *= 1.0 / noise
+        view[a:b, :d] = x
+
+
+def secondary_modes(model, cfg, dev_chunks, first_step, dev, steps=10, warmup=3):
+    """The other modes on the model the headline run leaves in memory: snapshot-mode SGNS steps, CBOW
+    Hogwild steps, and one retrieval call over the model's last 3 M rows (overwritten with clustered
+    stand-in vectors first, so this runs last).  Each entry: CUDA-event ms per step, the update (or
+    retrieval) kernels' time from the library's own events, algorithmic bytes or flops over that time,
+    and the fraction of the measured peak."""
+    import torch
+
+    from paper_1606_08495_b200 import binding
+
+    W, N, lr, d = cfg["window"], cfg["negatives"], cfg["lr"], cfg["d"]
+    peak, peak_kind = measured_peak()
+    out = {}
+    n_chunks = min(len(dev_chunks), warmup + steps)
+
+    def timed(step_fn, sample_fn, bytes_fn, label):
+        counts = []
+        for i in range(warmup, n_chunks):
+            model.set_step(first_step + i)
+            st = binding.StepStats()
+            sample_fn(dev_chunks[i], st)
+            counts.append((st.centres, st.pairs))
+        model.set_step(first_step)
+        for i in range(warmup):
+            step_fn(dev_chunks[i])
+        model.sync()
+        binding.w2v_profile_enable(model.h, True)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(dev)
+        ev0.record()
+        for i in range(warmup, n_chunks):
+            step_fn(dev_chunks[i])
+        ev1.record()
+        torch.cuda.synchronize(dev)
+        ms = ev0.elapsed_time(ev1)
+        kernel_ms, _ = binding.w2v_profile_read(model.h)
+        binding.w2v_profile_enable(model.h, False)
+        k = n_chunks - warmup
+        pairs = float(sum(p for _, p in counts))
+        nbytes = float(sum(bytes_fn(c, p) for c, p in counts))
+        achieved = nbytes / (kernel_ms * 1e-3) / 1e9 if kernel_ms > 0 else 0.0
+        out[label] = {"value": pairs / (ms * 1e-3), "unit": UNIT, "steps": k, "ms_per_step": ms / k,
+                      "kernel_ms_per_step": kernel_ms / k, "bound": "hbm", "achieved": achieved, "peak": peak,
+                      "roofline_unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}"}
+
+    timed(lambda t: binding.w2v_sgns_step(model.h, t, t.numel(), W, N, lr, binding.MODE_SNAPSHOT, None),
+          lambda t, st: binding.w2v_sample_pairs(model.h, t, t.numel(), W, N, None, None, None, 0, st,
+                                                 allow=(binding.W2V_ERR_CAPACITY,)),
+          lambda c, p: algorithmic_bytes_snapshot(d, c, p, N), "sgns_snapshot")
+    timed(lambda t: binding.w2v_cbow_step(model.h, t, t.numel(), W, N, lr, binding.MODE_HOGWILD, None),
+          lambda t, st: binding.w2v_sample_cbow(model.h, t, t.numel(), W, N, None, None, 0, st,
+                                                allow=(binding.W2V_ERR_CAPACITY,)),
+          lambda c, p: algorithmic_bytes_cbow(d, c, p, N), "cbow_hogwild")
+    out["cbow_hogwild"]["note"] = "pairs = (centre, context) pairs, i.e. context rows read"
+
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    if free_b > (5 << 30):
+        V = cfg["vocab"]
+        lo, hi, m, K = V - 3_000_000, V, 8192, 30
+        fill_clustered(model.U, V, d, lo, hi, seed=5)
+        g = torch.Generator(device=dev); g.manual_seed(6)
+        q = torch.randint(lo, hi, (m,), generator=g, device=dev, dtype=torch.int64)
+        ids = torch.empty(m * K, dtype=torch.int64, device=dev)
+        cs = torch.empty(m * K, dtype=torch.float32, device=dev)
+        tpeak, tkind = measured_tensor_peak()
+        for tau, label in ((0.65, "topk_cosine_tau_0.65"), (-2.0, "topk_cosine_top30")):
+            for _ in range(2):
+                binding.w2v_topk_cosine(model.h, 0, q, m, lo, hi, K, tau, ids, cs)
+            model.sync()
+            binding.w2v_profile_enable(model.h, True)
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize(dev)
+            ev0.record()
+            calls = 5
+            for _ in range(calls):
+                binding.w2v_topk_cosine(model.h, 0, q, m, lo, hi, K, tau, ids, cs)
+            ev1.record()
+            torch.cuda.synchronize(dev)
+            model.sync()
+            ms = ev0.elapsed_time(ev1)
+            kernel_ms, _ = binding.w2v_profile_read(model.h)
+            binding.w2v_profile_enable(model.h, False)
+            cosines = float(m) * (hi - lo) * calls
+            achieved = 2.0 * d * cosines / (kernel_ms * 1e-3) / 1e12 if kernel_ms > 0 else 0.0
+            out[label] = {"value": cosines / (ms * 1e-3), "unit": "cosines/s", "steps": calls, "ms_per_step": ms / calls,
+                          "kernel_ms_per_step": kernel_ms / calls, "bound": "tensor", "achieved": achieved,
+                          "peak": tpeak, "roofline_unit": "TFLOP/s", "frac": achieved / tpeak,
+                          "peak_kind": f"of {tkind}",
+                          "config": {"queries": m, "candidates": hi - lo, "K": K, "tau": tau,
+                                     "rows": "clustered stand-in vectors (cluster centre + noise), lists fill",
+                                     "lists_full": float(((ids.view(m, K) >= 0).sum(dim=1) == K).float().mean())}}
+    return out
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -325,6 +447,13 @@ def run_gpu(args):
     ms, e2e_ms, all_pairs, all_e2e_pairs, all_launches = reduce_over_ranks(
         ms, e2e_ms, tot_pairs, float(e2e_pairs), launches, world, dev)
 
+    default_shape = (name == "large" and args.mode == "hogwild" and not cbow and not args.row_stride
+                     and not args.rows_in_flight and not args.blocks_per_sm and not args.dense_rows
+                     and not args.tokens_per_step and IL == 1)
+    secondary = None
+    if world == 1 and default_shape and not args.no_secondary:
+        secondary = secondary_modes(model, cfg, dev_chunks, Wu + 2 * K, dev)
+
     if rank == 0:
         peak, peak_kind = measured_peak()
         achieved = tot_bytes / (kernel_ms * 1e-3) / 1e9 if kernel_ms > 0 else 0.0
@@ -353,10 +482,12 @@ def run_gpu(args):
                          "frac_of_8TBps": achieved / 8000.0,
                          "algorithmic_bytes_per_launch": per_launch_bytes,
                          "kernel_ms_per_launch": kernel_ms / max(1, groups),
-                         "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE * per_launch_bytes
-                                     if name == "large" and args.mode == "hogwild" and not cbow and not args.row_stride
-                                     and not args.rows_in_flight and not args.blocks_per_sm else None)},
+                         "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE * per_launch_bytes if default_shape else None),
+                         "traffic_kind": ("scaled from one ncu capture of this kernel and workload, not measured in this run"
+                                          if default_shape else None)},
         }
+        if secondary is not None:
+            line["secondary"] = secondary
         if world == 1 and not args.no_cpu_baseline:
             words = args.cpu_words
             p, s, store = time_oracle(cfg, cp, words, 1, 0)
@@ -477,13 +608,17 @@ def run_topk(args):
     model = binding.W2V(V, d, seed=1, device=dev, row_stride=row_stride_for(d, args.row_stride))
     tensor = args.retrieval_kernel != "fp32"
     binding.w2v_set_retrieval_kernel(model.h, {"fp32": 0, "tensor": 1, "screen": 2}[args.retrieval_kernel])
-    # spread-out vectors instead of the tiny uniform initial ones: normal rows, so that cosines have the
-    # spread of unrelated trained vectors (about N(0, 1/d)); written by torch, this is input data
+    # stand-in for trained vectors: clustered rows (centre + noise), so that queries have neighbours above
+    # tau and the lists fill; --unrelated-rows keeps the earlier i.i.d. normal rows (nothing reaches tau = 0.65:
+    # pure screening).  Written by torch: this is input data.
     g = torch.Generator(device=dev); g.manual_seed(5)
-    Uv = model.U.view(V, model.row_stride)
-    for a in range(0, V, 1 << 20):
-        b = min(V, a + (1 << 20))
-        Uv[a:b, :d] = torch.randn(b - a, d, generator=g, device=dev)
+    if args.unrelated_rows:
+        Uv = model.U.view(V, model.row_stride)
+        for a in range(0, V, 1 << 20):
+            b = min(V, a + (1 << 20))
+            Uv[a:b, :d] = torch.randn(b - a, d, generator=g, device=dev)
+    else:
+        fill_clustered(model.U, V, d, 0, V, seed=5)
     q = torch.randint(0, V, (m,), generator=g, device=dev, dtype=torch.int64)
     ids = torch.empty(m * K, dtype=torch.int64, device=dev)
     cs = torch.empty(m * K, dtype=torch.float32, device=dev)
@@ -551,6 +686,8 @@ def run_topk(args):
                    "kernel": {"tensor": "tcgen05 tf32, head/tail split (3 MMAs per product)",
                               "screen": "tcgen05 bf16 screen (1 MMA per product) + exact fp32 cosines near the cut",
                               "fp32": "fp32 CUDA cores"}[args.retrieval_kernel],
+                   "rows": "i.i.d. normal (no neighbours)" if args.unrelated_rows else "clustered (centre + noise): lists fill",
+                   "lists_full": float(((ids.view(m, K) >= 0).sum(dim=1) == K).float().mean()),
                    "l2": "3 M candidate rows (3.8 GB) streamed per call, far larger than L2"},
         "clocks": clocks,
         "e2e": {"value": cosines / (e2e_ms * 1e-3), "unit": "cosines/s", "h2d_bytes_per_step": 8 * m,
@@ -598,6 +735,10 @@ def main():
                     help="visit every chunk this many times, each time with 1/this of its input words "
                          "(interleaved minibatch formation)")
     ap.add_argument("--dense-rows", action="store_true", help="no padding between table rows")
+    ap.add_argument("--no-secondary", action="store_true",
+                    help="default run only: skip the snapshot / CBOW / retrieval measurements that follow the headline")
+    ap.add_argument("--unrelated-rows", action="store_true",
+                    help="--mode topk: i.i.d. normal rows (no neighbours above tau) instead of clustered ones")
     ap.add_argument("--exchange", choices=["p2p", "allreduce"], default="p2p",
                     help="--mode sharded: partial dots added into every shard's array by the producing kernel, "
                          "or stored per shard and summed afterwards")

@@ -108,3 +108,26 @@ class Corpus:
         mask[ends] = False
         out[mask] = toks
         return out
+
+
+def clustered_rows(n: int, d: int, seed: int, cluster_size: int = 50, noise: float = 0.55,
+                   loose: float = 0.2) -> np.ndarray:
+    """Stand-in for trained vectors as the retrieval stage sees them (Section 7.2): fp32 rows
+    [n, d] that have neighbours.  A row is a cluster centre plus `noise` times a standard normal
+    vector (cosine between two rows of a cluster about 1 / (1 + noise^2), 0.77 for 0.55, above the
+    paper's threshold of 0.65; rows of different clusters are nearly orthogonal); clusters have
+    `cluster_size` rows on average; a share `loose` of the rows is plain noise and has no neighbour.
+    Inputs only: written into a table by the caller."""
+    rng = np.random.default_rng([int(seed), 7])
+    n_clusters = max(1, n // cluster_size)
+    centres = rng.standard_normal((n_clusters, d), dtype=np.float32)
+    out = np.empty((n, d), dtype=np.float32)
+    for a in range(0, n, 1 << 18):
+        b = min(n, a + (1 << 18))
+        which = rng.integers(0, n_clusters, b - a)
+        is_loose = rng.random(b - a) < loose
+        rows = noise * rng.standard_normal((b - a, d), dtype=np.float32)
+        rows += np.where(is_loose[:, None], np.float32(0), centres[which])
+        rows[is_loose] *= np.float32(1.0 / noise)
+        out[a:b] = rows
+    return out

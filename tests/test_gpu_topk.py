@@ -37,12 +37,15 @@ def pair(V, d, seed, which=0, scale=1.0, row_stride=None, rows=None, kernel=0):
     return gpu, cpu, X
 
 
-def check(gpu, cpu, X, which, queries, lo, hi, K, tau, TOL=TOL):
-    gi, gc = gpu.topk_cosine(which, queries, lo, hi, K, tau)
-    wi, wc = cpu.topk_cosine(which, queries, lo, hi, K, tau)
+def compare(gi, gc, wi, wc, X, queries, lo, hi, K, tau, TOL=TOL):
+    """GPU lists (gi, gc) against the checker's (wi, wc) for the same queries; X holds the table rows."""
     assert gi.shape == wi.shape
-    Xd = X.astype(np.float64)
-    nrm = np.linalg.norm(Xd, axis=1)
+
+    def exact(q, a):                                       # fp64 cosine of rows q and a
+        x, y = X[q].astype(np.float64), X[a].astype(np.float64)
+        nx, ny = np.linalg.norm(x), np.linalg.norm(y)
+        return float(x @ y / (nx * ny)) if nx > 0 and ny > 0 else 0.0
+
     for r, q in enumerate(np.asarray(queries)):
         n_want = int((wi[r] >= 0).sum())
         n_got = int((gi[r] >= 0).sum())
@@ -56,10 +59,15 @@ def check(gpu, cpu, X, which, queries, lo, hi, K, tau, TOL=TOL):
             assert abs(gc[r, s] - wc[r, s]) <= TOL, (r, s, gc[r, s], wc[r, s])
             if gi[r, s] != wi[r, s]:
                 a = gi[r, s]
-                exact = Xd[q] @ Xd[a] / (nrm[q] * nrm[a]) if nrm[q] > 0 and nrm[a] > 0 else 0.0
-                assert abs(exact - wc[r, s]) <= TOL and lo <= a < hi and a != q, (r, s)
+                assert abs(exact(q, a) - wc[r, s]) <= TOL and lo <= a < hi and a != q, (r, s)
         assert np.all(gi[r, n_got:] == -1) and not gc[r, n_got:].any()
         assert len(set(gi[r, :n_got].tolist())) == n_got
+
+
+def check(gpu, cpu, X, which, queries, lo, hi, K, tau, TOL=TOL):
+    gi, gc = gpu.topk_cosine(which, queries, lo, hi, K, tau)
+    wi, wc = cpu.topk_cosine(which, queries, lo, hi, K, tau)
+    compare(gi, gc, wi, wc, X, queries, lo, hi, K, tau, TOL)
     return gi, gc
 
 

@@ -1,0 +1,59 @@
+"""Cosine retrieval at the shape the benchmark times (Section 7.2: K = 30, kept above tau = 0.65):
+8192 queries against 3 M candidate rows of 300 columns, rows on 128-byte boundaries, so that the
+default kernel runs with the benchmark's 64 query blocks x 9 candidate splits and the sharing of
+the best K-th cosine across splits.  The CPU checker's brute force (fp64) covers a sample of the
+queries; all three kernels are compared on that sample, the default kernel on the full call.
+
+The rows are clustered (cluster centre + noise) so that most queries have a few dozen neighbours
+above tau and the lists fill; a fifth of the rows are plain noise and have none."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import Oracle
+from paper_1606_08495_b200 import binding, corpus
+from test_gpu_topk import compare, tolerance
+
+pytestmark = pytest.mark.gpu
+
+V, D, K = 3_100_000, 300, 30
+LO, HI = 100_000, V                      # 3.0 M candidates, as many as the benchmark's call
+M, SAMPLE = 8192, 40
+
+
+def test_retrieval_at_the_benchmarked_shape():
+    need = 2 * V * 320 * 4 + (8 << 30)
+    torch.cuda.empty_cache()
+    free_b, _ = torch.cuda.mem_get_info()
+    if free_b < need:
+        pytest.skip("not enough free device memory")
+    rng = np.random.default_rng(77)
+    X = corpus.clustered_rows(V, D, seed=77)
+    gpu = binding.W2V(V, D, 1, row_stride=binding.aligned_row_stride(D))
+    cpu = Oracle(V, D, 1)
+    for a in range(0, V, 200_000):
+        ids = np.arange(a, min(V, a + 200_000))
+        gpu.write_rows(0, ids, X[ids]); cpu.write_rows(0, ids, X[ids])
+    q = rng.integers(0, V, M)
+    pick = np.sort(rng.choice(M, SAMPLE, replace=False))
+    kept = {}
+    for tau in (0.65, -2.0):
+        wi, wc = cpu.topk_cosine(0, q[pick], LO, HI, K, tau)
+        binding.w2v_set_retrieval_kernel(gpu.h, 2)                  # the default: bf16 screen + exact fp32
+        gi, gc = gpu.topk_cosine(0, q, LO, HI, K, tau)              # the benchmark's call
+        compare(gi[pick], gc[pick], wi, wc, X, q[pick], LO, HI, K, tau, tolerance(2, D))
+        n = (gi >= 0).sum(axis=1)
+        kept[tau] = n
+        # properties of every list of the full call: sorted, distinct, inside the range, above tau
+        assert (np.diff(gc, axis=1)[(gi[:, 1:] >= 0)] <= 0).all()
+        assert ((gi < 0) | ((gi >= LO) & (gi < HI) & (gi != q[:, None]))).all()
+        assert (gc[gi >= 0] > tau - 2e-6).all()
+        for kernel in (0, 1):                                       # the other two kernels on the sample
+            binding.w2v_set_retrieval_kernel(gpu.h, kernel)
+            si, sc = gpu.topk_cosine(0, q[pick], LO, HI, K, tau)
+            compare(si, sc, wi, wc, X, q[pick], LO, HI, K, tau, tolerance(kernel, D))
+    # the data does what it was made for: most lists fill at tau = 0.65, some stay empty
+    assert (kept[0.65] == K).mean() > 0.5 and (kept[0.65] == 0).mean() > 0.05
+    assert (kept[-2.0] == K).all()
+    gpu.close()
+    cpu.close()
