@@ -704,6 +704,48 @@ def run_topk(args):
     model.close()
 
 
+def run_probe(args):
+    """Memory-system ceilings for the step's access patterns (w2v_probe_rows) on the output table of
+    the chosen workload's model: each pattern with row numbers spread over the whole table and over
+    the first `--probe-span` rows only (the table is the same; only the address range differs)."""
+    import torch
+
+    from paper_1606_08495_b200 import binding
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    name = pick_workload(args.workload, free_b, args.row_stride)
+    cfg = corpus.CONFIGS[name]
+    cp = corpus.Corpus(cfg)
+    d = cfg["d"]
+    row_stride = d if args.dense_rows else row_stride_for(d, args.row_stride)
+    model = binding.W2V(cfg["vocab"], d, seed=1, device=dev, row_stride=row_stride)
+    model.build_alias(cp.counts, cfg["subsample_t"])
+    peak, peak_kind = measured_peak()
+    names = ["gather", "gather_red", "gather_alias", "gather_red_alias", "touch_red"]
+    rows = args.probe_rows
+    spans = sorted({cfg["vocab"], min(cfg["vocab"], args.probe_span)}, reverse=True)
+    result = {}
+    for span in spans:
+        per = {}
+        for access, label in enumerate(names):
+            best = None
+            for _ in range(1 + max(1, args.steps // 10)):          # first launch is the warm-up
+                ms, done = binding.w2v_probe_rows(model.h, access, span, rows)
+                best = ms if best is None or ms < best else best
+            moved = done * 4.0 * d * (2.0 if "red" in label else 1.0)
+            per[label] = {"ms": best, "row_GBps": moved / (best * 1e-3) / 1e9, "frac_of_copy_peak": moved / (best * 1e-3) / 1e9 / peak}
+        result[f"span_{span}_rows"] = per
+    line = {"metric": "random_row_traffic", "unit": "GB/s of row bytes (read + written)", "n_gpus": 1,
+            "config": {"workload": name + " (memory-system probe)", "vocab": cfg["vocab"], "d": d,
+                       "row_stride_floats": row_stride, "rows_per_launch": rows,
+                       "table_GB": cfg["vocab"] * row_stride * 4 / 1e9},
+            "peak": peak, "peak_kind": f"of {peak_kind}", "probe": result}
+    print(json.dumps(line), flush=True)
+    model.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -722,7 +764,10 @@ def main():
     ap.add_argument("--queries", type=int, default=8192, help="query rows per call of --mode topk")
     ap.add_argument("--retrieval-kernel", choices=["fp32", "tensor", "screen"], default="screen")
     ap.add_argument("--tau", type=float, default=0.65, help="similarity threshold of --mode topk (-2 keeps everything)")
-    ap.add_argument("--mode", choices=["hogwild", "snapshot", "sharded", "topk"], default="hogwild",
+    ap.add_argument("--probe-rows", type=int, default=20_000_000, help="--mode probe: rows touched per launch")
+    ap.add_argument("--probe-span", type=int, default=18_000_000,
+                    help="--mode probe: the second measurement draws its rows from the first this-many rows only")
+    ap.add_argument("--mode", choices=["hogwild", "snapshot", "sharded", "topk", "probe"], default="hogwild",
                     help="update mode of the timed steps (the headline number is hogwild); sharded = the "
                          "paper's column partition, --shards slices of one model on one GPU")
     ap.add_argument("--tokens-per-step", type=int, default=0,
@@ -751,6 +796,8 @@ def main():
         run_sharded(args)
     elif args.mode == "topk":
         run_topk(args)
+    elif args.mode == "probe":
+        run_probe(args)
     else:
         run_gpu(args)
 

@@ -392,6 +392,30 @@ int32_t w2v_profile_read(w2v_handle *h, double *kernel_ms, uint64_t *launches);
 int32_t w2v_get_launch_count(w2v_handle *h, uint64_t *launches);
 
 /*
+ * Memory-system ceiling for the step's access patterns (no counterpart in the paper: a measuring
+ * aid; Section 6 of the paper names the random cache-line rate as what bounds a shard).  Touches
+ * `rows` pseudo-random rows of the output table V, drawn uniformly from rows [0, span_rows), with
+ * the step kernels' own row layout, 16-byte loads, vector reductions and rows in flight per warp,
+ * but without sampling or arithmetic.  Additions add +0.0f: the table keeps its values.
+ *   access   W2V_PROBE_GATHER            read each row (what snapshot pass 1 does per target)
+ *            W2V_PROBE_GATHER_RED        read each row, then add to it (the Hogwild update)
+ *            W2V_PROBE_GATHER_ALIAS      GATHER plus one random 8-byte read of the alias table
+ *            W2V_PROBE_GATHER_RED_ALIAS  GATHER_RED plus that read (a negative draw per row)
+ *            W2V_PROBE_TOUCH_RED         one word per 64-byte burst, wait, then add (snapshot pass 2)
+ *   ms, rows_done  host; receive the kernel's duration (CUDA events on the handle's stream) and
+ *            the number of rows it touched (rows rounded up to whole rounds of its launch shape).
+ * Synchronises the stream.  Errors: W2V_ERR_ARG (unknown access, span_rows outside 1..vocab,
+ * rows outside 1..2^32, d > 512), W2V_ERR_STATE (an ALIAS pattern before w2v_build_alias).
+ */
+#define W2V_PROBE_GATHER 0u
+#define W2V_PROBE_GATHER_RED 1u
+#define W2V_PROBE_GATHER_ALIAS 2u
+#define W2V_PROBE_GATHER_RED_ALIAS 3u
+#define W2V_PROBE_TOUCH_RED 4u
+int32_t w2v_probe_rows(w2v_handle *h, uint32_t access, uint64_t span_rows, uint64_t rows, double *ms,
+                       uint64_t *rows_done);
+
+/*
  * Launch shape of the update kernels: rows in flight per warp (1..8; 0 = default)
  * and resident thread blocks per SM (0 = as many as fit).  Results do not depend
  * on it in snapshot mode.

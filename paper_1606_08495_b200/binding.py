@@ -27,7 +27,7 @@ EXPORTS = (
     "w2v_sgns_step_host", "w2v_sample_pairs", "w2v_partial_dots", "w2v_read_rows", "w2v_write_rows",
     "w2v_set_step", "w2v_get_step", "w2v_get_table_ptrs", "w2v_sync", "w2v_profile_enable",
     "w2v_profile_read", "w2v_get_launch_count", "w2v_set_tuning", "w2v_last_error",
-    "w2v_sample_pairs_noalloc", "w2v_peer_barrier",
+    "w2v_sample_pairs_noalloc", "w2v_peer_barrier", "w2v_probe_rows",
 )
 
 
@@ -73,6 +73,7 @@ def load():
         "w2v_shard_dots": [vp, vp, u64, u32, u32, C.POINTER(vp), u32, u64, C.POINTER(StepStats)],
         "w2v_shard_adjust": [vp, vp, C.c_float],
         "w2v_peer_barrier": [vp, C.POINTER(vp), u32, u32, u32, u32],
+        "w2v_probe_rows": [vp, u32, u64, u64, C.POINTER(C.c_double), C.POINTER(u64)],
         "w2v_destroy": [vp],
         "w2v_build_alias": [vp, vp, C.c_double],
         "w2v_get_tables": [vp, vp, vp, vp],
@@ -169,6 +170,16 @@ def w2v_peer_barrier(h, flags_peers, rank, epoch, timeout_ms):
     """flags_peers: device pointers (ints or tensors), one array of len(flags_peers) uint32 per shard."""
     ptrs = (C.c_void_p * len(flags_peers))(*[_ptr(f) for f in flags_peers])
     return _check(h, load().w2v_peer_barrier(h, ptrs, len(flags_peers), int(rank), int(epoch), int(timeout_ms)))
+
+
+PROBE_GATHER, PROBE_GATHER_RED, PROBE_GATHER_ALIAS, PROBE_GATHER_RED_ALIAS, PROBE_TOUCH_RED = range(5)
+
+
+def w2v_probe_rows(h, access, span_rows, rows):
+    """(milliseconds, rows touched) of one probe launch."""
+    ms, done = C.c_double(0.0), C.c_uint64(0)
+    _check(h, load().w2v_probe_rows(h, int(access), int(span_rows), int(rows), C.byref(ms), C.byref(done)))
+    return ms.value, int(done.value)
 
 
 def w2v_get_row_stride(h):

@@ -12,7 +12,7 @@ ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libw2v.so")
 BUILD = os.path.join(HERE, "_build")
 
-CU_SOURCES = ["w2v_api.cu", "w2v_sampling.cu", "w2v_sgns.cu", "w2v_rows.cu", "w2v_shard.cu", "w2v_cbow.cu", "w2v_topk.cu", "w2v_topk_tc.cu"]
+CU_SOURCES = ["w2v_api.cu", "w2v_sampling.cu", "w2v_sgns.cu", "w2v_rows.cu", "w2v_shard.cu", "w2v_cbow.cu", "w2v_topk.cu", "w2v_topk_tc.cu", "w2v_probe.cu"]
 CPP_SOURCES = ["w2v_tables.cpp"]
 HEADERS = ["w2v_device.cuh", "w2v_internal.h", "w2v_sample.cuh"]
 

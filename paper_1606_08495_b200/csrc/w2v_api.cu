@@ -812,6 +812,41 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
     return W2V_OK;
 }
 
+int32_t w2v_probe_rows(w2v_handle *h, uint32_t access, uint64_t span_rows, uint64_t rows, double *ms,
+                       uint64_t *rows_done)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (access > W2V_PROBE_TOUCH_RED) return fail(h, W2V_ERR_ARG, "unknown access pattern");
+    if (!ms || !rows_done) return fail(h, W2V_ERR_ARG, "ms or rows_done is NULL");
+    if (span_rows < 1 || span_rows > h->vocab) return fail(h, W2V_ERR_ARG, "need 1 <= span_rows <= vocab");
+    if (rows < 1 || rows > (1ull << 32)) return fail(h, W2V_ERR_ARG, "rows must be in 1..2^32");
+    const bool with_alias = access == W2V_PROBE_GATHER_ALIAS || access == W2V_PROBE_GATHER_RED_ALIAS;
+    if (with_alias && !h->have_tables) return fail(h, W2V_ERR_STATE, "w2v_build_alias has not been called");
+    DeviceGuard g(h->device);
+    cudaEvent_t e0, e1;
+    W2V_CUDA(h, cudaEventCreate(&e0));
+    W2V_CUDA(h, cudaEventCreate(&e1));
+    unsigned long long done = 0;
+    int k = -1;
+    cudaError_t ce = cudaEventRecord(e0, h->stream);
+    if (ce == cudaSuccess) {
+        k = launch_probe_rows(h->V, h->alias, (uint32_t)h->vocab, h->d / 4, h->ld / 4, (uint32_t)span_rows, rows, access,
+                              reinterpret_cast<float *>(h->st) + 15, h->sms, h->stream, &done);   // sink: the state's padding word
+        ce = cudaEventRecord(e1, h->stream);
+    }
+    if (ce == cudaSuccess) ce = cudaEventSynchronize(e1);
+    float t = 0.f;
+    if (ce == cudaSuccess && k > 0) ce = cudaEventElapsedTime(&t, e0, e1);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (k == -2) return fail(h, W2V_ERR_ARG, "the probe serves rows of at most 512 columns");
+    if (k < 0 || ce != cudaSuccess) return fail(h, W2V_ERR_CUDA, "probe launch", ce != cudaSuccess ? ce : cudaGetLastError());
+    h->launches += (uint64_t)k;
+    *ms = (double)t;
+    *rows_done = done;
+    return W2V_OK;
+}
+
 int32_t w2v_set_step(w2v_handle *h, uint64_t step_id)
 {
     if (!h) return W2V_ERR_ARG;

@@ -66,7 +66,7 @@ struct StepParams {
     double *DV;                 // [hot_rows * d] fp64 sums of G u(c) for the most-hit output rows
     uint32_t hot_rows;          // output rows [0, hot_rows) accumulate in DV (snapshot mode)
     uint32_t zero;              // always 0; ANDed with a loaded word it ties a later address to that load's arrival
-    uint32_t keep_negs;         // snapshot mode: pass 1 writes the negatives of every pair to l_negs, pass 2 reads them back
+    uint32_t keep_negs;         // snapshot mode: the negatives of every pair are in l_negs (SGNS: drawn by a launch of their own before pass 1; CBOW: written by pass 1) and read back by the passes
 };
 
 // F arrays of all shards (this one included) that receive a shard's partial dot products.
@@ -148,6 +148,11 @@ int launch_partial_dots(const float *U, const float *V, uint32_t vocab, uint32_t
                         float *out, DevState *st, int sms, cudaStream_t s);
 int launch_copy_rows(float *table, uint32_t vocab, uint32_t d, uint32_t ld, const int64_t *ids, uint64_t m,
                      float *buf, bool to_table, int sms, cudaStream_t s);
+
+// ---- memory-system probe (w2v_probe.cu): `rows` random rows of V in [0, span), returns -2 for d > 512 ----
+int launch_probe_rows(float *V, const uint2 *alias, uint32_t vocab, uint32_t d4, uint32_t ld4, uint32_t span,
+                      unsigned long long rows, uint32_t access, float *sink, int sms, cudaStream_t s,
+                      unsigned long long *rows_done);
 
 // ---- cosine retrieval (w2v_topk.cu) ----
 uint32_t topk_splits(uint64_t m, uint64_t n_candidates, int sms, uint32_t block_queries = 0, uint32_t tile_rows = 0);

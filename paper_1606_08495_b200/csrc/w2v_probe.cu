@@ -1,0 +1,116 @@
+// Memory-system ceilings for the access patterns of the update kernels, measured on the model's own
+// output table: random rows gathered (and optionally added to) with the same row layout, loads,
+// reductions and rows in flight per warp as the step, but with precomputable row numbers and no
+// sampling or arithmetic in the way.  What the step kernels reach is judged against these figures
+// rather than against a plain copy.  The additions add +0.0f, so the table's values do not change.
+#include "../../include/w2v.h"
+#include "w2v_device.cuh"
+#include "w2v_internal.h"
+
+namespace w2v {
+
+namespace {
+
+constexpr int kProbeTB = 4;            // rows in flight per warp, as in the step kernels at d = 300
+
+// row number of the i-th access: a mixing hash of i, reduced to [0, span)
+__device__ __forceinline__ uint32_t probe_row(unsigned long long i, uint32_t span, uint32_t salt)
+{
+    unsigned long long x = (i + 1ull) * 0x9E3779B97F4A7C15ull + salt;
+    x ^= x >> 30; x *= 0xBF58476D1CE4E5B9ull;
+    x ^= x >> 27; x *= 0x94D049BB133111EBull;
+    x ^= x >> 31;
+    return (uint32_t)(x % span);
+}
+
+template <int VPL, uint32_t access>
+__global__ void __launch_bounds__(kBlock, 2)
+probe_rows_kernel(float *V, const uint2 *alias, uint32_t vocab, uint32_t d4, uint32_t ld4, uint32_t span,
+                  unsigned long long per_warp, uint32_t zero, float *sink)
+{
+    constexpr int NCH = (VPL + 3) / 4;
+    const uint32_t lane = threadIdx.x & 31;
+    const unsigned long long warp = ((unsigned long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    float4 *V4 = reinterpret_cast<float4 *>(V);
+    constexpr bool with_alias = access == W2V_PROBE_GATHER_ALIAS || access == W2V_PROBE_GATHER_RED_ALIAS;
+    constexpr bool with_red = access == W2V_PROBE_GATHER_RED || access == W2V_PROBE_GATHER_RED_ALIAS ||
+                          access == W2V_PROBE_TOUCH_RED;
+    float acc = 0.f;
+    for (unsigned long long base = 0; base < per_warp; base += 32) {
+        // 32 row numbers per round, one per lane; with_alias: each goes through one random 8-byte
+        // read of the alias table first (what a negative draw costs)
+        uint32_t mine = probe_row(warp * per_warp + base + lane, span, 0u);
+        if (with_alias) {
+            const uint2 e = __ldg(alias + probe_row(warp * per_warp + base + lane, vocab, 77u));
+            if (e.x == 0u && e.y == 0xFFFFFFFFu) mine = 0u;          // never true for a built table
+        }
+        for (uint32_t j = 0; j < 32; j += kProbeTB) {
+            uint32_t r[kProbeTB];
+            Row<VPL> v[kProbeTB];
+            uint32_t x[kProbeTB][NCH];
+#pragma unroll
+            for (int t = 0; t < kProbeTB; ++t) {
+                r[t] = __shfl_sync(kFullMask, mine, j + t);
+                if (access == W2V_PROBE_TOUCH_RED) {
+                    row_touch<NCH>(x[t], V4 + (size_t)r[t] * ld4, d4, lane);
+                    row_zero(v[t]);
+                } else {
+                    row_load(v[t], V4 + (size_t)r[t] * ld4, d4, lane);
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < kProbeTB; ++t) {
+                uint32_t off = 0u;
+                float s = 0.f;
+                if (access == W2V_PROBE_TOUCH_RED) {
+                    off = touch_fence<NCH>(x[t], zero);
+                } else {
+                    Row<VPL> one;
+#pragma unroll
+                    for (int k = 0; k < VPL; ++k) one.x[k] = make_float4(1.f, 1.f, 1.f, 1.f);
+                    s = warp_sum(row_dot_partial(one, v[t]));
+                    acc += s;
+                }
+                if (with_red) {
+                    Row<VPL> z;
+                    row_zero(z);
+                    // the factor depends on the gathered row, so the addition cannot be issued before it arrived
+                    row_red_scaled(V4 + (size_t)r[t] * ld4 + off, s * 0.0f, z, d4, lane);
+                }
+            }
+        }
+    }
+    if (acc == 12345.678f) *sink = acc;
+}
+
+}  // namespace
+
+int launch_probe_rows(float *V, const uint2 *alias, uint32_t vocab, uint32_t d4, uint32_t ld4, uint32_t span,
+                      unsigned long long rows, uint32_t access, float *sink, int sms, cudaStream_t s,
+                      unsigned long long *rows_done)
+{
+    const int grid = sms * 2;
+    const unsigned long long warps = (unsigned long long)grid * (kBlock / 32);
+    unsigned long long per_warp = (rows + warps - 1) / warps;
+    per_warp = (per_warp + 31) / 32 * 32;
+    *rows_done = per_warp * warps;
+#define CALL_PROBE(VPL)                                                                                          \
+    switch (access) {                                                                                            \
+        case W2V_PROBE_GATHER: probe_rows_kernel<VPL, W2V_PROBE_GATHER><<<grid, kBlock, 0, s>>>(V, alias, vocab, d4, ld4, span, per_warp, 0u, sink); break; \
+        case W2V_PROBE_GATHER_RED: probe_rows_kernel<VPL, W2V_PROBE_GATHER_RED><<<grid, kBlock, 0, s>>>(V, alias, vocab, d4, ld4, span, per_warp, 0u, sink); break; \
+        case W2V_PROBE_GATHER_ALIAS: probe_rows_kernel<VPL, W2V_PROBE_GATHER_ALIAS><<<grid, kBlock, 0, s>>>(V, alias, vocab, d4, ld4, span, per_warp, 0u, sink); break; \
+        case W2V_PROBE_GATHER_RED_ALIAS: probe_rows_kernel<VPL, W2V_PROBE_GATHER_RED_ALIAS><<<grid, kBlock, 0, s>>>(V, alias, vocab, d4, ld4, span, per_warp, 0u, sink); break; \
+        default: probe_rows_kernel<VPL, W2V_PROBE_TOUCH_RED><<<grid, kBlock, 0, s>>>(V, alias, vocab, d4, ld4, span, per_warp, 0u, sink); break; \
+    }
+    switch ((d4 + 31) / 32) {
+        case 1: CALL_PROBE(1); break;
+        case 2: CALL_PROBE(2); break;
+        case 3: CALL_PROBE(3); break;
+        case 4: CALL_PROBE(4); break;
+        default: return -2;
+    }
+#undef CALL_PROBE
+    return cudaGetLastError() != cudaSuccess ? -1 : 1;
+}
+
+}  // namespace w2v

@@ -198,6 +198,7 @@ pair_offsets_kernel(const uint16_t *__restrict__ win, const unsigned long long *
 }
 
 // ---- explicit pair list ----------------------------------------------------------------
+// centre and context may both be NULL: only the negatives are written then (the snapshot step's list).
 __global__ void __launch_bounds__(kBlock)
 emit_pairs_kernel(StepParams p, int32_t *__restrict__ centre, int32_t *__restrict__ context,
                   int32_t *__restrict__ negs, uint64_t cap)
@@ -221,7 +222,7 @@ emit_pairs_kernel(StepParams p, int32_t *__restrict__ centre, int32_t *__restric
             uint32_t n0, n1;
             draw_pair_negatives(p, i, slot, w_out, lane, n0, n1, draws, redraws);
             if (pi < cap) {
-                if (lane == 0) { centre[pi] = c; context[pi] = (int32_t)w_out; }
+                if (lane == 0 && centre) { centre[pi] = c; context[pi] = (int32_t)w_out; }
                 if (lane < p.negatives) negs[pi * p.negatives + lane] = (int32_t)n0;
                 if (lane + 32u < p.negatives) negs[pi * p.negatives + lane + 32u] = (int32_t)n1;
             }

@@ -53,9 +53,22 @@ sgns_hogwild_kernel(StepParams p)
     flush_draw_counts(p.st, draws, redraws);
 }
 
+// negatives of pair number `pair` from the step's list (lane l: negative l in n0, negative l + 32 in n1)
+__device__ __forceinline__ void load_pair_negatives(const StepParams &p, unsigned long long pair, uint32_t lane,
+                                                    uint32_t &n0, uint32_t &n1)
+{
+    const int32_t *src = p.l_negs + pair * p.negatives;
+    n0 = 0; n1 = 0;
+    if (lane < p.negatives) n0 = (uint32_t)__ldcg(src + lane);
+    if (lane + 32u < p.negatives) n1 = (uint32_t)__ldcg(src + lane + 32u);
+}
+
 // ---- snapshot mode, pass 1 (Algorithm 1 + the client's aggregation): dots and coefficients ----
 // Reads only start-of-step tables.  Writes G for every target and the per-centre sum
 // DU[q] = sum G v(target) (the scratch area of Algorithm 2 for the centre's own row).
+// The step's negatives were drawn into l_negs by a flat launch before this one (a draw inside this
+// loop puts a random read of the alias table in front of every pair's gathers); the list entry of
+// the next pair is fetched while the current pair's rows are in flight.
 template <int VPL, int TB>
 __global__ void __launch_bounds__(kBlock)
 sgns_snap_dots_kernel(StepParams p)
@@ -67,27 +80,23 @@ sgns_snap_dots_kernel(StepParams p)
     const float4 *U4 = reinterpret_cast<const float4 *>(p.U);
     float4 *DU4 = reinterpret_cast<float4 *>(p.DU);
     const uint32_t n1p = p.negatives + 1u;
-    uint32_t draws = 0, redraws = 0;
     for (uint32_t q = warp; q < nk; q += nwarps) {
         const uint32_t w = p.win[q];
         const uint32_t left = w & 0xFFu, right = w >> 8;
         if (left + right == 0) continue;
         const uint32_t c = (uint32_t)p.ctok[q];
-        const uint32_t i = p.cidx[q];
         Row<VPL> u, du;
         row_load(u, U4 + (size_t)c * p.ld4, p.d4, lane);
         row_zero(du);
         unsigned long long pair = p.pair_off[q], gi = pair * n1p;
+        const unsigned long long pair_end = pair + left + right;
+        uint32_t nx0, nx1;
+        load_pair_negatives(p, pair, lane, nx0, nx1);
         for (uint32_t pp = q - left; pp <= q + right; ++pp) {
             if (pp == q) continue;
             const uint32_t w_out = (uint32_t)p.ctok[pp];
-            uint32_t n0, n1;
-            draw_pair_negatives(p, i, pp + p.window - q, w_out, lane, n0, n1, draws, redraws);
-            if (p.keep_negs) {
-                int32_t *dst = const_cast<int32_t *>(p.l_negs) + pair * p.negatives;     // this launch is the list's writer
-                if (lane < p.negatives) dst[lane] = (int32_t)n0;
-                if (lane + 32u < p.negatives) dst[lane + 32u] = (int32_t)n1;
-            }
+            const uint32_t n0 = nx0, n1 = nx1;
+            if (pair + 1 < pair_end) load_pair_negatives(p, pair + 1, lane, nx0, nx1);
             for_each_target_touched<VPL, TB>(p, u, w_out, n0, n1, lane,
                 [&](uint32_t t, uint32_t, const Row<VPL> &v, float f) {
                     const float s = sigmoidf_exact(f);
@@ -104,7 +113,6 @@ sgns_snap_dots_kernel(StepParams p)
             if (idx < p.d4) DU4[(size_t)q * p.d4 + idx] = du.x[v];
         }
     }
-    flush_draw_counts(p.st, draws, redraws);
 }
 
 // ---- snapshot mode, pass 2 (Algorithm 2, output rows): v(target) += G u(c) ------------------
@@ -136,9 +144,7 @@ sgns_snap_adjust_v_kernel(StepParams p)
             const uint32_t w_out = (uint32_t)p.ctok[pp];
             uint32_t n0 = 0, n1 = 0;
             if (p.keep_negs) {
-                const int32_t *src = p.l_negs + pair * p.negatives;
-                if (lane < p.negatives) n0 = (uint32_t)__ldcg(src + lane);
-                if (lane + 32u < p.negatives) n1 = (uint32_t)__ldcg(src + lane + 32u);
+                load_pair_negatives(p, pair, lane, n0, n1);
             } else {
                 draw_pair_negatives(p, i, pp + p.window - q, w_out, lane, n0, n1, draws, redraws);
             }
@@ -323,10 +329,17 @@ int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t block
 {
     const int vpl = (int)((p.d4 + 31) / 32);
     const int tb = pick_tb(rows_in_flight, vpl, p.negatives);
+    int launched = 1;
+    if (!p.keep_negs || !p.l_negs) return -1;
+    {                          // the step's negatives, drawn once for both passes
+        const int k = launch_emit_pairs(p, nullptr, nullptr, const_cast<int32_t *>(p.l_negs), ~0ull, sms * 8, s);
+        if (k < 0) return -1;
+        launched += k;
+    }
     W2V_FOR_VPL(snap_dots(p, blocks_per_sm, sms, s))
     if (cudaGetLastError() != cudaSuccess) return -1;
     const int k = launch_snapshot_apply(p, blocks_per_sm, sms, s);
-    return k < 0 ? -1 : 1 + k;
+    return k < 0 ? -1 : launched + k;
 }
 
 }  // namespace w2v

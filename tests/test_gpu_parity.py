@@ -464,3 +464,23 @@ def test_sampled_indices_random_chunk_structures():
         c1, n1, _ = gpu.sample_cbow(toks, W, N, allow=(binding.W2V_ERR_TOKEN_RANGE,)) if len(toks) else (c0, n0, None)
         assert np.array_equal(c0, c1) and np.array_equal(n0, n1)
         gpu.close()
+
+
+def test_memory_probe_leaves_the_table_as_it_was():
+    # the probe's additions add zero: V keeps its bits; every access pattern runs and reports a time
+    cfg = corpus.scaled(corpus.CONFIGS["tiny"], vocab=5000, d=100)
+    gpu, cpu, cp = make_pair(cfg, row_stride=128)
+    ids = np.arange(cfg["vocab"])
+    rng = np.random.default_rng(2)
+    Vv = rng.normal(scale=0.1, size=(cfg["vocab"], cfg["d"])).astype(np.float32)
+    gpu.write_rows(1, ids, Vv)
+    for access in range(5):
+        for span in (cfg["vocab"], 17):
+            ms, done = binding.w2v_probe_rows(gpu.h, access, span, 100_000)
+            assert ms > 0 and done >= 100_000
+    assert np.array_equal(gpu.read_rows(1, ids), Vv)
+    for args in ((5, 10, 10), (0, 0, 10), (0, cfg["vocab"] + 1, 10), (0, 10, 0)):
+        with pytest.raises(binding.W2VError) as e:
+            binding.w2v_probe_rows(gpu.h, *args)
+        assert e.value.code == binding.W2V_ERR_ARG
+    gpu.close()

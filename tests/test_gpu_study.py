@@ -1,0 +1,161 @@
+"""Minibatch size, staleness and convergence (Section 5.1, last paragraph: minibatches of input words
+that are far apart; Section 7.1: minibatches of 50-200 input words per client, and too many clients
+at once "fail to converge"), on the small synthetic corpus.
+
+One pass over the corpus in each setting, same chunks, step numbers and learning-rate schedule as
+the stored run of the sequential CPU checker (tests/golden/hogwild_losses.txt); the held-out loss of
+the vectors read back is evaluated by the checker's loss().  What varies is how many input words
+are processed against one state of the tables:
+  * snapshot mode with interleaved minibatches of B input words: B is exactly the paper's
+    minibatch, every update of a step is computed from the vectors as they were before the step;
+  * Hogwild mode with chunks of n tokens: the GPU runs ~2400 warps (one input word each) at a time,
+    whatever the chunk size.
+The table printed by the first test is the one in the design notes."""
+import numpy as np
+import pytest
+
+from oracle import Oracle
+from paper_1606_08495_b200 import binding, corpus
+from paper_1606_08495_b200.train import gpu_step, train
+from conftest import load_golden
+
+pytestmark = pytest.mark.gpu
+
+SEED = 41
+HELD = (1_000_000, 1_000_001)
+HELD_STEP_BASE = 10 ** 9
+UNTRAINED = 6 * np.log(2.0)            # (1 + N) log 2 with N = 5: every dot product is zero
+
+
+def heldout(model, cfg, cp):
+    ev = Oracle(cfg["vocab"], cfg["d"], SEED)
+    ev.build_tables(cp.counts, cfg["subsample_t"])
+    ids = np.arange(cfg["vocab"])
+    ev.write_rows(0, ids, model.read_rows(0, ids))
+    ev.write_rows(1, ids, model.read_rows(1, ids))
+    tot, P = 0.0, 0
+    for j in HELD:
+        s, p = ev.loss(cp.chunk(j), cfg["window"], cfg["negatives"], step_id=HELD_STEP_BASE + j)
+        tot += s; P += p
+    ev.close()
+    return tot / P
+
+
+def regroup(chunks, tokens_per_step):
+    """The same token stream cut into pieces of about `tokens_per_step` entries: whole sentences of
+    one chunk, or several chunks joined."""
+    n = len(chunks[0])
+    if tokens_per_step >= n:
+        k = max(1, tokens_per_step // n)
+        return [np.concatenate(chunks[i:i + k]) for i in range(0, len(chunks), k)]
+    out = []
+    for c in chunks:
+        ends = np.flatnonzero(c == -1) + 1
+        per = max(1, int(round(len(ends) * tokens_per_step / n)))
+        cuts = [0] + [int(ends[i]) for i in range(per - 1, len(ends), per)]
+        if cuts[-1] != len(c):
+            cuts.append(len(c))
+        out += [c[a:b] for a, b in zip(cuts, cuts[1:])]
+    return out
+
+
+def run(cfg, cp, chunks, mode, stride=1):
+    g = binding.W2V(cfg["vocab"], cfg["d"], SEED, row_stride=binding.aligned_row_stride(cfg["d"]))
+    g.build_alias(cp.counts, cfg["subsample_t"])
+    train(gpu_step(g, cfg["window"], cfg["negatives"], mode), chunks, epochs=1, lr0=cfg["lr"], stride=stride)
+    g.set_interleave(0, 1)
+    loss = heldout(g, cfg, cp)
+    g.close()
+    return loss
+
+
+def test_loss_against_minibatch_size_and_staleness():
+    cfg_name, n_chunks, words, _, want = load_golden("hogwild_losses.txt")["small"][0]
+    cfg = corpus.CONFIGS[cfg_name]
+    cp = corpus.Corpus(cfg)
+    chunks = [cp.chunk(i) for i in range(int(n_chunks))]
+    want = float(want)
+    centres = 0.52 * cfg["minibatch"]                        # kept input words per chunk, about
+    rows = []
+    for B in (50, 200, 1000, 2500, 5000, 10_000, None):
+        stride = 1 if B is None else max(1, int(round(centres / B)))
+        loss = run(cfg, cp, chunks, binding.MODE_SNAPSHOT, stride)
+        rows.append(("snapshot", "%d input words" % round(centres / stride), loss))
+    for n in (4096, 16_384, 65_536, 262_144, 1_048_576):
+        loss = run(cfg, cp, regroup(chunks, n), binding.MODE_HOGWILD)
+        rows.append(("hogwild", "chunks of %d tokens" % n, loss))
+    print("\nSTUDY small corpus, one pass, lr0 %.3f; sequential checker %.5f, untrained %.5f" % (cfg["lr"], want, UNTRAINED))
+    for mode, what, loss in rows:
+        print("STUDY %-9s %-26s held-out loss %.5f  (%+.2f %% of the sequential checker's)" %
+              (mode, what, loss, 100.0 * (loss - want) / want))
+    snap = [l for m, w, l in rows if m == "snapshot"]
+    hog = [l for m, w, l in rows if m == "hogwild"]
+    # the paper's minibatch sizes (50-200 input words, and 1000) train as well as one pair after another
+    assert all(np.isfinite(l) and abs(l - want) <= 0.01 * want for l in snap[:3])
+    # a whole chunk (34 k input words) against one state of the tables does not converge at this
+    # learning rate: the summed updates of a frequent word overshoot (the checker shows the same, below)
+    assert not np.isfinite(snap[-1]) or snap[-1] >= UNTRAINED
+    # Hogwild: the staleness window is the ~2400 input words in flight, not the chunk
+    assert all(np.isfinite(l) and abs(l - want) <= 0.01 * want for l in hog)
+
+
+def test_whole_chunk_minibatches_diverge_in_the_checker_too():
+    # the first whole-chunk snapshot steps on the small corpus: the vectors of both implementations
+    # grow by orders of magnitude, while minibatches of ~200 input words keep them small
+    cfg = corpus.CONFIGS["small"]
+    cp = corpus.Corpus(cfg)
+    W, N, lr = cfg["window"], cfg["negatives"], cfg["lr"]
+    gpu = binding.W2V(cfg["vocab"], cfg["d"], SEED)
+    cpu = Oracle(cfg["vocab"], cfg["d"], SEED)
+    gpu.build_alias(cp.counts, cfg["subsample_t"]); cpu.build_tables(cp.counts, cfg["subsample_t"])
+    ids = np.arange(2000)                                    # the most frequent words
+    for i in range(8):
+        for m in (gpu, cpu):
+            m.set_step(i)
+        gpu.sgns_step(cp.chunk(i), W, N, lr, binding.MODE_SNAPSHOT)
+        cpu.step(cp.chunk(i), W, N, lr, 0)
+    big_gpu = float(np.abs(gpu.read_rows(1, ids)).max())
+    big_cpu = float(np.abs(cpu.read_rows(1, ids)).max())
+    small = binding.W2V(cfg["vocab"], cfg["d"], SEED)
+    small.build_alias(cp.counts, cfg["subsample_t"])
+    train(gpu_step(small, W, N, binding.MODE_SNAPSHOT), [cp.chunk(i) for i in range(8)], epochs=1, lr0=lr, stride=170)
+    calm = float(np.abs(small.read_rows(1, ids)).max())
+    print("largest |v| among the 2000 most frequent words after 8 chunks: whole-chunk minibatches gpu %.3g checker %.3g; "
+          "minibatches of ~200 input words %.3g" % (big_gpu, big_cpu, calm))
+    assert big_gpu > 100.0 and big_cpu > 100.0 and calm < 5.0
+    gpu.close(); cpu.close(); small.close()
+
+
+def test_snapshot_training_at_the_papers_minibatch_equals_the_checker():
+    # deterministic mode, minibatches of ~50 input words (Section 7.1), one pass over the tiny corpus
+    # on both sides: same held-out loss to 1e-4 (the steps themselves agree to 1e-5 per row)
+    cfg = corpus.CONFIGS["tiny"]
+    cp = corpus.Corpus(cfg)
+    W, N = cfg["window"], cfg["negatives"]
+    chunks = [cp.chunk(i) for i in range(cfg["corpus_tokens"] // cfg["minibatch"])]
+    stride = 40                                              # 4096 tokens, about 2000 kept: ~50 input words per step
+    gpu = binding.W2V(cfg["vocab"], cfg["d"], SEED)
+    cpu = Oracle(cfg["vocab"], cfg["d"], SEED)
+    gpu.build_alias(cp.counts, cfg["subsample_t"]); cpu.build_tables(cp.counts, cfg["subsample_t"])
+
+    def cpu_step(t, lr, num, ph, st):
+        cpu.set_step(num); cpu.set_interleave(ph, st)
+        cpu.step(t, W, N, lr, 0)
+
+    train(gpu_step(gpu, W, N, binding.MODE_SNAPSHOT), chunks, epochs=1, lr0=cfg["lr"], stride=stride)
+    train(cpu_step, chunks, epochs=1, lr0=cfg["lr"], stride=stride)
+    gpu.set_interleave(0, 1); cpu.set_interleave(0, 1)
+    tot_c = tot_g = 0.0
+    P = 0
+    ev = Oracle(cfg["vocab"], cfg["d"], SEED)
+    ev.build_tables(cp.counts, cfg["subsample_t"])
+    ids = np.arange(cfg["vocab"])
+    ev.write_rows(0, ids, gpu.read_rows(0, ids)); ev.write_rows(1, ids, gpu.read_rows(1, ids))
+    for j in HELD:
+        s, p = cpu.loss(cp.chunk(j), W, N, step_id=HELD_STEP_BASE + j)
+        tot_c += s; P += p
+        tot_g += ev.loss(cp.chunk(j), W, N, step_id=HELD_STEP_BASE + j)[0]
+    want, got = tot_c / P, tot_g / P
+    print("tiny corpus, snapshot mode, ~50 input words per step: held-out loss checker %.6f gpu %.6f" % (want, got))
+    assert want < 0.9 * UNTRAINED and abs(got - want) <= 1e-4 * want
+    gpu.close(); cpu.close(); ev.close()
