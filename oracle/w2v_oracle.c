@@ -16,35 +16,36 @@
  *
  * What each part follows:
  *   philox4x32_10      the published Philox4x32-10 counter-based generator
- *                      (Salmon et al., SC'11); stands in for the "Random Number
- *                      Generator initialized with seed" of Algorithms 1 and 2,
+ *                      (Salmon et al., SC'11); stands in for the seeded random
+ *                      number generator of Algorithms 1 and 2,
  *                      so that the same seed regenerates the same negatives.
- *   orc_init_row       "vectors are initialized ... as in word2vec"
+ *   orc_init_row       initial values as in the word2vec program
  *                      (Section 5.1): input rows uniform in [-0.5/d, 0.5/d),
  *                      output rows zero.
- *   build_alias        negative-example distribution "derived from the
- *                      vocabulary histogram" (Section 5.1, dotprod item):
+ *   build_alias        negative-example distribution computed from the
+ *                      word counts (Section 5.1, dotprod item):
  *                      unigram^(3/4), sampled through a Vose alias table.
  *   build_keep         sub-sampling of frequent words (Section 3, last lines).
  *   sample_chunk       Eq. (1)/(3) index sets: dirty contexts (footnote to
  *                      Section 3), random window radius b, N negatives != w_O
- *                      (Algorithm 1, "NS <- Array(N negative word indices")).
+ *                      (Algorithm 1, the array NS of negatives).
  *   orc_step mode 0    Algorithm 1 + Algorithm 3 (aggregation, G+ / G-) +
  *                      Algorithm 2 literally: all reads see start-of-call
- *                      values, deltas are applied at the end (Section 5.1,
- *                      "not updated until the end of the call").
+ *                      values, deltas are applied at the end (Section 5.1:
+ *                      vectors change only when the call ends).
  *   orc_step mode 1    the sequential limit of the lock-free operation of
  *                      Section 5.1: targets one after another, every read sees
  *                      every earlier write.
  *   orc_set_interleave interleaved minibatch formation (Section 5.1, last
  *                      paragraph): the input words of one call are a stride apart.
  *   orc_cbow_*         the continuous-bag-of-words variant (footnote to
- *                      Section 5: "readily extends to CBOW"): the mean of the
+ *                      Section 5, which only notes that the design carries
+ *                      over to CBOW): the mean of the
  *                      context words' input vectors predicts the centre word;
  *                      same index sets, same two modes, exact gradient.
- *   orc_topk_cosine    retrieval by cosine similarity (Section 2: "the K queries
- *                      with the highest similarity are retrieved"; Section 7.2:
- *                      K nearest, kept only above a threshold tau): brute force.
+ *   orc_topk_cosine    retrieval by cosine similarity (Section 2: top-K by
+ *                      cosine; Section 7.2: K nearest, kept only above a
+ *                      threshold tau): brute force.
  *   orc_partial_dots   u_s(w_I) v_s(w_O)^T of Algorithm 1 for one column slice.
  *   orc_loss           minus Eq. (1) restricted to a chunk, per positive pair.
  *

@@ -142,7 +142,7 @@ int32_t grow(w2v_handle *h, T **p, uint64_t *cap, uint64_t need, bool slack)
     return W2V_OK;
 }
 
-// Scratch of the deferred-update passes (Algorithm 2's "not updated until the end of the call"):
+// Scratch of the deferred-update passes (Algorithm 2 applies its updates only when the call ends):
 // coefficients G for `targets` targets, per-centre sums DU for every token the chunk scratch holds,
 // fp64 sums DV of the most-hit output rows (zero between steps).
 int32_t ensure_update_scratch(w2v_handle *h, uint64_t targets, bool slack)

@@ -1,4 +1,4 @@
-// Continuous bag of words (footnote to Section 5: the system "readily extends to the CBOW variant").
+// Continuous bag of words (footnote to Section 5: the paper notes that its design carries over to CBOW).
 // One example per kept token q with at least one context word:
 //   hbar = mean of the input vectors u(w_k) of the window's context words,
 //   targets = the centre word (label 1) and N negatives != centre word (label 0),

@@ -1,4 +1,4 @@
-// Table-level kernels: initialisation (Section 5.1, "initialized ... as in word2vec"),
+// Table-level kernels: initialisation (Section 5.1: the same initial values as the word2vec program),
 // row export/import (Section 6.1, vector export) and the column-slice partial dot
 // products of Algorithm 1 for caller-given index pairs.
 #include <math_constants.h>

@@ -114,7 +114,7 @@ coefficients_kernel(const float *__restrict__ F, float *__restrict__ G, unsigned
 
 // ---- Algorithm 2, input rows: DU[q] = sum over the centre's targets of G v(target) -----------
 // Reads V only; the additions to V happen in a later launch, so every v(target) is the
-// start-of-call vector ("not updated until the end of the call").
+// start-of-call vector (Section 5.1: vectors change only when the call ends).
 template <int VPL, int TB>
 __global__ void __launch_bounds__(kBlock)
 shard_du_kernel(StepParams p)

@@ -1,5 +1,5 @@
-"""The training loop around the step (Section 5.1: "the data set is iterated over multiple times and
-after each iteration, the learning rate is reduced in a manner similar to" word2vec; optional
+"""The training loop around the step (Section 5.1: several passes over the data, with the learning
+rate lowered from pass to pass in the way the word2vec program lowers it; optional
 interleaved minibatch formation).
 
 Harness level only: it decides which chunk, which step number, which learning rate and which
@@ -18,8 +18,8 @@ def learning_rate(lr0: float, words_done: int, words_total: int, schedule: str =
                   epoch: int = 0, epochs: int = 1) -> float:
     """"linear": lr0 * max(1 - words_done / (words_total + 1), 1e-4), evaluated once per step (the
     open-source word2vec program's decay, to which the paper refers); "epoch": the same line
-    evaluated at the start of each pass over the data and held during it (the paper's wording:
-    reduced after each iteration)."""
+    evaluated at the start of each pass over the data and held during it (Section 5.1 speaks of a
+    reduction per pass)."""
     if schedule == "linear":
         frac = 1.0 - words_done / (words_total + 1.0)
     elif schedule == "epoch":

@@ -1,6 +1,6 @@
 """Minibatch size, staleness and convergence (Section 5.1, last paragraph: minibatches of input words
 that are far apart; Section 7.1: minibatches of 50-200 input words per client, and too many clients
-at once "fail to converge"), on the small synthetic corpus.
+at once no longer converge), on the small synthetic corpus.
 
 One pass over the corpus in each setting, same chunks, step numbers and learning-rate schedule as
 the stored run of the sequential CPU checker (tests/golden/hogwild_losses.txt); the held-out loss of

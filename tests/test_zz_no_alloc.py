@@ -44,7 +44,9 @@ def test_noalloc_sampler_matches_the_ordinary_one_twice_in_a_row():
     W, N = cfg["window"], cfg["negatives"]
     # first a large chunk, then a smaller one with another step number: whatever the first call
     # left behind in the fixed array must not show up in the second result
-    for step, words in ((0, 60_000), (3, 9_000)):
+    # the third chunk is small enough for the ordinary call's one-launch sampler (at most 8192 tokens),
+    # which the allocation-free call never uses: two different kernel sequences, one answer
+    for step, words in ((0, 60_000), (3, 9_000), (4, 5_000)):
         model.set_step(step)
         toks = cp.chunk(step, words)
         assert len(toks) <= MAX_TOKENS
@@ -53,6 +55,30 @@ def test_noalloc_sampler_matches_the_ordinary_one_twice_in_a_row():
         for a, b in zip(ref[1:4], got[1:4]):
             assert np.array_equal(a, b)
         assert ref[4] == got[4]
+    model.close()
+
+
+def test_noalloc_sampler_empty_chunk_and_ids_outside_the_vocabulary():
+    model = binding.W2V(50, 8, seed=2)
+    model.build_alias(np.full(50, 4, dtype=np.uint64), 0.0)
+    t = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for fn in (binding.w2v_sample_pairs, binding.w2v_sample_pairs_noalloc):
+        st = binding.StepStats()
+        rc, P = fn(model.h, t, 0, 3, 2, None, None, None, 0, st)           # n = 0
+        assert rc == binding.W2V_OK and P == 0 and st.kept == 0 and st.pairs == 0
+    toks = np.array([1, 2, 50, 3, -1, 4, -5, 6, 7, -1, 9], dtype=np.int32)  # 50 and -5 are not word ids
+    t = torch.from_numpy(toks).cuda()
+    cap = len(toks) * 6
+    res = []
+    for fn in (binding.w2v_sample_pairs, binding.w2v_sample_pairs_noalloc):
+        centre = torch.full((cap,), -7, dtype=torch.int32, device="cuda")
+        context = torch.full((cap,), -7, dtype=torch.int32, device="cuda")
+        negs = torch.full((cap * 2,), -7, dtype=torch.int32, device="cuda")
+        st = binding.StepStats()
+        rc, P = fn(model.h, t, len(toks), 3, 2, centre, context, negs, cap, st, allow=(binding.W2V_ERR_TOKEN_RANGE,))
+        assert rc == binding.W2V_ERR_TOKEN_RANGE and st.oov == 2 and (st.status & 1)
+        res.append((P, centre[:P].tolist(), context[:P].tolist(), negs[: 2 * P].tolist(), st.as_dict()))
+    assert res[0] == res[1] and res[0][0] > 0
     model.close()
 
 
