@@ -30,12 +30,13 @@ from paper_1606_08495_b200 import corpus  # noqa: E402
 METRIC = "sgns_positive_pairs_per_sec"
 UNIT = "pairs/s"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes moved per algorithmic byte by the Hogwild update kernel on the large workload, from one
-# one-pass ncu capture of that kernel ((dram__bytes_read.sum + dram__bytes_write.sum) / model bytes of the
-# captured launch: 126.42 / 121.9 GB, rows on 128-byte boundaries).  It is a constant taken once, not a
-# counter read during this run (the JSON line says so in "traffic_kind"), and applies to the large workload
-# in Hogwild mode with the default row stride and launch shape only; anything else reports null.
-TRAFFIC_PER_ALGORITHMIC_BYTE = 1.037
+# DRAM bytes moved per algorithmic byte by the update kernels of a Hogwild step on the large workload (the
+# launch that draws the step's negatives plus the gather / update kernel), from one one-pass ncu capture of
+# those kernels ((dram__bytes_read.sum + dram__bytes_write.sum) / model bytes of the captured step:
+# (5.01 + 120.61) / 121.9 GB, rows on 128-byte boundaries).  It is a constant taken once, not a counter read
+# during this run (the JSON line says so in "traffic_kind"), and applies to the large workload in Hogwild
+# mode with the default row stride and launch shape only; anything else reports null.
+TRAFFIC_PER_ALGORITHMIC_BYTE = 1.031
 
 
 def algorithmic_bytes(d, centres, pairs, negatives):
@@ -476,7 +477,9 @@ def run_gpu(args):
                     "h2d_bytes_per_step": h2d // K, "d2h_bytes_per_step": d2h // K},
             "gpu_launches": all_launches,
             "roofline": {"bound": "hbm",
-                         "kernel": ("cbow_" if cbow else "sgns_") + ("hogwild_kernel" if args.mode == "hogwild" else "snap_* (3 passes)"),
+                         "kernel": ("cbow_hogwild_kernel" if cbow and args.mode == "hogwild" else "cbow_snap_* (3 passes)" if cbow
+                                    else "draw_negatives_kernel + sgns_hogwild_kernel" if args.mode == "hogwild"
+                                    else "draw_negatives_kernel + sgns_snap_* (3 passes)"),
                          "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "frac_of_8TBps": achieved / 8000.0,

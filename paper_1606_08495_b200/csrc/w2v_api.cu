@@ -182,6 +182,7 @@ int32_t ensure_error_word(w2v_handle *h)
 // the pair count nor re-allocates.  Larger bounds (wide windows on long chunks) fall back to
 // reading the pair count.
 constexpr uint64_t kSnapshotBoundBudget = 1ull << 30;
+constexpr uint64_t kListChunk = 200000;       // Hogwild mode: chunks of at least this many tokens use a list of negatives
 
 int32_t check_step_args(w2v_handle *h, const void *tokens, uint64_t n, uint32_t window, uint32_t negatives)
 {
@@ -290,7 +291,19 @@ int32_t step_impl(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t win
     int32_t rc = enqueue_sampling(h, tokens, n, window);
     if (rc != W2V_OK) return rc;
     if (mode == W2V_MODE_HOGWILD) {
+        // long chunks draw their negatives into a list first (four more launches, a faster update
+        // kernel: measured equal at 0.26 M tokens, 6 % faster at 1 M tokens with 5 negatives), when
+        // the list for the worst case fits the budget
+        const uint64_t negs_cap = n * 2ull * window * negatives;
+        const bool list = n >= kListChunk && negs_cap * sizeof(int32_t) <= kSnapshotBoundBudget;
+        if (list) {
+            int k = launch_pair_offsets(n, h->sc, h->st, h->stream);
+            if (k < 0) return fail(h, W2V_ERR_CUDA, "pair offset launch", cudaGetLastError());
+            h->launches += (uint64_t)k;
+            if ((rc = grow(h, &h->l_negs, &h->l_cap_negs, negs_cap, false)) != W2V_OK) return rc;
+        }
         StepParams p = make_params(h, window, negatives, lr);
+        p.keep_negs = list ? 1u : 0u;
         if ((rc = profile_mark(h)) != W2V_OK) return rc;
         int k = launch_hogwild(p, h->rows_in_flight, h->blocks_per_sm, h->sms, h->stream);
         if (k < 0) return fail(h, W2V_ERR_CUDA, "update kernel launch", cudaGetLastError());

@@ -198,7 +198,6 @@ pair_offsets_kernel(const uint16_t *__restrict__ win, const unsigned long long *
 }
 
 // ---- explicit pair list ----------------------------------------------------------------
-// centre and context may both be NULL: only the negatives are written then (the snapshot step's list).
 __global__ void __launch_bounds__(kBlock)
 emit_pairs_kernel(StepParams p, int32_t *__restrict__ centre, int32_t *__restrict__ context,
                   int32_t *__restrict__ negs, uint64_t cap)
@@ -222,11 +221,43 @@ emit_pairs_kernel(StepParams p, int32_t *__restrict__ centre, int32_t *__restric
             uint32_t n0, n1;
             draw_pair_negatives(p, i, slot, w_out, lane, n0, n1, draws, redraws);
             if (pi < cap) {
-                if (lane == 0 && centre) { centre[pi] = c; context[pi] = (int32_t)w_out; }
+                if (lane == 0) { centre[pi] = c; context[pi] = (int32_t)w_out; }
                 if (lane < p.negatives) negs[pi * p.negatives + lane] = (int32_t)n0;
                 if (lane + 32u < p.negatives) negs[pi * p.negatives + lane + 32u] = (int32_t)n1;
             }
             ++pi;
+        }
+    }
+    flush_draw_counts(p.st, draws, redraws);
+}
+
+// ---- the step's negatives as a list ---------------------------------------------------------
+// negs[pair * N + k] for every pair of the chunk, pairs numbered as in the pair list.  A draw is a
+// dependent chain (generator, one random 8-byte read of the alias table, compare); inside an update
+// kernel that chain sits in front of every pair's row gathers with N of 32 lanes busy.  Here the
+// lanes of a warp share out all cnt * N draws of a centre, so every lane has a draw in flight.
+__global__ void __launch_bounds__(kBlock)
+draw_negatives_kernel(StepParams p, int32_t *__restrict__ negs)
+{
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    const uint32_t nk = (uint32_t)p.st->n_kept;
+    const uint32_t N = p.negatives;
+    uint32_t draws = 0, redraws = 0;
+    for (uint32_t q = warp; q < nk; q += nwarps) {
+        const uint32_t w = p.win[q];
+        const uint32_t left = w & 0xFFu, cnt = left + (w >> 8);
+        if (cnt == 0) continue;
+        const uint32_t i = p.cidx[q];
+        int32_t *dst = negs + p.pair_off[q] * N;
+        const uint32_t items = cnt * N;
+        for (uint32_t it = lane; it < items; it += 32) {
+            const uint32_t j = it / N, k = it - j * N;
+            const uint32_t pp = q - left + j + (j >= left ? 1u : 0u);      // position of the centre's j-th context
+            const uint32_t w_out = (uint32_t)p.ctok[pp];
+            dst[it] = (int32_t)draw_negative(p.tab.alias, p.vocab, p.k0, p.k1, i, p.step_lo, pp + p.window - q, k, w_out,
+                                             draws, redraws);
         }
     }
     flush_draw_counts(p.st, draws, redraws);
@@ -356,6 +387,13 @@ int launch_pair_offsets(uint64_t n, const Scratch &sc, DevState *st, cudaStream_
     pair_offsets_kernel<<<nt, kScanBlock, 0, s>>>(sc.win, sc.cnt_tile, sc.pair_off, st, examples);
     if (cudaGetLastError() != cudaSuccess) return -1;
     return 3;
+}
+
+int launch_draw_negatives(const StepParams &p, int32_t *negs, int grid, cudaStream_t s)
+{
+    draw_negatives_kernel<<<grid, kBlock, 0, s>>>(p, negs);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    return 1;
 }
 
 int launch_emit_pairs(const StepParams &p, int32_t *centre, int32_t *context, int32_t *negs,

@@ -11,8 +11,21 @@
 
 namespace w2v {
 
+// negatives of pair number `pair` from the step's list (lane l: negative l in n0, negative l + 32 in n1)
+__device__ __forceinline__ void load_pair_negatives(const StepParams &p, unsigned long long pair, uint32_t lane,
+                                                    uint32_t &n0, uint32_t &n1)
+{
+    const int32_t *src = p.l_negs + pair * p.negatives;
+    n0 = 0; n1 = 0;
+    if (lane < p.negatives) n0 = (uint32_t)__ldcg(src + lane);
+    if (lane + 32u < p.negatives) n1 = (uint32_t)__ldcg(src + lane + 32u);
+}
+
 // ---- Hogwild mode: one pass, updates land as they are computed ---------------------------
-template <int VPL, int TB>
+// LIST: the step's negatives were drawn into l_negs by a launch of their own (draw_negatives_kernel)
+// and the entry of the next pair is fetched while the current pair's rows are in flight; otherwise
+// every pair draws its own (small chunks, where one more launch would cost more than it saves).
+template <int VPL, int TB, bool LIST>
 __global__ void __launch_bounds__(kBlock)
 sgns_hogwild_kernel(StepParams p)
 {
@@ -32,11 +45,23 @@ sgns_hogwild_kernel(StepParams p)
         Row<VPL> u, etot;
         row_load(u, U4 + (size_t)c * p.ld4, p.d4, lane);
         row_zero(etot);
+        unsigned long long pair = 0, pair_end = 0;
+        uint32_t nx0 = 0, nx1 = 0;
+        if (LIST) {
+            pair = p.pair_off[q];
+            pair_end = pair + left + right;
+            load_pair_negatives(p, pair, lane, nx0, nx1);
+        }
         for (uint32_t pp = q - left; pp <= q + right; ++pp) {
             if (pp == q) continue;
             const uint32_t w_out = (uint32_t)p.ctok[pp];
             uint32_t n0, n1;
-            draw_pair_negatives(p, i, pp + p.window - q, w_out, lane, n0, n1, draws, redraws);
+            if (LIST) {
+                n0 = nx0; n1 = nx1;
+                if (++pair < pair_end) load_pair_negatives(p, pair, lane, nx0, nx1);
+            } else {
+                draw_pair_negatives(p, i, pp + p.window - q, w_out, lane, n0, n1, draws, redraws);
+            }
             Row<VPL> e;
             row_zero(e);
             for_each_target<VPL, TB>(p, u, w_out, n0, n1, lane,
@@ -50,17 +75,7 @@ sgns_hogwild_kernel(StepParams p)
         }
         row_red_scaled(U4 + (size_t)c * p.ld4, 1.0f, etot, p.d4, lane);          // u(c) += sum e
     }
-    flush_draw_counts(p.st, draws, redraws);
-}
-
-// negatives of pair number `pair` from the step's list (lane l: negative l in n0, negative l + 32 in n1)
-__device__ __forceinline__ void load_pair_negatives(const StepParams &p, unsigned long long pair, uint32_t lane,
-                                                    uint32_t &n0, uint32_t &n1)
-{
-    const int32_t *src = p.l_negs + pair * p.negatives;
-    n0 = 0; n1 = 0;
-    if (lane < p.negatives) n0 = (uint32_t)__ldcg(src + lane);
-    if (lane + 32u < p.negatives) n1 = (uint32_t)__ldcg(src + lane + 32u);
+    if (!LIST) flush_draw_counts(p.st, draws, redraws);
 }
 
 // ---- snapshot mode, pass 1 (Algorithm 1 + the client's aggregation): dots and coefficients ----
@@ -216,8 +231,13 @@ struct Shape {
     static void hogwild(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s)
     {
         if constexpr (VPL * TB <= kMaxRowRegs) {
-            const int grid = grid_for(sgns_hogwild_kernel<VPL, TB>, blocks_per_sm, sms);
-            sgns_hogwild_kernel<VPL, TB><<<grid, kBlock, 0, s>>>(p);
+            if (p.keep_negs) {
+                const int grid = grid_for(sgns_hogwild_kernel<VPL, TB, true>, blocks_per_sm, sms);
+                sgns_hogwild_kernel<VPL, TB, true><<<grid, kBlock, 0, s>>>(p);
+            } else {
+                const int grid = grid_for(sgns_hogwild_kernel<VPL, TB, false>, blocks_per_sm, sms);
+                sgns_hogwild_kernel<VPL, TB, false><<<grid, kBlock, 0, s>>>(p);
+            }
         }
     }
     static void snap_dots(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s)
@@ -275,9 +295,15 @@ int launch_hogwild(const StepParams &p, uint32_t rows_in_flight, uint32_t blocks
 {
     const int vpl = (int)((p.d4 + 31) / 32);
     const int tb = pick_tb(rows_in_flight, vpl, p.negatives);
+    int launched = 1;
+    if (p.keep_negs) {         // the step's negatives, drawn by a launch of their own
+        const int k = launch_draw_negatives(p, const_cast<int32_t *>(p.l_negs), sms * 8, s);
+        if (k < 0) return -1;
+        launched += k;
+    }
     W2V_FOR_VPL(hogwild(p, blocks_per_sm, sms, s))
     if (cudaGetLastError() != cudaSuccess) return -1;
-    return 1;
+    return launched;
 }
 
 int launch_snapshot_apply(const StepParams &p, uint32_t blocks_per_sm, int sms, cudaStream_t s)
@@ -332,7 +358,7 @@ int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t block
     int launched = 1;
     if (!p.keep_negs || !p.l_negs) return -1;
     {                          // the step's negatives, drawn once for both passes
-        const int k = launch_emit_pairs(p, nullptr, nullptr, const_cast<int32_t *>(p.l_negs), ~0ull, sms * 8, s);
+        const int k = launch_draw_negatives(p, const_cast<int32_t *>(p.l_negs), sms * 8, s);
         if (k < 0) return -1;
         launched += k;
     }
