@@ -401,15 +401,19 @@ topk_cosine_tc_kernel(TcParams p)
 // Both sides are converted by pre-passes into global scratch that has exactly the layout of the
 // shared-memory operands ([K-block][16-byte chunk][row][8 bf16]), so the main kernel moves them
 // with bulk copies only and has no loader warps.  The query block stays in shared memory for the
-// whole kernel (d <= 320: 80 KB); candidates stream through eight 16 KB stages (one K-block of 32
-// columns of a 256-candidate tile: two MMAs of K = 16), each filled by one `cp.async.bulk` that a
-// single producer lane issues as soon as the stage's previous MMAs have committed.  The bf16 copy
-// halves what every query block pulls through L2, which is what bounds this kernel.
+// whole kernel (d <= 320: 80 KB); candidates stream through three 48 KB stages (three K-blocks of 32
+// columns of a 256-candidate tile: six MMAs of K = 16), each filled by one `cp.async.bulk` that a
+// single producer lane issues as soon as the stage's previous MMAs have committed.  The stage is
+// that large because one lane hands over a stage every ~330 ns whatever its size (a ring of bulk
+// copies alone, without MMAs, moves 50 GB/s per SM with 16 KB stages at any depth and 99 GB/s with
+// 32 KB stages): with 16 KB stages that hand-over rate, not bytes or MMAs, bounded the kernel
+// (19.0 -> 16.6 ms for 8192 queries x 3 M candidates; 32 KB x 4 and 64 KB x 2 measure the same).
 constexpr float kScreenEps = 8.5e-3f;
 constexpr int kScKB = 32;                                        // columns per stage
 constexpr int kScCh = kScKB / 8;                                 // 16-byte chunks (8 bf16) per row and stage
 constexpr int kScMaxKB = 10;                                     // K-blocks of a query block that can stay in shared memory: d <= 320
-constexpr int kScStages = 8;
+constexpr int kScStages = 3;
+constexpr int kScKPS = 3;                                        // K-blocks per stage (consecutive K-blocks of a tile are contiguous in the packed copy)
 constexpr int kScAChunk = kTcM * 16;                             // query operand, one 16-byte chunk of all rows
 constexpr int kScABlock = kScCh * kScAChunk;                     // bytes of one K-block of the query operand
 constexpr int kScBChunk = kTcN * 16;                             // candidate operand
@@ -525,6 +529,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t (&v)[32], uint32_t taddr)
                  : "r"(taddr));
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
 // Floats as unsigned integers in the same order (0 is below every float): for atomicMax.
 __device__ __forceinline__ unsigned int ordered_bits(float f)
 {
@@ -543,10 +554,10 @@ __global__ void __launch_bounds__(kScThreads, 1)
 topk_cosine_screen_kernel(TcParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    // RES: [kScMaxKB query K-blocks][kScStages candidate stages]; else [kScStages stages of (query K-block, candidate K-block)]
-    constexpr int kStage = RES ? kScStageBytes : kScABlock + kScStageBytes;
+    // RES: [kScMaxKB query K-blocks][kScStages candidate stages]; else [kScStages stages of (kScKPS query K-blocks, kScKPS candidate K-blocks)]
+    constexpr int kStage = kScKPS * (RES ? kScStageBytes : kScABlock + kScStageBytes);
     unsigned char *a_op = smem;
-    unsigned char *b_op = smem + (RES ? kScMaxKB * kScABlock : kScABlock);
+    unsigned char *b_op = smem + (RES ? kScMaxKB * kScABlock : kScKPS * kScABlock);
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + (RES ? kScMaxKB * kScABlock : 0) + kScStages * kStage);
     uint64_t *empty = full + kScStages;
     uint64_t *tfull = empty + kScStages;
@@ -562,6 +573,7 @@ topk_cosine_screen_kernel(TcParams p)
     const uint64_t tiles = (nc + kTcN - 1) / kTcN;
     const uint64_t t_lo = tiles * blockIdx.y / p.splits, t_hi = tiles * (blockIdx.y + 1) / p.splits;
     const uint32_t nkb = (4u * p.d4 + kScKB - 1) / kScKB;
+    const uint32_t nst = (nkb + kScKPS - 1) / kScKPS;                       // stages per tile
     const uint64_t n_tiles = t_hi - t_lo;
 
     if (tid == 0) {
@@ -616,11 +628,18 @@ topk_cosine_screen_kernel(TcParams p)
         auto screen_chunk = [&](const uint32_t (&v)[32], uint32_t cc) {
             __syncwarp();
             const float cut = fmaxf(have < p.K ? p.tau : fmaxf(p.tau, thr), flo) - kScreenEps;
-            float top = __uint_as_float(v[0]);
+            // the largest of the 32 columns, as a tree of three-input maxima (11 + 4 + 1 operations, depth 4)
+            float t1[11];
 #pragma unroll
-            for (int j = 1; j < 32; ++j) top = fmaxf(top, __uint_as_float(v[j]));
+            for (int j = 0; j < 10; ++j) t1[j] = max3(__uint_as_float(v[3 * j]), __uint_as_float(v[3 * j + 1]), __uint_as_float(v[3 * j + 2]));
+            t1[10] = fmaxf(__uint_as_float(v[30]), __uint_as_float(v[31]));
+            const float top = max3(max3(t1[0], t1[1], t1[2]), max3(t1[3], t1[4], t1[5]),
+                                   max3(max3(t1[6], t1[7], t1[8]), t1[9], t1[10]));
+            const bool hit = mine && c0 + cc < nc && top * qinv >= cut;
+            // a chunk with a column near the cut is rare: everything below sits behind one warp-wide branch
+            if (!__any_sync(kFullMask, hit)) return;
             uint32_t maybe = 0u;
-            if (mine && c0 + cc < nc && top * qinv >= cut) {              // rare: which of them?
+            if (hit) {                                                     // which of them?
 #pragma unroll
                 for (int j = 0; j < 32; ++j) maybe |= (__uint_as_float(v[j]) * qinv >= cut ? 1u : 0u) << j;
                 const uint64_t left = nc - (c0 + cc);                      // candidates of the range from column cc on
@@ -749,19 +768,22 @@ topk_cosine_screen_kernel(TcParams p)
                 ok = mbar_wait(tempty + b, (uint32_t)(((i >> 1) & 1) ^ 1), abort_flag);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t dst = tmem_base + b * kTcN;
-                for (uint32_t kb = 0; kb < nkb && ok; ++kb, ++g) {
+                for (uint32_t st = 0; st < nst && ok; ++st, ++g) {
                     const uint32_t s = (uint32_t)(g % kScStages);
                     ok = mbar_wait(full + s, (uint32_t)((g / kScStages) & 1), abort_flag);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t abase = smem_addr(a_op + (RES ? (size_t)kb * kScABlock : (size_t)s * kStage));
-                    const uint32_t bbase = smem_addr(b_op + (size_t)s * kStage);
-                    const uint32_t cols = 4u * p.d4 - kb * kScKB < (uint32_t)kScKB ? 4u * p.d4 - kb * kScKB : (uint32_t)kScKB;
-                    const uint32_t nk = (cols + 15u) / 16u;                              // MMAs of K = 16 columns with data
-                    for (uint32_t kk = 0; kk < nk; ++kk) {
-                        const uint64_t qa = umma_desc(abase + 2 * kk * kScAChunk, kScAChunk, 128);
-                        const uint64_t cb = umma_desc(bbase + 2 * kk * kScBChunk, kScBChunk, 128);
-                        umma_bf16(dst, qa, cb, idesc, (kb | kk) ? 1u : 0u);
+                    for (uint32_t kb = st * kScKPS; kb < nkb && kb < (st + 1) * kScKPS; ++kb) {
+                        const uint32_t j = kb - st * kScKPS;                                 // K-block within the stage
+                        const uint32_t abase = smem_addr(a_op + (RES ? (size_t)kb * kScABlock : (size_t)s * kStage + (size_t)j * kScABlock));
+                        const uint32_t bbase = smem_addr(b_op + (size_t)s * kStage + (size_t)j * kScStageBytes);
+                        const uint32_t cols = 4u * p.d4 - kb * kScKB < (uint32_t)kScKB ? 4u * p.d4 - kb * kScKB : (uint32_t)kScKB;
+                        const uint32_t nk = (cols + 15u) / 16u;                              // MMAs of K = 16 columns with data
+                        for (uint32_t kk = 0; kk < nk; ++kk) {
+                            const uint64_t qa = umma_desc(abase + 2 * kk * kScAChunk, kScAChunk, 128);
+                            const uint64_t cb = umma_desc(bbase + 2 * kk * kScBChunk, kScBChunk, 128);
+                            umma_bf16(dst, qa, cb, idesc, (kb | kk) ? 1u : 0u);
+                        }
                     }
                     umma_commit(empty + s);                       // the stage is free once these MMAs have read it
                 }
@@ -773,18 +795,20 @@ topk_cosine_screen_kernel(TcParams p)
         // one bulk copy per stage, issued when the MMAs that read the stage's previous contents have
         // committed; its bytes complete the stage's "full" barrier
         if (lane == 0) {
-            const uint64_t total_g = n_tiles * nkb;
+            const uint64_t total_g = n_tiles * nst;
             uint64_t g = 0;
             for (; g < total_g; ++g) {
                 const uint32_t s = (uint32_t)(g % kScStages);
                 if (!mbar_wait(empty + s, (uint32_t)(((g / kScStages) & 1) ^ 1), abort_flag)) break;
+                const uint32_t kb0 = (uint32_t)(g % nst) * kScKPS;                               // first K-block of the stage
+                const uint32_t nkbs = nkb - kb0 < (uint32_t)kScKPS ? nkb - kb0 : (uint32_t)kScKPS;  // K-blocks it holds
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
-                             ::"r"(smem_addr(full + s)), "r"((uint32_t)kStage) : "memory");
+                             ::"r"(smem_addr(full + s)), "r"(nkbs * (uint32_t)(RES ? kScStageBytes : kScABlock + kScStageBytes)) : "memory");
                 if (!RES)
-                    bulk_to_smem(a_op + (size_t)s * kStage, p.qsplit + ((size_t)blockIdx.x * nkb + g % nkb) * kScABlock,
-                                 (uint32_t)kScABlock, full + s);
+                    bulk_to_smem(a_op + (size_t)s * kStage, p.qsplit + ((size_t)blockIdx.x * nkb + kb0) * kScABlock,
+                                 nkbs * (uint32_t)kScABlock, full + s);
                 bulk_to_smem(b_op + (size_t)s * kStage,
-                             p.ctiles + ((t_lo + g / nkb) * nkb + g % nkb) * (size_t)kScStageBytes, (uint32_t)kScStageBytes, full + s);
+                             p.ctiles + ((t_lo + g / nst) * nkb + kb0) * (size_t)kScStageBytes, nkbs * (uint32_t)kScStageBytes, full + s);
             }
             if (*abort_flag) {
                 // the block is giving up: let the copies still in flight land before shared memory is released
@@ -806,8 +830,8 @@ topk_cosine_screen_kernel(TcParams p)
 
 static size_t topk_screen_smem_bytes(bool resident)
 {
-    const size_t operands = resident ? (size_t)kScMaxKB * kScABlock + (size_t)kScStages * kScStageBytes
-                                     : (size_t)kScStages * (kScABlock + kScStageBytes);
+    const size_t operands = resident ? (size_t)kScMaxKB * kScABlock + (size_t)kScStages * kScKPS * kScStageBytes
+                                     : (size_t)kScStages * kScKPS * (kScABlock + kScStageBytes);
     return operands + (2 * kScStages + 5) * 8 + 8 + kTcM * 8 + 128;
 }
 
