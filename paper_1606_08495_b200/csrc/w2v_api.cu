@@ -182,7 +182,7 @@ int32_t ensure_error_word(w2v_handle *h)
 // the pair count nor re-allocates.  Larger bounds (wide windows on long chunks) fall back to
 // reading the pair count.
 constexpr uint64_t kSnapshotBoundBudget = 1ull << 30;
-constexpr uint64_t kListChunk = 200000;       // Hogwild mode: chunks of at least this many tokens use a list of negatives
+constexpr uint64_t kListChunk = 500000;       // Hogwild mode: chunks of at least this many tokens use a list of negatives
 
 int32_t check_step_args(w2v_handle *h, const void *tokens, uint64_t n, uint32_t window, uint32_t negatives)
 {
@@ -292,7 +292,7 @@ int32_t step_impl(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t win
     if (rc != W2V_OK) return rc;
     if (mode == W2V_MODE_HOGWILD) {
         // long chunks draw their negatives into a list first (four more launches, a faster update
-        // kernel: measured equal at 0.26 M tokens, 6 % faster at 1 M tokens with 5 negatives), when
+        // kernel: measured equal on the device at 0.26 M tokens but slower end to end, 6 % faster at 1 M tokens with 5 negatives), when
         // the list for the worst case fits the budget
         const uint64_t negs_cap = n * 2ull * window * negatives;
         const bool list = n >= kListChunk && negs_cap * sizeof(int32_t) <= kSnapshotBoundBudget;
