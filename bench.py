@@ -292,6 +292,10 @@ def secondary_modes(model, cfg, dev_chunks, first_step, dev, steps=10, warmup=3)
                                                 allow=(binding.W2V_ERR_CAPACITY,)),
           lambda c, p: algorithmic_bytes_cbow(d, c, p, N), "cbow_hogwild")
     out["cbow_hogwild"]["note"] = "pairs = (centre, context) pairs, i.e. context rows read"
+    timed(lambda t: binding.w2v_cbow_step(model.h, t, t.numel(), W, N, lr, binding.MODE_SNAPSHOT, None),
+          lambda t, st: binding.w2v_sample_cbow(model.h, t, t.numel(), W, N, None, None, 0, st,
+                                                allow=(binding.W2V_ERR_CAPACITY,)),
+          lambda c, p: algorithmic_bytes_cbow(d, c, p, N, True), "cbow_snapshot")
 
     free_b, _ = torch.cuda.mem_get_info(dev)
     if free_b > (5 << 30):

@@ -394,6 +394,17 @@ int32_t w2v_profile_read(w2v_handle *h, double *kernel_ms, uint64_t *launches);
 int32_t w2v_get_launch_count(w2v_handle *h, uint64_t *launches);
 
 /*
+ * Exercises the give-up path of the tensor-core retrieval kernels without a fault (no counterpart
+ * in the paper: a diagnostic).  Those kernels hand shared-memory stages and accumulators over with
+ * barriers, and every wait has a time limit so that a lost hand-over can never hang the GPU; this
+ * call enqueues one block that waits, with the same routine, `timeout_ms` (1..2000) on a barrier
+ * that nobody arrives at.  The wait runs out, the block raises the handle's error word and returns;
+ * the next w2v_sync returns W2V_ERR_CUDA once, and the stream and the device stay usable.
+ * Asynchronous.
+ */
+int32_t w2v_selftest_bounded_wait(w2v_handle *h, uint32_t timeout_ms);
+
+/*
  * Memory-system ceiling for the step's access patterns (no counterpart in the paper: a measuring
  * aid; Section 6 of the paper names the random cache-line rate as what bounds a shard).  Touches
  * `rows` pseudo-random rows of the output table V, drawn uniformly from rows [0, span_rows), with

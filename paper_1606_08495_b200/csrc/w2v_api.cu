@@ -918,6 +918,19 @@ int32_t w2v_sync(w2v_handle *h)
     return W2V_OK;
 }
 
+int32_t w2v_selftest_bounded_wait(w2v_handle *h, uint32_t timeout_ms)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (timeout_ms < 1 || timeout_ms > 2000) return fail(h, W2V_ERR_ARG, "timeout_ms must be in 1..2000");
+    DeviceGuard g(h->device);
+    int32_t rc;
+    if ((rc = ensure_error_word(h)) != W2V_OK) return rc;
+    const int k = launch_bounded_wait_selftest(timeout_ms, h->tc_error, h->stream);
+    if (k < 0) return fail(h, W2V_ERR_CUDA, "self-test launch", cudaGetLastError());
+    h->launches += (uint64_t)k;
+    return W2V_OK;
+}
+
 int32_t w2v_set_retrieval_kernel(w2v_handle *h, uint32_t kind)
 {
     if (!h) return W2V_ERR_ARG;

@@ -172,6 +172,8 @@ int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, 
 // size, each with its own partial lists); bytes of the packed bf16 copy of one chunk.
 uint64_t topk_screen_chunk(uint64_t n_candidates, uint32_t d);
 size_t topk_screen_ctiles_bytes(uint64_t n_candidates, uint32_t d);
+// one block that waits `timeout_ms` on a barrier nobody arrives at and then raises *error (w2v_topk_tc.cu)
+int launch_bounded_wait_selftest(uint32_t timeout_ms, int *error, cudaStream_t s);
 int launch_inv_norms(const float *table, uint32_t d, uint32_t ld, uint64_t lo, uint64_t count, float *inv_norm,
                      int sms, cudaStream_t s);
 // Returns launches made, -1 on a launch error, -2 if the shape does not fit shared memory.

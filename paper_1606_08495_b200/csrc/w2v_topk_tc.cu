@@ -67,14 +67,15 @@ __device__ __forceinline__ unsigned long long global_ns()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                          unsigned long long limit_ns = kTcWaitNs)
 {
     const unsigned long long t0 = global_ns();
     for (uint32_t spin = 0; spin < (1u << 30); ++spin) {
         if (mbar_try(bar, parity)) return true;
         if ((spin & 1023u) == 1023u) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > kTcWaitNs) break;
+            if (global_ns() - t0 > limit_ns) break;
         }
     }
     *abort_flag = 1;
@@ -826,6 +827,34 @@ topk_cosine_screen_kernel(TcParams p)
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * kTcN));
     }
+}
+
+// The give-up path of the retrieval kernels on its own: one block waits, with the kernels' own wait
+// routine and a short limit, on a barrier that nobody arrives at; when the limit has passed it raises
+// the error word exactly as a retrieval block does, and returns.
+__global__ void __launch_bounds__(64)
+bounded_wait_selftest_kernel(unsigned long long limit_ns, int *error)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_word;
+    volatile int *abort_flag = &abort_word;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    // lane 0 of warp 0 waits for the arrival that never comes; lane 0 of warp 1 waits behind it and must
+    // leave through the abort flag as soon as the first has given up
+    if ((threadIdx.x & 31) == 0) mbar_wait(&bar, 0u, abort_flag, threadIdx.x == 0 ? limit_ns : 100 * limit_ns);
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) atomicExch(error, 1);
+}
+
+int launch_bounded_wait_selftest(uint32_t timeout_ms, int *error, cudaStream_t s)
+{
+    bounded_wait_selftest_kernel<<<1, 64, 0, s>>>((unsigned long long)timeout_ms * 1000000ull, error);
+    return cudaGetLastError() != cudaSuccess ? -1 : 1;
 }
 
 static size_t topk_screen_smem_bytes(bool resident)

@@ -155,3 +155,23 @@ def test_topk_rows_that_are_all_alike(kernel):
     check(gpu, cpu, X, 0, q, 0, V, 10, -2.0, tolerance(kernel, d))
     check(gpu, cpu, X, 0, q, 100, 3000, 30, 0.999, tolerance(kernel, d))
     gpu.close()
+
+
+def test_a_wait_that_runs_out_is_reported_once_and_nothing_faults():
+    # the retrieval kernels' bounded wait on a barrier nobody arrives at: the block gives up after the
+    # limit, w2v_sync reports it once, and the same handle goes on to answer a query correctly
+    import time
+    gpu, cpu, X = pair(500, 32, seed=4, kernel=2)
+    t0 = time.time()
+    binding.w2v_selftest_bounded_wait(gpu.h, 250)
+    with pytest.raises(binding.W2VError) as e:
+        gpu.sync()
+    waited = time.time() - t0
+    assert e.value.code == binding.W2V_ERR_CUDA and "gave up waiting" in str(e.value)
+    assert 0.2 <= waited < 3.0, waited
+    gpu.sync()                                            # reported once
+    check(gpu, cpu, X, 0, np.arange(40), 0, 500, 5, -2.0, tolerance(2, 32))
+    with pytest.raises(binding.W2VError) as e:
+        binding.w2v_selftest_bounded_wait(gpu.h, 0)
+    assert e.value.code == binding.W2V_ERR_ARG
+    gpu.close()
