@@ -71,7 +71,7 @@ typedef struct {
     uint64_t neg_draws;    /* alias-table draws, re-draws included */
     uint64_t neg_redraws;  /* draws thrown away because they hit the context word */
     uint64_t oov;          /* ids outside [-1, vocab) */
-    uint32_t status;       /* bit 0: out-of-vocabulary ids seen */
+    uint32_t status;       /* bit 0: out-of-vocabulary ids seen; bit 1: a time-limited wait inside a kernel ran out (W2V_ERR_CUDA) */
     uint32_t reserved;
 } w2v_step_stats;
 

@@ -339,6 +339,7 @@ int32_t step_impl(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t win
     h->step_id += 1;
     if (stats) {
         if ((rc = read_state(h, n, stats)) != W2V_OK) return rc;
+        if (stats->status & 2u) return fail(h, W2V_ERR_CUDA, "a copy into shared memory did not arrive in time; the step is incomplete");
         if (stats->status & 1u) return fail(h, W2V_ERR_TOKEN_RANGE, "token ids outside [-1, vocab) were skipped");
     }
     return W2V_OK;

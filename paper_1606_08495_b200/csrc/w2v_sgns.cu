@@ -130,6 +130,191 @@ sgns_snap_dots_kernel(StepParams p)
     }
 }
 
+// ---- snapshot mode, pass 1 with the target rows staged in shared memory -----------------------
+// The register-staged kernel above holds four rows per warp in flight (48 of its 128 registers),
+// 64 per SM, and a read-only gather wants more than that.  Here the rows of a warp's targets arrive
+// by `cp.async.bulk` in a ring of NG groups of RR slots in shared memory, one mbarrier per group: while
+// group g is reduced from shared memory, groups g+1 .. g+NG-1 are in flight, also across the boundary
+// between two centres, and no register holds a row that is still on its way.  The warp is
+// its own producer: after it has consumed a group it arms the barrier and lets lanes 0..3 issue
+// the copies of the group NG-1 ahead.  Two cursors walk the same sequence of (centre, group of
+// targets): the issuing one ahead, the consuming one behind.  Every wait has a time limit, after
+// which the warp raises status bit 1 and stops issuing and consuming (nothing is left in flight
+// into shared memory that is still being waited for by anyone else: the block ends together).
+constexpr int kRingMaxGroups = 8;
+constexpr unsigned long long kRingWaitNs = 2000000000ull;
+
+__device__ __forceinline__ uint32_t ring_saddr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+struct RingCursor {
+    uint32_t q;            // kept position of the centre
+    uint32_t left, cnt;    // contexts to the left / in all
+    uint32_t k;            // next target of the centre, 0 .. cnt * (1 + N)
+    unsigned long long pair0;
+    bool done;
+};
+
+// moves the cursor to the next centre (at or after q) that has a context
+__device__ __forceinline__ void ring_seek(const StepParams &p, RingCursor &c, uint32_t nk, uint32_t nwarps)
+{
+    for (; c.q < nk; c.q += nwarps) {
+        const uint32_t w = p.win[c.q];
+        c.left = w & 0xFFu; c.cnt = c.left + (w >> 8);
+        if (c.cnt) { c.pair0 = p.pair_off[c.q]; c.k = 0; return; }
+    }
+    c.done = true;
+}
+
+// RR: rows per group (= per barrier); BT: threads of the one block per SM (all of its shared memory is ring)
+template <int VPL, int RR, int BT>
+__global__ void __launch_bounds__(BT, 1)
+sgns_snap_dots_ring_kernel(StepParams p, uint32_t ngroups, uint32_t slot_bytes)
+{
+    constexpr int kRingRows = RR, kRingBlock = BT;
+    extern __shared__ __align__(128) unsigned char ring_smem[];
+    const uint32_t lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    const uint32_t nk = (uint32_t)p.st->n_kept;
+    const uint32_t n1p = p.negatives + 1u;
+    const uint32_t group_bytes = kRingRows * slot_bytes;
+    unsigned char *slots = ring_smem + (size_t)wib * ngroups * group_bytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(ring_smem + (size_t)(kRingBlock / 32) * ngroups * group_bytes) + wib * kRingMaxGroups;
+    const float4 *U4 = reinterpret_cast<const float4 *>(p.U);
+    const float4 *V4 = reinterpret_cast<const float4 *>(p.V);
+    float4 *DU4 = reinterpret_cast<float4 *>(p.DU);
+    if (lane == 0)
+        for (uint32_t g = 0; g < ngroups; ++g)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(ring_saddr(bars + g)), "r"(1));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncwarp();
+
+    RingCursor is, co;                         // issuing and consuming cursor
+    is.q = co.q = warp; is.done = co.done = false; is.k = co.k = 0; is.left = is.cnt = co.left = co.cnt = 0; is.pair0 = co.pair0 = 0;
+    ring_seek(p, is, nk, nwarps);
+    co = is;
+    uint32_t issued = 0, consumed = 0;
+    bool failed = false;
+
+    // The next group of the issuing cursor (at most kRingRows targets of one centre) in two steps, so that
+    // the loads of the target numbers are not waited for where they are issued: plan_group() reads them
+    // for the group after the one that issue_group() sends off.
+    uint32_t pl_rows = 0, pl_tgt = 0;
+    auto plan_group = [&]() {
+        pl_rows = 0;
+        if (is.done) return;
+        const uint32_t nt = is.cnt * n1p;
+        pl_rows = nt - is.k < (uint32_t)kRingRows ? nt - is.k : (uint32_t)kRingRows;
+        if (lane < pl_rows) {
+            const uint32_t k = is.k + lane, pr = k / n1p, t = k - pr * n1p;
+            const uint32_t pp = is.q - is.left + pr + (pr >= is.left ? 1u : 0u);
+            pl_tgt = t == 0 ? (uint32_t)p.ctok[pp] : (uint32_t)__ldcg(p.l_negs + (is.pair0 + pr) * p.negatives + (t - 1u));
+        }
+        is.k += pl_rows;
+        if (is.k >= nt) { is.q += nwarps; ring_seek(p, is, nk, nwarps); }
+    };
+    auto issue_group = [&]() {
+        const uint32_t rows = pl_rows, tgt = pl_tgt, gi = issued % ngroups;
+        // the slots were read with ordinary loads; the copies write them through the async proxy
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        if (lane == 0)
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                         ::"r"(ring_saddr(bars + gi)), "r"(rows * 16u * p.d4) : "memory");
+        __syncwarp();
+        if (lane < rows)
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(ring_saddr(slots + (size_t)gi * group_bytes + (size_t)lane * slot_bytes)),
+                           "l"(V4 + (size_t)tgt * p.ld4), "r"(16u * p.d4), "r"(ring_saddr(bars + gi)) : "memory");
+        ++issued;
+        plan_group();
+    };
+
+    plan_group();
+    for (uint32_t g = 0; g + 1 < ngroups && pl_rows; ++g) issue_group();
+    Row<VPL> u, du;
+    row_zero(u); row_zero(du);
+    while (!co.done && !failed) {
+        if (pl_rows) issue_group();
+        if (co.k == 0) {                       // a new centre
+            row_load(u, U4 + (size_t)(uint32_t)p.ctok[co.q] * p.ld4, p.d4, lane);
+            row_zero(du);
+        }
+        // wait for the group's rows
+        const uint32_t gi = consumed % ngroups, parity = (consumed / ngroups) & 1u;
+        {
+            unsigned long long t0 = 0;
+            for (uint32_t spin = 0;; ++spin) {
+                uint32_t ok;
+                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                             : "=r"(ok) : "r"(ring_saddr(bars + gi)), "r"(parity) : "memory");
+                if (ok) break;
+                if ((spin & 255u) == 255u) {
+                    unsigned long long now;
+                    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+                    if (t0 == 0) t0 = now;
+                    else if (now - t0 > kRingWaitNs) { failed = true; break; }
+                }
+            }
+            failed = __any_sync(kFullMask, failed);
+            if (failed) break;
+        }
+        const uint32_t nt = co.cnt * n1p;
+        const uint32_t rows = nt - co.k < (uint32_t)kRingRows ? nt - co.k : (uint32_t)kRingRows;
+        const float4 *slot = reinterpret_cast<const float4 *>(slots + (size_t)gi * group_bytes);
+        Row<VPL> v[kRingRows];
+        float f[kRingRows];
+#pragma unroll
+        for (int b = 0; b < kRingRows; ++b) {
+#pragma unroll
+            for (int j = 0; j < VPL; ++j) {
+                const uint32_t idx = lane + 32u * j;
+                v[b].x[j] = ((uint32_t)b < rows && idx < p.d4) ? slot[(size_t)b * (slot_bytes / 16u) + idx] : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            f[b] = row_dot_partial(u, v[b]);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+            for (int b = 0; b < kRingRows; ++b) f[b] += __shfl_xor_sync(kFullMask, f[b], o);
+        }
+        const unsigned long long gbase = co.pair0 * n1p + co.k;
+#pragma unroll
+        for (int b = 0; b < kRingRows; ++b) {
+            if ((uint32_t)b < rows) {
+                const uint32_t t = (co.k + b) % n1p;
+                const float sg = sigmoidf_exact(f[b]);
+                const float g = t == 0 ? p.lr * (1.0f - sg) : -p.lr * sg;
+                if (lane == (uint32_t)b) p.G[gbase + b] = g;
+                row_axpy(du, g, v[b]);
+            }
+        }
+        ++consumed;
+        co.k += rows;
+        if (co.k >= nt) {
+#pragma unroll
+            for (int j = 0; j < VPL; ++j) {
+                const uint32_t idx = lane + 32u * j;
+                if (idx < p.d4) DU4[(size_t)co.q * p.d4 + idx] = du.x[j];
+            }
+            co.q += nwarps;
+            ring_seek(p, co, nk, nwarps);
+        }
+    }
+    if (failed) {
+        // copies already issued may still land: give them their time before the block's shared memory goes away
+        for (uint32_t g = consumed; g < issued; ++g) {
+            const uint32_t gi = g % ngroups, parity = (g / ngroups) & 1u;
+            for (uint32_t spin = 0; spin < (1u << 20); ++spin) {
+                uint32_t ok;
+                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                             : "=r"(ok) : "r"(ring_saddr(bars + gi)), "r"(parity) : "memory");
+                if (ok) break;
+            }
+        }
+        if (lane == 0) atomicOr(&p.st->status, 2u);
+    }
+}
+
 // ---- snapshot mode, pass 2 (Algorithm 2, output rows): v(target) += G u(c) ------------------
 // U is still untouched, so u(c) is the start-of-step vector; V is only added to (adjust_targets).
 // The negatives are read back from pass 1's list when there is one (a draw costs a random read of the
@@ -350,6 +535,36 @@ int launch_snapshot_tail(const StepParams &p, uint32_t blocks_per_sm, int sms, c
     return launched;
 }
 
+// Pass 1 with the shared-memory ring, when at least three groups of rows fit a warp's share of the SM's
+// shared memory (d <= 512) and the caller has not asked for a register shape; false = not launched.
+template <int VPL, int RR, int BT>
+static bool snap_dots_ring_for(const StepParams &p, int sms, cudaStream_t s)
+{
+    const uint32_t slot = 16u * p.d4;
+    const size_t budget = 220u * 1024u, bars = (size_t)(BT / 32) * kRingMaxGroups * 8;
+    uint32_t ng = (uint32_t)((budget - bars) / (BT / 32) / ((size_t)RR * slot));
+    if (ng > (uint32_t)kRingMaxGroups) ng = kRingMaxGroups;
+    if (ng < 2) return false;
+    const size_t sm = (size_t)(BT / 32) * ng * RR * slot + bars;
+    if (cudaFuncSetAttribute(sgns_snap_dots_ring_kernel<VPL, RR, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    sgns_snap_dots_ring_kernel<VPL, RR, BT><<<sms, BT, sm, s>>>(p, ng, slot);
+    return true;
+}
+
+// Instantiated for rows of 260..384 columns (the paper's d = 300): 16 warps per SM, groups of four rows,
+// two groups per warp (measured on the 60 M x 300 workload: 10.9 ms against 12.3 ms for the register-staged
+// kernel; eight or twelve warps, or groups of two or three rows, are slower: the per-group work of the warp,
+// not the bytes in flight, is then the limit).  Other widths keep the register-staged kernel.
+static bool launch_snap_dots_ring(const StepParams &p, uint32_t rows_in_flight, int sms, cudaStream_t s)
+{
+    if (rows_in_flight) return false;                       // the caller asked for a register shape
+    if ((p.d4 + 31) / 32 != 3) return false;
+    return snap_dots_ring_for<3, 4, 512>(p, sms, s);
+}
+
 int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t blocks_per_sm, int sms,
                     cudaStream_t s)
 {
@@ -362,7 +577,9 @@ int launch_snapshot(const StepParams &p, uint32_t rows_in_flight, uint32_t block
         if (k < 0) return -1;
         launched += k;
     }
-    W2V_FOR_VPL(snap_dots(p, blocks_per_sm, sms, s))
+    if (!launch_snap_dots_ring(p, rows_in_flight, sms, s)) {
+        W2V_FOR_VPL(snap_dots(p, blocks_per_sm, sms, s))
+    }
     if (cudaGetLastError() != cudaSuccess) return -1;
     const int k = launch_snapshot_apply(p, blocks_per_sm, sms, s);
     return k < 0 ? -1 : launched + k;

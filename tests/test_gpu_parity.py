@@ -178,8 +178,10 @@ def test_read_write_rows_roundtrip():
 
 
 # ---------------------------------------------------------------- snapshot mode
-def check_snapshot_steps(cfg, steps, words=None, seed=11, row_stride=None):
+def check_snapshot_steps(cfg, steps, words=None, seed=11, row_stride=None, tuning=None):
     gpu, cpu, cp = make_pair(cfg, seed=seed, row_stride=row_stride)
+    if tuning is not None:
+        gpu.set_tuning(*tuning)
     W, N, lr = cfg["window"], cfg["negatives"], cfg["lr"]
     worst = 0.0
     for i in range(steps):
@@ -227,6 +229,16 @@ def test_snapshot_other_negative_counts(N, W):
     # more targets per pair than one batch of row touches (12), than one register of draws per lane (32)
     cfg = corpus.scaled(TINY, vocab=3000, d=100, negatives=N, window=W, minibatch=400, corpus_tokens=60_000)
     check_snapshot_steps(cfg, steps=2)
+
+
+@pytest.mark.parametrize("d,N,W,tuned", [(300, 10, 5, False), (300, 10, 5, True), (260, 1, 3, False), (384, 13, 2, False),
+                                         (300, 64, 1, False), (320, 5, 127, False)])
+def test_snapshot_rows_of_the_papers_width(d, N, W, tuned):
+    # rows of 260..384 columns take pass 1 through the shared-memory ring (bulk copies, groups of four
+    # rows that also run across the boundary between two centres); a requested register shape
+    # (tuned) takes the other kernel: both must give the checker's step
+    cfg = corpus.scaled(TINY, vocab=3000, d=d, negatives=N, window=W, minibatch=1200, corpus_tokens=80_000)
+    check_snapshot_steps(cfg, steps=2, tuning=(4, 0) if tuned else None)
 
 
 @pytest.mark.parametrize("d,row_stride", [(300, 320), (300, 304), (100, 128), (8, 16), (132, 2048)])
