@@ -614,7 +614,7 @@ def run_topk(args):
     lo, hi = int(V * 0.85), V
     model = binding.W2V(V, d, seed=1, device=dev, row_stride=row_stride_for(d, args.row_stride))
     tensor = args.retrieval_kernel != "fp32"
-    binding.w2v_set_retrieval_kernel(model.h, {"fp32": 0, "tensor": 1, "screen": 2}[args.retrieval_kernel])
+    binding.w2v_set_retrieval_kernel(model.h, {"fp32": 0, "tensor": 1, "screen": 2, "pairs": 3}[args.retrieval_kernel])
     # stand-in for trained vectors: clustered rows (centre + noise), so that queries have neighbours above
     # tau and the lists fill; --unrelated-rows keeps the earlier i.i.d. normal rows (nothing reaches tau = 0.65:
     # pure screening).  Written by torch: this is input data.
@@ -692,6 +692,7 @@ def run_topk(args):
                    "candidates": hi - lo, "K": K, "tau": tau, "row_stride_floats": model.row_stride,
                    "kernel": {"tensor": "tcgen05 tf32, head/tail split (3 MMAs per product)",
                               "screen": "tcgen05 bf16 screen (1 MMA per product) + exact fp32 cosines near the cut",
+                              "pairs": "the same screen with cta_group::2 MMAs on pairs of SMs",
                               "fp32": "fp32 CUDA cores"}[args.retrieval_kernel],
                    "rows": "i.i.d. normal (no neighbours)" if args.unrelated_rows else "clustered (centre + noise): lists fill",
                    "lists_full": float(((ids.view(m, K) >= 0).sum(dim=1) == K).float().mean()),
@@ -701,6 +702,7 @@ def run_topk(args):
                 "d2h_bytes_per_step": 12 * m * K},
         "gpu_launches": launches,
         "roofline": {"bound": bound, "kernel": {"tensor": "topk_cosine_tc_kernel", "screen": "topk_cosine_screen_kernel",
+                                                "pairs": "topk_cosine_screen_pair_kernel",
                                                 "fp32": "topk_cosine_kernel"}[args.retrieval_kernel],
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "mma_tflops_issued": mma_per_product * achieved if tensor else None,
@@ -769,7 +771,7 @@ def main():
     ap.add_argument("--ref-words", type=int, default=20_000, help="word tokens per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--queries", type=int, default=8192, help="query rows per call of --mode topk")
-    ap.add_argument("--retrieval-kernel", choices=["fp32", "tensor", "screen"], default="screen")
+    ap.add_argument("--retrieval-kernel", choices=["fp32", "tensor", "screen", "pairs"], default="screen")
     ap.add_argument("--tau", type=float, default=0.65, help="similarity threshold of --mode topk (-2 keeps everything)")
     ap.add_argument("--probe-rows", type=int, default=20_000_000, help="--mode probe: rows touched per launch")
     ap.add_argument("--probe-span", type=int, default=18_000_000,

@@ -24,7 +24,7 @@ struct w2v_handle {
     uint64_t l_cap_pairs = 0, l_cap_negs = 0;
     float *inv_norm = nullptr; uint64_t inv_norm_cap = 0;                      // retrieval scratch
     float *part_cos = nullptr; long long *part_ids = nullptr; uint64_t part_cap = 0;
-    uint32_t retrieval_kernel = 2;       // 0: fp32 on the CUDA cores, 1: tensor cores (3 x TF32), 2: tensor-core screen + exact fp32
+    uint32_t retrieval_kernel = 2;       // 0: fp32 on the CUDA cores, 1: tensor cores (3 x TF32), 2: tensor-core screen + exact fp32, 3: the screen on pairs of SMs
     int *tc_error = nullptr;             // device word raised by a tensor-core block whose wait ran out
     unsigned char *qsplit = nullptr; uint64_t qsplit_cap = 0;   // query rows split into TF32 head and tail
     unsigned char *ctiles = nullptr; uint64_t ctiles_cap = 0;   // candidate rows packed as bf16 operand blocks (screening kernel)
@@ -764,7 +764,7 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
     }
     // few query blocks: split the candidates over several blocks per query block, merge afterwards
     const bool tc = h->retrieval_kernel >= 1;
-    const bool screen = h->retrieval_kernel == 2;
+    const bool screen = h->retrieval_kernel >= 2;
     // the screening kernel takes the candidates in chunks, each with its own set of partial lists
     const uint64_t chunk = screen ? topk_screen_chunk(nc, h->d) : nc;
     const uint64_t chunks = chunk ? (nc + chunk - 1) / chunk : 0;
@@ -807,7 +807,7 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
     if (tc) {
         k2 = launch_topk_tc(table, h->d, h->ld, h->vocab, reinterpret_cast<const long long *>(queries), m, cand_lo,
                             cand_hi, K, tau, h->inv_norm, h->qsplit, h->ctiles, h->floor_q, h->part_cos, h->part_ids, (uint32_t)splits,
-                            h->tc_error, screen, h->sms, h->stream);
+                            h->tc_error, screen, h->retrieval_kernel == 3, h->sms, h->stream);
         if (k2 >= 0) {
             const int k3 = launch_topk_merge(h->part_cos, h->part_ids, m, K, (uint32_t)lists, out_cos,
                                              reinterpret_cast<long long *>(out_ids), h->sms, h->stream);
@@ -935,7 +935,7 @@ int32_t w2v_selftest_bounded_wait(w2v_handle *h, uint32_t timeout_ms)
 int32_t w2v_set_retrieval_kernel(w2v_handle *h, uint32_t kind)
 {
     if (!h) return W2V_ERR_ARG;
-    if (kind > 2) return fail(h, W2V_ERR_ARG, "kind must be 0 (fp32 CUDA cores), 1 (tensor cores) or 2 (tensor-core screen)");
+    if (kind > 3) return fail(h, W2V_ERR_ARG, "kind must be 0 (fp32 CUDA cores), 1 (tensor cores), 2 (tensor-core screen) or 3 (screen on pairs of SMs)");
     h->retrieval_kernel = kind;
     return W2V_OK;
 }

@@ -165,7 +165,7 @@ size_t topk_tc_qsplit_bytes(uint64_t m, uint32_t d);
 int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, const long long *queries, uint64_t m,
                    uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, float *inv_norm,
                    unsigned char *qsplit, unsigned char *ctiles, unsigned int *floor_q, float *part_cos, long long *part_ids,
-                   uint32_t splits, int *error, bool screen, int sms, cudaStream_t s);
+                   uint32_t splits, int *error, bool screen, bool pairs, int sms, cudaStream_t s);
 // inv_norm: 1/|row| of the candidates, an input for the three-MMA kernel (launch_inv_norms); the screening
 // variant computes it itself while it packs the candidates.
 // The screening variant: how many candidates it handles per launch (a range is cut into chunks of that

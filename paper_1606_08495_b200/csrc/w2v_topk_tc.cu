@@ -454,19 +454,21 @@ topk_round_queries_kernel(const float *__restrict__ table, const long long *__re
 }
 
 // Candidate rows cand_lo + [0, nc), scaled to unit length, as bf16 operand blocks:
-// [tile of 256 rows][K-block][chunk][row][8 bf16], zeros past the end of the range and of the row;
+// [tile of NT rows][K-block][chunk][row][8 bf16] for `tiles` tiles, zeros past the end of the range and of
+// the row (NT = 256 for the one-block kernel, 128 for the pair kernel, whose blocks take a half tile each);
 // inv_norm[c] = 1/|row c| (0 for a zero row) is written on the way, for the exact cosines.
 // One block per tile, one thread per row: a thread reads its row once for the norm and once more,
-// 128 bytes (one K-block) at a time through L1 and L2, for the operand; the 256 threads' 16-byte
+// 128 bytes (one K-block) at a time through L1 and L2, for the operand; the NT threads' 16-byte
 // stores of one chunk are contiguous.
-__global__ void __launch_bounds__(kTcN)
+template <int NT>
+__global__ void __launch_bounds__(NT)
 topk_pack_candidates_kernel(const float *__restrict__ table, float *__restrict__ inv_norm, uint32_t d4, uint32_t ld4,
-                            uint64_t cand_lo, uint64_t nc, uint32_t nkb, unsigned char *__restrict__ out)
+                            uint64_t cand_lo, uint64_t nc, uint64_t tiles, uint32_t nkb, unsigned char *__restrict__ out)
 {
-    const uint64_t tiles = (nc + kTcN - 1) / kTcN;
+    constexpr int kBChunk = NT * 16, kBStage = kScCh * kBChunk;
     const uint32_t r = threadIdx.x;
     for (uint64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-        const uint64_t c = tile * kTcN + r;
+        const uint64_t c = tile * NT + r;
         const bool valid = c < nc;
         const float4 *row = reinterpret_cast<const float4 *>(table) + (size_t)(cand_lo + (valid ? c : 0)) * ld4;
         float ic = 0.f;                                            // unit rows: an accumulator column times 1/|query| is a cosine
@@ -480,14 +482,14 @@ topk_pack_candidates_kernel(const float *__restrict__ table, float *__restrict__
             inv_norm[c] = ic;
         }
         for (uint32_t kb = 0; kb < nkb; ++kb) {
-            unsigned char *dst = out + (tile * nkb + kb) * (size_t)kScStageBytes + r * 16;
+            unsigned char *dst = out + (tile * nkb + kb) * (size_t)kBStage + r * 16;
 #pragma unroll
             for (int ch = 0; ch < kScCh; ++ch) {
                 const uint32_t c4 = kb * (kScKB / 4) + 2 * ch;
                 float4 x = make_float4(0.f, 0.f, 0.f, 0.f), y = x;
                 if (valid && c4 < d4) x = __ldg(row + c4);
                 if (valid && c4 + 1 < d4) y = __ldg(row + c4 + 1);
-                *reinterpret_cast<uint4 *>(dst + ch * kScBChunk) =
+                *reinterpret_cast<uint4 *>(dst + ch * kBChunk) =
                     make_uint4(bf16x2(x.x * ic, x.y * ic), bf16x2(x.z * ic, x.w * ic), bf16x2(y.x * ic, y.y * ic), bf16x2(y.z * ic, y.w * ic));
             }
         }
@@ -548,6 +550,166 @@ __device__ __forceinline__ float ordered_float(unsigned int o)
     return __uint_as_float((o & 0x80000000u) ? (o & 0x7FFFFFFFu) : ~o);
 }
 
+// ================= epilogue of the screening kernels: one thread per query row =================
+// Called by the four epilogue warps (threads 0..127) of a block whose accumulators (two buffers of
+// 256 columns) start at tmem_base; `list` is the number of the partial list the block fills;
+// arrive_tempty(b) tells the MMA issuer that this thread is done with accumulator buffer b.
+template <typename Arrive>
+__device__ __forceinline__ void screen_epilogue(const TcParams &p, const long long *qrow, uint64_t q0, uint64_t nc, uint64_t t_lo,
+                                                uint64_t n_tiles, uint32_t tmem_base, uint64_t *tfull, volatile int *abort_flag,
+                                                uint32_t list, Arrive &&arrive_tempty)
+{
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t r = tid;
+    const long long my_q = qrow[r];
+    const bool live = q0 + r < p.m;
+    const float4 *T4 = reinterpret_cast<const float4 *>(p.table);
+    float *lc = p.part_cos + ((size_t)list * p.m + (q0 + r)) * p.K;      // this query's list (global, private)
+    long long *li = p.part_ids + ((size_t)list * p.m + (q0 + r)) * p.K;
+    float qinv = 0.f;
+    if (my_q >= 0) {
+        const float4 *row = T4 + (size_t)my_q * p.ld4;
+        float s = 0.f;
+        for (uint32_t j = 0; j < p.d4; ++j) {
+            const float4 x = __ldcg(row + j);
+            s = fmaf(x.x, x.x, s); s = fmaf(x.y, x.y, s); s = fmaf(x.z, x.z, s); s = fmaf(x.w, x.w, s);
+        }
+        qinv = s > 0.f ? 1.0f / sqrtf(s) : 0.f;
+    }
+    if (live) for (uint32_t s = 0; s < p.K; ++s) { lc[s] = 0.f; li[s] = -1; }
+    const bool mine = my_q >= 0 && live;
+    uint32_t have = 0;
+    float thr = p.tau;
+    // The blocks that work on other candidates of the same queries publish the K-th best cosine they
+    // have reached (floor_q, raised by atomicMax); K candidates at or above it exist, so whatever is
+    // below it cannot be among the query's final K, in any block.  Read once per tile.
+    float flo = -INFINITY;
+    // one chunk of 32 columns of the current tile (first candidate c0 + cc)
+    uint64_t c0 = 0;
+    auto screen_chunk = [&](const uint32_t (&v)[32], uint32_t cc) {
+        __syncwarp();
+        const float cut = fmaxf(have < p.K ? p.tau : fmaxf(p.tau, thr), flo) - kScreenEps;
+        // the largest of the 32 columns, as a tree of three-input maxima (11 + 4 + 1 operations, depth 4)
+        float t1[11];
+#pragma unroll
+        for (int j = 0; j < 10; ++j) t1[j] = max3(__uint_as_float(v[3 * j]), __uint_as_float(v[3 * j + 1]), __uint_as_float(v[3 * j + 2]));
+        t1[10] = fmaxf(__uint_as_float(v[30]), __uint_as_float(v[31]));
+        const float top = max3(max3(t1[0], t1[1], t1[2]), max3(t1[3], t1[4], t1[5]),
+                               max3(max3(t1[6], t1[7], t1[8]), t1[9], t1[10]));
+        const bool hit = mine && c0 + cc < nc && top * qinv >= cut;
+        // a chunk with a column near the cut is rare: everything below sits behind one warp-wide branch
+        if (!__any_sync(kFullMask, hit)) return;
+        uint32_t maybe = 0u;
+        if (hit) {                                                     // which of them?
+#pragma unroll
+            for (int j = 0; j < 32; ++j) maybe |= (__uint_as_float(v[j]) * qinv >= cut ? 1u : 0u) << j;
+            const uint64_t left = nc - (c0 + cc);                      // candidates of the range from column cc on
+            if (left < 32) maybe &= (1u << (uint32_t)left) - 1u;
+        }
+        // Exact pass: the set bits of all lanes, up to kExact queries (lanes) at a time.  The whole warp
+        // works on each (query, candidate): 32 lanes on the fp32 dot product of the two table rows
+        // (the loads of all kExact pairs are issued before the first sum is reduced), then on the
+        // insertion into that query's sorted list, lane l holding entries l and l + 32.
+        for (;;) {
+            uint32_t owners = __ballot_sync(kFullMask, maybe != 0u);
+            if (!owners) break;
+            bool on[kExact];
+            uint32_t src[kExact], hv[kExact];
+            float th[kExact], fl[kExact], qi[kExact], dot[kExact], e0[kExact], e1[kExact];
+            long long i0[kExact], i1[kExact], qr[kExact];
+            uint64_t cnd[kExact];
+#pragma unroll
+            for (int e = 0; e < kExact; ++e) {
+                on[e] = owners != 0u;
+                src[e] = on[e] ? (uint32_t)__ffs((int)owners) - 1u : 0u;
+                owners &= owners - 1u;
+                const uint32_t j = __shfl_sync(kFullMask, (uint32_t)__ffs((int)maybe) - 1u, src[e]);
+                cnd[e] = c0 + cc + j;
+                qr[e] = qrow[warp * 32u + src[e]];
+                hv[e] = __shfl_sync(kFullMask, have, src[e]);
+                th[e] = __shfl_sync(kFullMask, thr, src[e]);
+                fl[e] = __shfl_sync(kFullMask, flo, src[e]);
+                qi[e] = __shfl_sync(kFullMask, qinv, src[e]);
+                if (on[e] && lane == src[e]) maybe &= maybe - 1u;
+                e0[e] = 0.f; e1[e] = 0.f; i0[e] = -1; i1[e] = -1; dot[e] = 0.f;
+                if (on[e]) {
+                    const size_t lb = ((size_t)list * p.m + (q0 + warp * 32u + src[e])) * p.K;
+                    if (lane < hv[e]) { e0[e] = __ldcg(p.part_cos + lb + lane); i0[e] = __ldcg(p.part_ids + lb + lane); }
+                    if (lane + 32u < hv[e]) { e1[e] = __ldcg(p.part_cos + lb + lane + 32u); i1[e] = __ldcg(p.part_ids + lb + lane + 32u); }
+                }
+            }
+            for (uint32_t idx = lane; idx < p.d4; idx += 32) {
+#pragma unroll
+                for (int e = 0; e < kExact; ++e) {
+                    if (on[e]) {
+                        const float4 x = __ldcg(T4 + (size_t)qr[e] * p.ld4 + idx);
+                        const float4 y = __ldcg(T4 + (size_t)(p.cand_lo + cnd[e]) * p.ld4 + idx);
+                        dot[e] = fmaf(x.x, y.x, dot[e]); dot[e] = fmaf(x.y, y.y, dot[e]);
+                        dot[e] = fmaf(x.z, y.z, dot[e]); dot[e] = fmaf(x.w, y.w, dot[e]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                for (int e = 0; e < kExact; ++e) dot[e] += __shfl_xor_sync(kFullMask, dot[e], o);
+            }
+#pragma unroll
+            for (int e = 0; e < kExact; ++e) {
+                if (!on[e]) continue;                                                   // same for every lane
+                const float cs = dot[e] * qi[e] * __ldg(p.inv_norm + cnd[e]);
+                const long long cid = (long long)(p.cand_lo + cnd[e]);
+                if (!(cs > p.tau) || cid == qr[e] || (hv[e] == p.K && cs < th[e]) || cs < fl[e]) continue;
+                const size_t lb = ((size_t)list * p.m + (q0 + warp * 32u + src[e])) * p.K;
+                float *wl = p.part_cos + lb;
+                long long *wi = p.part_ids + lb;
+                const bool a0 = lane < hv[e] && !ranks_ahead_tc(cs, cid, e0[e], i0[e]);         // entries that stay ahead: a prefix
+                const bool a1 = lane + 32u < hv[e] && !ranks_ahead_tc(cs, cid, e1[e], i1[e]);
+                const uint32_t pos = (uint32_t)__popc(__ballot_sync(kFullMask, a0)) + (uint32_t)__popc(__ballot_sync(kFullMask, a1));
+                const uint32_t km2 = p.K >= 2u ? p.K - 2u : 0u;
+                const float e_km2 = km2 < 32u ? __shfl_sync(kFullMask, e0[e], km2) : __shfl_sync(kFullMask, e1[e], km2 - 32u);
+                if (pos < p.K) {
+                    if (lane < hv[e] && !a0 && lane + 1u < p.K) { wl[lane + 1u] = e0[e]; wi[lane + 1u] = i0[e]; }
+                    if (lane + 32u < hv[e] && !a1 && lane + 33u < p.K) { wl[lane + 33u] = e1[e]; wi[lane + 33u] = i1[e]; }
+                    if (lane == 0) { wl[pos] = cs; wi[pos] = cid; }
+                    if (lane == src[e]) {
+                        have = hv[e] < p.K ? hv[e] + 1u : p.K;
+                        thr = have == p.K ? (pos == p.K - 1u ? cs : e_km2) : p.tau;
+                        if (have == p.K) atomicMax(p.floor_q + (q0 + warp * 32u + src[e]), ordered_bits(thr));
+                    }
+                }
+            }
+            __syncwarp();
+        }
+    };
+    for (uint64_t i = 0; i < n_tiles; ++i) {
+        const uint32_t b = (uint32_t)(i & 1);
+        c0 = (t_lo + i) * kTcN;
+        if (mine) { const unsigned int o = __ldcg(p.floor_q + (q0 + r)); if (o) flo = ordered_float(o); }
+        // the tensor-memory loads below are warp-wide: the whole warp goes on or gives up together
+        if (!__all_sync(kFullMask, mbar_wait(tfull + b, (uint32_t)((i >> 1) & 1), abort_flag))) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        // Two chunks of 32 accumulator columns are in flight: the load of chunk k + 1 is issued before
+        // chunk k is looked at.  The candidate rows were packed as unit vectors, so a column times
+        // 1/|query| is the screened cosine; the largest of the 32 decides whether the chunk needs a
+        // closer look at all.
+        uint32_t va[32], vb[32];
+        tmem_ld32(va, tmem_base + ((warp * 32u) << 16) + b * kTcN);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll 1
+        for (uint32_t cc = 0; cc < (uint32_t)kTcN; cc += 64) {
+            tmem_ld32(vb, tmem_base + ((warp * 32u) << 16) + b * kTcN + cc + 32u);
+            screen_chunk(va, cc);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (cc + 64u < (uint32_t)kTcN) tmem_ld32(va, tmem_base + ((warp * 32u) << 16) + b * kTcN + cc + 64u);
+            screen_chunk(vb, cc + 32u);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        arrive_tempty(b);                                     // this accumulator buffer may be overwritten
+    }
+}
+
 // RES: the query block is resident in shared memory (d <= 320); otherwise its K-blocks stream through
 // the stages beside the candidates' (8 KB + 16 KB per stage).
 template <bool RES>
@@ -599,155 +761,8 @@ topk_cosine_screen_kernel(TcParams p)
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp < 4) {
-        // ================= epilogue: one thread per query row =================
-        const uint32_t r = tid;
-        const long long my_q = qrow[r];
-        const bool live = q0 + r < p.m;
-        const float4 *T4 = reinterpret_cast<const float4 *>(p.table);
-        float *lc = p.part_cos + ((size_t)blockIdx.y * p.m + (q0 + r)) * p.K;      // this query's list (global, private)
-        long long *li = p.part_ids + ((size_t)blockIdx.y * p.m + (q0 + r)) * p.K;
-        float qinv = 0.f;
-        if (my_q >= 0) {
-            const float4 *row = T4 + (size_t)my_q * p.ld4;
-            float s = 0.f;
-            for (uint32_t j = 0; j < p.d4; ++j) {
-                const float4 x = __ldcg(row + j);
-                s = fmaf(x.x, x.x, s); s = fmaf(x.y, x.y, s); s = fmaf(x.z, x.z, s); s = fmaf(x.w, x.w, s);
-            }
-            qinv = s > 0.f ? 1.0f / sqrtf(s) : 0.f;
-        }
-        if (live) for (uint32_t s = 0; s < p.K; ++s) { lc[s] = 0.f; li[s] = -1; }
-        const bool mine = my_q >= 0 && live;
-        uint32_t have = 0;
-        float thr = p.tau;
-        // The blocks that work on other candidates of the same queries publish the K-th best cosine they
-        // have reached (floor_q, raised by atomicMax); K candidates at or above it exist, so whatever is
-        // below it cannot be among the query's final K, in any block.  Read once per tile.
-        float flo = -INFINITY;
-        // one chunk of 32 columns of the current tile (first candidate c0 + cc)
-        uint64_t c0 = 0;
-        auto screen_chunk = [&](const uint32_t (&v)[32], uint32_t cc) {
-            __syncwarp();
-            const float cut = fmaxf(have < p.K ? p.tau : fmaxf(p.tau, thr), flo) - kScreenEps;
-            // the largest of the 32 columns, as a tree of three-input maxima (11 + 4 + 1 operations, depth 4)
-            float t1[11];
-#pragma unroll
-            for (int j = 0; j < 10; ++j) t1[j] = max3(__uint_as_float(v[3 * j]), __uint_as_float(v[3 * j + 1]), __uint_as_float(v[3 * j + 2]));
-            t1[10] = fmaxf(__uint_as_float(v[30]), __uint_as_float(v[31]));
-            const float top = max3(max3(t1[0], t1[1], t1[2]), max3(t1[3], t1[4], t1[5]),
-                                   max3(max3(t1[6], t1[7], t1[8]), t1[9], t1[10]));
-            const bool hit = mine && c0 + cc < nc && top * qinv >= cut;
-            // a chunk with a column near the cut is rare: everything below sits behind one warp-wide branch
-            if (!__any_sync(kFullMask, hit)) return;
-            uint32_t maybe = 0u;
-            if (hit) {                                                     // which of them?
-#pragma unroll
-                for (int j = 0; j < 32; ++j) maybe |= (__uint_as_float(v[j]) * qinv >= cut ? 1u : 0u) << j;
-                const uint64_t left = nc - (c0 + cc);                      // candidates of the range from column cc on
-                if (left < 32) maybe &= (1u << (uint32_t)left) - 1u;
-            }
-            // Exact pass: the set bits of all lanes, up to kExact queries (lanes) at a time.  The whole warp
-            // works on each (query, candidate): 32 lanes on the fp32 dot product of the two table rows
-            // (the loads of all kExact pairs are issued before the first sum is reduced), then on the
-            // insertion into that query's sorted list, lane l holding entries l and l + 32.
-            for (;;) {
-                uint32_t owners = __ballot_sync(kFullMask, maybe != 0u);
-                if (!owners) break;
-                bool on[kExact];
-                uint32_t src[kExact], hv[kExact];
-                float th[kExact], fl[kExact], qi[kExact], dot[kExact], e0[kExact], e1[kExact];
-                long long i0[kExact], i1[kExact], qr[kExact];
-                uint64_t cnd[kExact];
-#pragma unroll
-                for (int e = 0; e < kExact; ++e) {
-                    on[e] = owners != 0u;
-                    src[e] = on[e] ? (uint32_t)__ffs((int)owners) - 1u : 0u;
-                    owners &= owners - 1u;
-                    const uint32_t j = __shfl_sync(kFullMask, (uint32_t)__ffs((int)maybe) - 1u, src[e]);
-                    cnd[e] = c0 + cc + j;
-                    qr[e] = qrow[warp * 32u + src[e]];
-                    hv[e] = __shfl_sync(kFullMask, have, src[e]);
-                    th[e] = __shfl_sync(kFullMask, thr, src[e]);
-                    fl[e] = __shfl_sync(kFullMask, flo, src[e]);
-                    qi[e] = __shfl_sync(kFullMask, qinv, src[e]);
-                    if (on[e] && lane == src[e]) maybe &= maybe - 1u;
-                    e0[e] = 0.f; e1[e] = 0.f; i0[e] = -1; i1[e] = -1; dot[e] = 0.f;
-                    if (on[e]) {
-                        const size_t lb = ((size_t)blockIdx.y * p.m + (q0 + warp * 32u + src[e])) * p.K;
-                        if (lane < hv[e]) { e0[e] = __ldcg(p.part_cos + lb + lane); i0[e] = __ldcg(p.part_ids + lb + lane); }
-                        if (lane + 32u < hv[e]) { e1[e] = __ldcg(p.part_cos + lb + lane + 32u); i1[e] = __ldcg(p.part_ids + lb + lane + 32u); }
-                    }
-                }
-                for (uint32_t idx = lane; idx < p.d4; idx += 32) {
-#pragma unroll
-                    for (int e = 0; e < kExact; ++e) {
-                        if (on[e]) {
-                            const float4 x = __ldcg(T4 + (size_t)qr[e] * p.ld4 + idx);
-                            const float4 y = __ldcg(T4 + (size_t)(p.cand_lo + cnd[e]) * p.ld4 + idx);
-                            dot[e] = fmaf(x.x, y.x, dot[e]); dot[e] = fmaf(x.y, y.y, dot[e]);
-                            dot[e] = fmaf(x.z, y.z, dot[e]); dot[e] = fmaf(x.w, y.w, dot[e]);
-                        }
-                    }
-                }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-                    for (int e = 0; e < kExact; ++e) dot[e] += __shfl_xor_sync(kFullMask, dot[e], o);
-                }
-#pragma unroll
-                for (int e = 0; e < kExact; ++e) {
-                    if (!on[e]) continue;                                                   // same for every lane
-                    const float cs = dot[e] * qi[e] * __ldg(p.inv_norm + cnd[e]);
-                    const long long cid = (long long)(p.cand_lo + cnd[e]);
-                    if (!(cs > p.tau) || cid == qr[e] || (hv[e] == p.K && cs < th[e]) || cs < fl[e]) continue;
-                    const size_t lb = ((size_t)blockIdx.y * p.m + (q0 + warp * 32u + src[e])) * p.K;
-                    float *wl = p.part_cos + lb;
-                    long long *wi = p.part_ids + lb;
-                    const bool a0 = lane < hv[e] && !ranks_ahead_tc(cs, cid, e0[e], i0[e]);         // entries that stay ahead: a prefix
-                    const bool a1 = lane + 32u < hv[e] && !ranks_ahead_tc(cs, cid, e1[e], i1[e]);
-                    const uint32_t pos = (uint32_t)__popc(__ballot_sync(kFullMask, a0)) + (uint32_t)__popc(__ballot_sync(kFullMask, a1));
-                    const uint32_t km2 = p.K >= 2u ? p.K - 2u : 0u;
-                    const float e_km2 = km2 < 32u ? __shfl_sync(kFullMask, e0[e], km2) : __shfl_sync(kFullMask, e1[e], km2 - 32u);
-                    if (pos < p.K) {
-                        if (lane < hv[e] && !a0 && lane + 1u < p.K) { wl[lane + 1u] = e0[e]; wi[lane + 1u] = i0[e]; }
-                        if (lane + 32u < hv[e] && !a1 && lane + 33u < p.K) { wl[lane + 33u] = e1[e]; wi[lane + 33u] = i1[e]; }
-                        if (lane == 0) { wl[pos] = cs; wi[pos] = cid; }
-                        if (lane == src[e]) {
-                            have = hv[e] < p.K ? hv[e] + 1u : p.K;
-                            thr = have == p.K ? (pos == p.K - 1u ? cs : e_km2) : p.tau;
-                            if (have == p.K) atomicMax(p.floor_q + (q0 + warp * 32u + src[e]), ordered_bits(thr));
-                        }
-                    }
-                }
-                __syncwarp();
-            }
-        };
-        for (uint64_t i = 0; i < n_tiles; ++i) {
-            const uint32_t b = (uint32_t)(i & 1);
-            c0 = (t_lo + i) * kTcN;
-            if (mine) { const unsigned int o = __ldcg(p.floor_q + (q0 + r)); if (o) flo = ordered_float(o); }
-            // the tensor-memory loads below are warp-wide: the whole warp goes on or gives up together
-            if (!__all_sync(kFullMask, mbar_wait(tfull + b, (uint32_t)((i >> 1) & 1), abort_flag))) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            // Two chunks of 32 accumulator columns are in flight: the load of chunk k + 1 is issued before
-            // chunk k is looked at.  The candidate rows were packed as unit vectors, so a column times
-            // 1/|query| is the screened cosine; the largest of the 32 decides whether the chunk needs a
-            // closer look at all.
-            uint32_t va[32], vb[32];
-            tmem_ld32(va, tmem_base + ((warp * 32u) << 16) + b * kTcN);
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll 1
-            for (uint32_t cc = 0; cc < (uint32_t)kTcN; cc += 64) {
-                tmem_ld32(vb, tmem_base + ((warp * 32u) << 16) + b * kTcN + cc + 32u);
-                screen_chunk(va, cc);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (cc + 64u < (uint32_t)kTcN) tmem_ld32(va, tmem_base + ((warp * 32u) << 16) + b * kTcN + cc + 64u);
-                screen_chunk(vb, cc + 32u);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            }
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            mbar_arrive(tempty + b);                              // this accumulator buffer may be overwritten
-        }
+        screen_epilogue(p, qrow, q0, nc, t_lo, n_tiles, tmem_base, tfull, abort_flag, blockIdx.y,
+                        [&](uint32_t b) { mbar_arrive(tempty + b); });
     } else if (warp == 4) {
         // ================= MMA issue: one lane =================
         if (lane == 0) {
@@ -829,6 +844,242 @@ topk_cosine_screen_kernel(TcParams p)
     }
 }
 
+// =================================================================================================
+// The screening kernel on a pair of SMs (`cta_group::2`): a cluster of two thread blocks, each with
+// its own resident query block (M = 2 x 128 accumulator rows) and HALF of every candidate tile (N = 256
+// as 2 x 128 rows), so every candidate byte that an SM pulls through L2 now serves 256 queries and the
+// stage memory of both SMs works for one tile stream.  The even block of the pair (the leader) issues
+// the MMAs for both; each block's tensor core reads its own query block and both halves of the tile and
+// writes the 128 x 256 accumulator of its own queries into its own tensor memory, where the block's
+// epilogue warps screen it exactly as in the one-block kernel.
+//
+// Hand-overs (every barrier lives in one block's shared memory; nothing is broadcast):
+//   full[s]   own half of stage s has landed (bulk copy, complete_tx)          waited by: leader's MMA lane / follower's relay
+//   fullF[s]  (leader) the follower's half has landed; its relay lane arrives remotely
+//   empty[s]  the MMAs that read stage s are done: leader's by tcgen05.commit, follower's by a remote
+//             arrival from the leader's relay lane, which waits on the leader's empty[s]
+//   tfull[b]  accumulator b complete: leader's by tcgen05.commit, follower's through the leader's second relay lane
+//   tempty[b] (leader) all 256 epilogue threads of the pair are done with accumulator b (128 remote arrivals)
+// All waits are the time-limited mbar_wait; a block that gives up still reaches the cluster barrier at
+// the end, so its partner (whose waits then run out too) is never left behind.
+constexpr int kPrStages = 3;
+constexpr int kPrKPS = 5;                                         // K-blocks per stage
+constexpr int kPrHalf = kTcN / 2;                                 // candidate rows of a tile per block
+constexpr int kPrBChunk = kPrHalf * 16;
+constexpr int kPrKBlock = kScCh * kPrBChunk;                      // one K-block of a half tile: 8 KB
+constexpr int kPrStage = kPrKPS * kPrKBlock;                      // 40 KB
+constexpr int kPrThreads = 8 * 32;                                // 4 epilogue warps, MMA, producer, two relay warps
+
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrival on the barrier at the same shared-memory offset in block `rank` of the cluster
+__device__ __forceinline__ void mbar_arrive_in(uint64_t *bar, uint32_t rank)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_addr(bar)), "r"(rank));
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+// the time-limited wait for a barrier that another block of the cluster arrives at
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    const unsigned long long t0 = global_ns();
+    for (uint32_t spin = 0; spin < (1u << 30); ++spin) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+        if (done) return true;
+        if ((spin & 1023u) == 1023u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > kTcWaitNs) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}\n"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0) : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPrThreads, 1)
+topk_cosine_screen_pair_kernel(TcParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char *a_op = smem;                                              // [kScMaxKB] K-blocks of the own query block
+    unsigned char *b_op = smem + kScMaxKB * kScABlock;                       // [kPrStages] stages of the own half tile
+    uint64_t *full = reinterpret_cast<uint64_t *>(b_op + kPrStages * kPrStage);
+    uint64_t *fullF = full + kPrStages;
+    uint64_t *empty = fullF + kPrStages;
+    uint64_t *tfull = empty + kPrStages;
+    uint64_t *tempty = tfull + 2;
+    uint64_t *afull = tempty + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(afull + 1);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    long long *qrow = reinterpret_cast<long long *>(tmem_slot + 2);          // [128]
+
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_rank();                                     // 0: leader, 1: follower
+    const bool leader = rank == 0;
+    const uint64_t q0 = (uint64_t)blockIdx.x * kTcM;
+    const uint64_t nc = p.cand_hi - p.cand_lo;
+    const uint64_t tiles = (nc + kTcN - 1) / kTcN;                            // tiles of 256 candidates, as two half tiles in the packed copy
+    const uint64_t t_lo = tiles * blockIdx.y / p.splits, t_hi = tiles * (blockIdx.y + 1) / p.splits;
+    const uint32_t nkb = (4u * p.d4 + kScKB - 1) / kScKB;
+    const uint32_t nst = (nkb + kPrKPS - 1) / kPrKPS;
+    const uint64_t n_tiles = t_hi - t_lo;
+    const uint64_t total_g = n_tiles * nst;
+
+    if (tid == 0) {
+        for (int s = 0; s < kPrStages; ++s) { mbar_init(full + s, 1); mbar_init(fullF + s, 1); mbar_init(empty + s, 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull + b, 1); mbar_init(tempty + b, 2 * kTcM); }
+        mbar_init(afull, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (tid < (uint32_t)kTcM) {
+        long long r = q0 + tid < p.m ? p.queries[q0 + tid] : -1;
+        if (r < 0 || (unsigned long long)r >= p.vocab) r = -1;
+        qrow[tid] = r;
+    }
+    if (warp == 4) {       // the same warp of both blocks, the same slot: the pair's tensor memory is allocated together
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(2 * kTcN));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    cluster_sync_all();                                                       // both blocks' barriers exist before anyone arrives remotely
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp < 4) {
+        if (leader)
+            screen_epilogue(p, qrow, q0, nc, t_lo, n_tiles, tmem_base, tfull, abort_flag, blockIdx.y,
+                            [&](uint32_t b) { mbar_arrive(tempty + b); });
+        else
+            screen_epilogue(p, qrow, q0, nc, t_lo, n_tiles, tmem_base, tfull, abort_flag, blockIdx.y,
+                            [&](uint32_t b) { mbar_arrive_in(tempty + b, 0u); });
+    } else if (warp == 4) {
+        if (lane == 0) {
+            // the own query block: one bulk copy per K-block, all on one barrier
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                         ::"r"(smem_addr(afull)), "r"(nkb * (uint32_t)kScABlock) : "memory");
+            for (uint32_t kb = 0; kb < nkb; ++kb)
+                bulk_to_smem(a_op + (size_t)kb * kScABlock, p.qsplit + ((size_t)blockIdx.x * nkb + kb) * kScABlock,
+                             (uint32_t)kScABlock, afull);
+            bool ok = mbar_wait(afull, 0u, abort_flag);
+            if (leader) {
+                // bf16 x bf16 -> fp32, both operands K-major, M = 256 and N = 256 over the pair
+                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcN >> 3) << 17) | ((uint32_t)((2 * kTcM) >> 4) << 24);
+                uint64_t g = 0;
+                for (uint64_t i = 0; i < n_tiles && ok; ++i) {
+                    const uint32_t b = (uint32_t)(i & 1);
+                    ok = mbar_wait_cluster(tempty + b, (uint32_t)(((i >> 1) & 1) ^ 1), abort_flag);
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t dst = tmem_base + b * kTcN;
+                    for (uint32_t st = 0; st < nst && ok; ++st, ++g) {
+                        const uint32_t s = (uint32_t)(g % kPrStages), ph = (uint32_t)((g / kPrStages) & 1);
+                        ok = mbar_wait(full + s, ph, abort_flag) && mbar_wait_cluster(fullF + s, ph, abort_flag);
+                        if (!ok) break;
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        for (uint32_t kb = st * kPrKPS; kb < nkb && kb < (st + 1) * kPrKPS; ++kb) {
+                            const uint32_t abase = smem_addr(a_op + (size_t)kb * kScABlock);
+                            const uint32_t bbase = smem_addr(b_op + (size_t)s * kPrStage + (size_t)(kb - st * kPrKPS) * kPrKBlock);
+                            const uint32_t cols = 4u * p.d4 - kb * kScKB < (uint32_t)kScKB ? 4u * p.d4 - kb * kScKB : (uint32_t)kScKB;
+                            const uint32_t nk = (cols + 15u) / 16u;
+                            for (uint32_t kk = 0; kk < nk; ++kk) {
+                                const uint64_t qa = umma_desc(abase + 2 * kk * kScAChunk, kScAChunk, 128);
+                                const uint64_t cb = umma_desc(bbase + 2 * kk * kPrBChunk, kPrBChunk, 128);
+                                umma_bf16_pair(dst, qa, cb, idesc, (kb | kk) ? 1u : 0u);
+                            }
+                        }
+                        umma_commit_pair(empty + s);
+                    }
+                    if (ok) umma_commit_pair(tfull + b);
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // producer: the own half of every stage
+        if (lane == 0) {
+            uint64_t g = 0;
+            for (; g < total_g; ++g) {
+                const uint32_t s = (uint32_t)(g % kPrStages), ph = (uint32_t)(((g / kPrStages) & 1) ^ 1);
+                if (!(leader ? mbar_wait(empty + s, ph, abort_flag) : mbar_wait_cluster(empty + s, ph, abort_flag))) break;
+                const uint32_t kb0 = (uint32_t)(g % nst) * kPrKPS;
+                const uint32_t nkbs = nkb - kb0 < (uint32_t)kPrKPS ? nkb - kb0 : (uint32_t)kPrKPS;
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                             ::"r"(smem_addr(full + s)), "r"(nkbs * (uint32_t)kPrKBlock) : "memory");
+                // half tile number 2 T + rank of the packed copy (tiles of 128 rows)
+                bulk_to_smem(b_op + (size_t)s * kPrStage,
+                             p.ctiles + ((2 * (t_lo + g / nst) + rank) * nkb + kb0) * (size_t)kPrKBlock, nkbs * (uint32_t)kPrKBlock, full + s);
+            }
+            if (*abort_flag) {
+                for (uint64_t j = g > (uint64_t)kPrStages ? g - kPrStages : 0; j < g; ++j)
+                    for (uint32_t spin = 0; spin < kTcSpinLimit; ++spin)
+                        if (mbar_try(full + j % kPrStages, (uint32_t)((j / kPrStages) & 1))) break;
+            }
+        }
+    } else if (warp == 6) {
+        if (lane == 0) {
+            if (leader) {
+                // relay: a stage whose MMAs are done is free in the follower as well
+                for (uint64_t g = 0; g < total_g; ++g) {
+                    const uint32_t s = (uint32_t)(g % kPrStages);
+                    if (!mbar_wait(empty + s, (uint32_t)((g / kPrStages) & 1), abort_flag)) break;
+                    mbar_arrive_in(empty + s, 1u);
+                }
+            } else {
+                // relay: the follower's half of a stage (and, first of all, its query block) has landed
+                bool ok = mbar_wait(afull, 0u, abort_flag);
+                for (uint64_t g = 0; g < total_g && ok; ++g) {
+                    const uint32_t s = (uint32_t)(g % kPrStages);
+                    ok = mbar_wait(full + s, (uint32_t)((g / kPrStages) & 1), abort_flag);
+                    if (ok) mbar_arrive_in(fullF + s, 0u);
+                }
+            }
+        }
+    } else {
+        if (lane == 0 && leader) {
+            // relay: a complete accumulator is complete in the follower's tensor memory as well
+            for (uint64_t i = 0; i < n_tiles; ++i) {
+                const uint32_t b = (uint32_t)(i & 1);
+                if (!mbar_wait(tfull + b, (uint32_t)((i >> 1) & 1), abort_flag)) break;
+                mbar_arrive_in(tfull + b, 1u);
+            }
+        }
+    }
+    // ================= common exit =================
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (tid == 0 && *abort_flag) atomicExch(p.error, 1);
+    cluster_sync_all();                                   // neither block leaves while its partner may still reach into it
+    if (warp == 4) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * kTcN));
+    }
+}
+
+static size_t topk_screen_pair_smem_bytes()
+{
+    return (size_t)kScMaxKB * kScABlock + (size_t)kPrStages * kPrStage + (3 * kPrStages + 5) * 8 + 8 + kTcM * 8 + 128;
+}
+
 // The give-up path of the retrieval kernels on its own: one block waits, with the kernels' own wait
 // routine and a short limit, on a barrier that nobody arrives at; when the limit has passed it raises
 // the error word exactly as a retrieval block does, and returns.
@@ -903,7 +1154,7 @@ size_t topk_screen_ctiles_bytes(uint64_t nc, uint32_t d)
 int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, const long long *queries, uint64_t m,
                    uint64_t cand_lo, uint64_t cand_hi, uint32_t K, float tau, float *inv_norm,
                    unsigned char *qsplit, unsigned char *ctiles, unsigned int *floor_q, float *part_cos, long long *part_ids,
-                   uint32_t splits, int *error, bool screen, int sms, cudaStream_t s)
+                   uint32_t splits, int *error, bool screen, bool pairs, int sms, cudaStream_t s)
 {
     if (m == 0) return 0;
     const unsigned qblocks = (unsigned)((m + kTcM - 1) / kTcM);
@@ -925,26 +1176,34 @@ int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, 
         return 2;
     }
     const uint32_t nkb = (d + kScKB - 1) / kScKB;
-    topk_round_queries_kernel<<<qblocks * nkb, 256, 0, s>>>(table, queries, m, vocab, d / 4, ld / 4, nkb, qsplit);
+    topk_round_queries_kernel<<<((qblocks + 1) / 2 * 2) * nkb, 256, 0, s>>>(table, queries, m, vocab, d / 4, ld / 4, nkb, qsplit);
     if (cudaGetLastError() != cudaSuccess) return -1;
     if (cudaMemsetAsync(floor_q, 0, m * sizeof(unsigned int), s) != cudaSuccess) return -1;   // 0 = no floor yet
     const bool resident = topk_screen_resident(d);
-    const size_t sm = topk_screen_smem_bytes(resident);
-    if (cudaFuncSetAttribute(resident ? topk_cosine_screen_kernel<true> : topk_cosine_screen_kernel<false>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess)
-        return -1;
+    // on request, with more than one query block of resident width: pairs of blocks on pairs of SMs share every candidate tile
+    const bool pair = pairs && resident && qblocks >= 2;
+    const size_t sm = pair ? topk_screen_pair_smem_bytes() : topk_screen_smem_bytes(resident);
+    const void *kernel = pair ? (const void *)topk_cosine_screen_pair_kernel
+                         : resident ? (const void *)topk_cosine_screen_kernel<true> : (const void *)topk_cosine_screen_kernel<false>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess) return -1;
+    if (pair) grid.x = (qblocks + 1) / 2 * 2;                  // whole pairs; the rows of a padded block are zeros
     int launched = 1;
     const uint64_t nc = cand_hi - cand_lo, chunk = topk_screen_chunk(nc, d);
     uint64_t list = 0;
     for (uint64_t c0 = 0; c0 < nc; c0 += chunk, ++list) {
         const uint64_t n = nc - c0 < chunk ? nc - c0 : chunk;
-        topk_pack_candidates_kernel<<<sms * 16, kTcN, 0, s>>>(table, inv_norm + c0, d / 4, ld / 4, cand_lo + c0, n, nkb, ctiles);
+        const uint64_t tiles = (n + kTcN - 1) / kTcN;
+        if (pair)
+            topk_pack_candidates_kernel<kPrHalf><<<sms * 32, kPrHalf, 0, s>>>(table, inv_norm + c0, d / 4, ld / 4, cand_lo + c0, n, 2 * tiles, nkb, ctiles);
+        else
+            topk_pack_candidates_kernel<kTcN><<<sms * 16, kTcN, 0, s>>>(table, inv_norm + c0, d / 4, ld / 4, cand_lo + c0, n, tiles, nkb, ctiles);
         if (cudaGetLastError() != cudaSuccess) return -1;
         p.cand_lo = cand_lo + c0; p.cand_hi = cand_lo + c0 + n;
         p.inv_norm = inv_norm + c0;
         p.part_cos = part_cos + list * splits * m * K;
         p.part_ids = part_ids + list * splits * m * K;
-        if (resident) topk_cosine_screen_kernel<true><<<grid, kScThreads, sm, s>>>(p);
+        if (pair) topk_cosine_screen_pair_kernel<<<grid, kPrThreads, sm, s>>>(p);
+        else if (resident) topk_cosine_screen_kernel<true><<<grid, kScThreads, sm, s>>>(p);
         else topk_cosine_screen_kernel<false><<<grid, kScThreads, sm, s>>>(p);
         if (cudaGetLastError() != cudaSuccess) return -1;
         launched += 2;

@@ -48,7 +48,7 @@ def test_retrieval_at_the_benchmarked_shape():
         assert (np.diff(gc, axis=1)[(gi[:, 1:] >= 0)] <= 0).all()
         assert ((gi < 0) | ((gi >= LO) & (gi < HI) & (gi != q[:, None]))).all()
         assert (gc[gi >= 0] > tau - 2e-6).all()
-        for kernel in (0, 1):                                       # the other two kernels on the sample
+        for kernel in (0, 1, 3):                                    # the other kernels on the sample
             binding.w2v_set_retrieval_kernel(gpu.h, kernel)
             si, sc = gpu.topk_cosine(0, q[pick], LO, HI, K, tau)
             compare(si, sc, wi, wc, X, q[pick], LO, HI, K, tau, tolerance(kernel, D))
