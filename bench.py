@@ -746,7 +746,18 @@ def run_probe(args):
             moved = done * 4.0 * d * (2.0 if "red" in label else 1.0)
             per[label] = {"ms": best, "row_GBps": moved / (best * 1e-3) / 1e9, "frac_of_copy_peak": moved / (best * 1e-3) / 1e9 / peak}
         result[f"span_{span}_rows"] = per
+    # the ring of bulk copies that feeds the retrieval kernels: GB/s per SM against stage size, depth and producer lanes
+    ring = {}
+    for stage, stages, producers in ((16384, 8, 1), (16384, 4, 1), (32768, 4, 1), (49152, 3, 1), (16384, 8, 2), (8192, 16, 1)):
+        best = None
+        for _ in range(3):
+            ms, done = binding.w2v_probe_bulk_ring(model.h, stage, stages, producers, 64 << 20)
+            best = ms if best is None or ms < best else best
+        model.sync()
+        ring[f"{stage}B_x{stages}_stages_{producers}_producer"] = {"ms": best, "GBps_per_sm": done / (best * 1e-3) / 1e9,
+                                                                   "ns_per_stage": best * 1e6 / (done / stage)}
     line = {"metric": "random_row_traffic", "unit": "GB/s of row bytes (read + written)", "n_gpus": 1,
+            "bulk_copy_ring": ring,
             "config": {"workload": name + " (memory-system probe)", "vocab": cfg["vocab"], "d": d,
                        "row_stride_floats": row_stride, "rows_per_launch": rows,
                        "table_GB": cfg["vocab"] * row_stride * 4 / 1e9},

@@ -435,6 +435,22 @@ int32_t w2v_probe_rows(w2v_handle *h, uint32_t access, uint64_t span_rows, uint6
                        uint64_t *rows_done);
 
 /*
+ * Second measuring aid (no counterpart in the paper): how fast one SM pulls L2-resident bytes into
+ * shared memory through a ring of bulk copies, the way the retrieval kernels stream their
+ * candidates.  One block per SM; `producers` lanes issue `cp.async.bulk` copies of stage_bytes
+ * from the first 64 MB of V into a ring of `stages` slots as a consumer lane releases them; the
+ * consumer only waits and releases.  The retrieval kernels' stage size follows from this figure:
+ * a lane hands over about one stage per 250 ns whatever the stage's size.
+ *   stage_bytes  a multiple of 16; stage_bytes * stages at most 200 KB;  stages 1..64;  producers 1..4.
+ *   bytes_per_sm bytes every block pulls (rounded down to whole stages).
+ *   ms, bytes_done  host; the launch's duration and the bytes per block actually copied.
+ * Reads V only.  Synchronises the stream.  All waits are bounded; a block that gives up makes
+ * the next w2v_sync return W2V_ERR_CUDA.
+ */
+int32_t w2v_probe_bulk_ring(w2v_handle *h, uint32_t stage_bytes, uint32_t stages, uint32_t producers,
+                            uint64_t bytes_per_sm, double *ms, uint64_t *bytes_done);
+
+/*
  * Launch shape of the update kernels: rows in flight per warp (1..8; 0 = default)
  * and resident thread blocks per SM (0 = as many as fit).  Results do not depend
  * on it in snapshot mode.

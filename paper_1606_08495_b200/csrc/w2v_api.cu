@@ -861,6 +861,44 @@ int32_t w2v_probe_rows(w2v_handle *h, uint32_t access, uint64_t span_rows, uint6
     return W2V_OK;
 }
 
+int32_t w2v_probe_bulk_ring(w2v_handle *h, uint32_t stage_bytes, uint32_t stages, uint32_t producers,
+                            uint64_t bytes_per_sm, double *ms, uint64_t *bytes_done)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (!ms || !bytes_done) return fail(h, W2V_ERR_ARG, "ms or bytes_done is NULL");
+    if (stage_bytes < 16 || (stage_bytes % 16) != 0 || stages < 1 || stages > 64 ||
+        (uint64_t)stage_bytes * stages > 200u * 1024u)
+        return fail(h, W2V_ERR_ARG, "need stage_bytes a multiple of 16, 1..64 stages and at most 200 KB of ring");
+    if (producers < 1 || producers > 4) return fail(h, W2V_ERR_ARG, "producers must be in 1..4");
+    const uint64_t span = (uint64_t)h->vocab * h->ld * sizeof(float) < (64ull << 20) ? (uint64_t)h->vocab * h->ld * sizeof(float) : (64ull << 20);
+    if (span < 2ull * stage_bytes * producers) return fail(h, W2V_ERR_ARG, "the table is smaller than two rounds of stages");
+    const uint64_t copies = bytes_per_sm / stage_bytes;
+    if (copies < 1 || copies > (1ull << 24)) return fail(h, W2V_ERR_ARG, "bytes_per_sm must give between 1 and 2^24 copies");
+    DeviceGuard g(h->device);
+    int32_t rc;
+    if ((rc = ensure_error_word(h)) != W2V_OK) return rc;
+    cudaEvent_t e0, e1;
+    W2V_CUDA(h, cudaEventCreate(&e0));
+    W2V_CUDA(h, cudaEventCreate(&e1));
+    int k = -1;
+    cudaError_t ce = cudaEventRecord(e0, h->stream);
+    if (ce == cudaSuccess) {
+        k = launch_probe_bulk_ring(reinterpret_cast<const unsigned char *>(h->V), span, stage_bytes, stages, (uint32_t)copies,
+                                   producers, h->tc_error, h->sms, h->stream);
+        ce = cudaEventRecord(e1, h->stream);
+    }
+    if (ce == cudaSuccess) ce = cudaEventSynchronize(e1);
+    float t = 0.f;
+    if (ce == cudaSuccess && k > 0) ce = cudaEventElapsedTime(&t, e0, e1);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (k < 0 || ce != cudaSuccess) return fail(h, W2V_ERR_CUDA, "probe launch", ce != cudaSuccess ? ce : cudaGetLastError());
+    h->launches += (uint64_t)k;
+    *ms = (double)t;
+    *bytes_done = copies * stage_bytes;
+    return W2V_OK;
+}
+
 int32_t w2v_set_step(w2v_handle *h, uint64_t step_id)
 {
     if (!h) return W2V_ERR_ARG;
@@ -910,6 +948,7 @@ int32_t w2v_sync(w2v_handle *h)
         W2V_CUDA(h, cudaMemcpy(&flag, h->tc_error, sizeof(int), cudaMemcpyDeviceToHost));
         if (flag) {
             W2V_CUDA(h, cudaMemset(h->tc_error, 0, sizeof(int)));
+            if (flag & 4) return fail(h, W2V_ERR_CUDA, "a block of the bulk-copy probe gave up waiting; its timing is void");
             if (flag & 2)
                 return fail(h, W2V_ERR_CUDA, "a peer barrier gave up waiting for another shard; the step that followed it "
                                              "used incomplete dot products");

@@ -156,6 +156,10 @@ int launch_probe_rows(float *V, const uint2 *alias, uint32_t vocab, uint32_t d4,
                       unsigned long long rows, uint32_t access, float *sink, int sms, cudaStream_t s,
                       unsigned long long *rows_done);
 
+// one block per SM pulls `copies` bulk copies of stage_bytes from src[0, span) through a ring of `stages` slots
+int launch_probe_bulk_ring(const unsigned char *src, unsigned long long span, uint32_t stage_bytes, uint32_t stages,
+                           uint32_t copies, uint32_t producers, int *error, int sms, cudaStream_t s);
+
 // ---- cosine retrieval (w2v_topk.cu) ----
 uint32_t topk_splits(uint64_t m, uint64_t n_candidates, int sms, uint32_t block_queries = 0, uint32_t tile_rows = 0);
 int launch_topk_merge(const float *part_cos, const long long *part_ids, uint64_t m, uint32_t K, uint32_t splits,

@@ -83,7 +83,87 @@ probe_rows_kernel(float *V, const uint2 *alias, uint32_t vocab, uint32_t d4, uin
     if (acc == 12345.678f) *sink = acc;
 }
 
+// ---- ring of bulk copies: how fast one SM can pull L2-resident bytes into shared memory -----------
+// One block per SM; `producers` lanes (one per warp) issue cp.async.bulk copies of `stage_bytes` into a
+// ring of `stages` slots, each on the slot's "full" barrier once a consumer lane has released the slot;
+// the consumer lane does nothing but wait for "full" and arrive on "empty".  Every block reads the same
+// stream (as the blocks of one candidate split of the retrieval kernels do), so after the first pass the
+// source sits in L2.  Waits are bounded; a block that gives up raises *error.
+__device__ __forceinline__ uint32_t probe_saddr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool probe_try(uint64_t *bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(probe_saddr(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+__device__ __forceinline__ bool probe_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    for (uint32_t spin = 0; spin < (1u << 24); ++spin) {
+        if (probe_try(bar, parity)) return true;
+        if ((spin & 1023u) == 1023u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__global__ void __launch_bounds__(256, 1)
+probe_bulk_ring_kernel(const unsigned char *src, unsigned long long span, uint32_t stage_bytes, uint32_t stages,
+                       uint32_t copies, uint32_t producers, int *error)
+{
+    extern __shared__ __align__(128) unsigned char probe_smem[];
+    uint64_t *bars = reinterpret_cast<uint64_t *>(probe_smem + (size_t)stage_bytes * stages);     // [stages] (full, empty)
+    __shared__ int abort_word;
+    volatile int *abort_flag = &abort_word;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        abort_word = 0;
+        for (uint32_t i = 0; i < 2 * stages; ++i)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(probe_saddr(bars + i)), "r"(1));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (lane == 0 && warp < producers) {
+        unsigned long long off = ((unsigned long long)warp * stage_bytes) % span;
+        for (uint32_t g = warp; g < copies; g += producers) {
+            const uint32_t s = g % stages;
+            uint64_t *full = bars + 2 * s, *empty = full + 1;
+            if (!probe_wait(empty, ((g / stages) & 1) ^ 1, abort_flag)) break;
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(probe_saddr(full)), "r"(stage_bytes) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(probe_saddr(probe_smem + (size_t)s * stage_bytes)), "l"(src + off), "r"(stage_bytes), "r"(probe_saddr(full)) : "memory");
+            off += (unsigned long long)stage_bytes * producers;
+            if (off + stage_bytes > span) off = ((unsigned long long)warp * stage_bytes) % span;
+        }
+    } else if (lane == 0 && warp == producers) {
+        uint32_t g = 0;
+        for (; g < copies; ++g) {
+            const uint32_t s = g % stages;
+            uint64_t *full = bars + 2 * s, *empty = full + 1;
+            if (!probe_wait(full, (g / stages) & 1, abort_flag)) break;
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(probe_saddr(empty)) : "memory");
+        }
+        if (g < copies) {
+            // giving up: copies already issued may still land; give them their time before shared memory goes away
+            for (uint32_t j = g; j < g + stages && j < copies; ++j)
+                for (uint32_t spin = 0; spin < (1u << 20); ++spin)
+                    if (probe_try(bars + 2 * (j % stages), (j / stages) & 1)) break;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_word) atomicExch(error, 4);
+}
+
 }  // namespace
+
+int launch_probe_bulk_ring(const unsigned char *src, unsigned long long span, uint32_t stage_bytes, uint32_t stages,
+                           uint32_t copies, uint32_t producers, int *error, int sms, cudaStream_t s)
+{
+    const size_t sm = (size_t)stage_bytes * stages + 16 * (size_t)stages;
+    if (cudaFuncSetAttribute(probe_bulk_ring_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess) return -1;
+    probe_bulk_ring_kernel<<<sms, 256, sm, s>>>(src, span, stage_bytes, stages, copies, producers, error);
+    return cudaGetLastError() != cudaSuccess ? -1 : 1;
+}
 
 int launch_probe_rows(float *V, const uint2 *alias, uint32_t vocab, uint32_t d4, uint32_t ld4, uint32_t span,
                       unsigned long long rows, uint32_t access, float *sink, int sms, cudaStream_t s,

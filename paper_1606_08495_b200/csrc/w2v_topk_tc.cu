@@ -405,10 +405,11 @@ topk_cosine_tc_kernel(TcParams p)
 // whole kernel (d <= 320: 80 KB); candidates stream through three 48 KB stages (three K-blocks of 32
 // columns of a 256-candidate tile: six MMAs of K = 16), each filled by one `cp.async.bulk` that a
 // single producer lane issues as soon as the stage's previous MMAs have committed.  The stage is
-// that large because one lane hands over a stage every ~330 ns whatever its size (a ring of bulk
-// copies alone, without MMAs, moves 50 GB/s per SM with 16 KB stages at any depth and 99 GB/s with
-// 32 KB stages): with 16 KB stages that hand-over rate, not bytes or MMAs, bounded the kernel
-// (19.0 -> 16.6 ms for 8192 queries x 3 M candidates; 32 KB x 4 and 64 KB x 2 measure the same).
+// that large because one lane hands over a stage every 250-330 ns whatever its size (w2v_probe_bulk_ring:
+// a ring of bulk copies alone, without MMAs, moves 50-66 GB/s per SM with 16 KB stages at any depth,
+// twice that with 32 KB and three times with 48 KB stages): with 16 KB stages that hand-over rate, not
+// bytes or MMAs, bounded the kernel (19.0 -> 16.6 ms for 8192 queries x 3 M candidates; 32 KB x 4 and
+// 64 KB x 2 measure the same).
 constexpr float kScreenEps = 8.5e-3f;
 constexpr int kScKB = 32;                                        // columns per stage
 constexpr int kScCh = kScKB / 8;                                 // 16-byte chunks (8 bf16) per row and stage

@@ -493,6 +493,16 @@ def test_memory_probe_leaves_the_table_as_it_was():
             ms, done = binding.w2v_probe_rows(gpu.h, access, span, 100_000)
             assert ms > 0 and done >= 100_000
     assert np.array_equal(gpu.read_rows(1, ids), Vv)
+    # the ring of bulk copies only reads the table too
+    for stage, stages, producers in ((4096, 4, 1), (16384, 3, 2), (1024, 64, 4)):
+        ms, done = binding.w2v_probe_bulk_ring(gpu.h, stage, stages, producers, 1 << 20)
+        assert ms > 0 and done == (1 << 20) // stage * stage
+    gpu.sync()
+    assert np.array_equal(gpu.read_rows(1, ids), Vv)
+    for args in ((24, 4, 1, 1 << 20), (4096, 0, 1, 1 << 20), (65536, 4, 1, 1 << 20), (4096, 4, 5, 1 << 20), (4096, 4, 1, 100)):
+        with pytest.raises(binding.W2VError) as e:
+            binding.w2v_probe_bulk_ring(gpu.h, *args)
+        assert e.value.code == binding.W2V_ERR_ARG
     for args in ((5, 10, 10), (0, 0, 10), (0, cfg["vocab"] + 1, 10), (0, 10, 0)):
         with pytest.raises(binding.W2VError) as e:
             binding.w2v_probe_rows(gpu.h, *args)
