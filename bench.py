@@ -455,6 +455,15 @@ def run_gpu(args):
     default_shape = (name == "large" and args.mode == "hogwild" and not cbow and not args.row_stride
                      and not args.rows_in_flight and not args.blocks_per_sm and not args.dense_rows
                      and not args.tokens_per_step and IL == 1)
+    # the memory system's own ceiling for the update's access pattern on this table (random rows gathered and
+    # added to, no sampling, no arithmetic: w2v_probe_rows), measured right after the timed steps
+    ceiling = None
+    if rank == 0 and not cbow and args.mode == "hogwild" and d <= 512:
+        best, done = None, 0
+        for _ in range(3):
+            pms, done = binding.w2v_probe_rows(model.h, binding.PROBE_GATHER_RED, cfg["vocab"], min(20_000_000, 40 * cfg["vocab"]))
+            best = pms if best is None or pms < best else best
+        ceiling = 2.0 * 4 * d * done / (best * 1e-3) / 1e9
     secondary = None
     if world == 1 and default_shape and not args.no_secondary:
         secondary = secondary_modes(model, cfg, dev_chunks, Wu + 2 * K, dev)
@@ -489,6 +498,9 @@ def run_gpu(args):
                          "frac_of_8TBps": achieved / 8000.0,
                          "algorithmic_bytes_per_launch": per_launch_bytes,
                          "kernel_ms_per_launch": kernel_ms / max(1, groups),
+                         "access_pattern_ceiling": (None if ceiling is None else
+                                                    {"what": "random rows of the same table gathered and added to (w2v_probe_rows), GB/s of row bytes",
+                                                     "GBps": ceiling, "achieved_over_ceiling": achieved / ceiling}),
                          "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE * per_launch_bytes if default_shape else None),
                          "traffic_kind": ("scaled from one ncu capture of this kernel and workload, not measured in this run"
                                           if default_shape else None)},
