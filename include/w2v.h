@@ -147,11 +147,17 @@ int32_t w2v_get_tables(w2v_handle *h, uint32_t *thr, uint32_t *alias, uint32_t *
  *           later reads may or may not see them (Section 5.1, no locking).
  *   stats   host, may be NULL.  Non-NULL: the call waits for the step and fills
  *           it, and returns W2V_ERR_TOKEN_RANGE if bad ids were skipped.  NULL:
- *           the step is only enqueued (Hogwild mode never waits; snapshot mode
- *           waits once to size its coefficient array).
+ *           the step is only enqueued and the call does not wait.
  * Adds one to the step number.  Scratch is grown on the first call with a
- * larger n and reused afterwards: no allocation in the steady state.
- * Errors: W2V_ERR_ARG, W2V_ERR_STATE (no tables), W2V_ERR_NOMEM, W2V_ERR_CUDA.
+ * larger n and reused afterwards: no allocation and no waiting in the steady
+ * state.  The arrays with one entry per target (snapshot mode's coefficients, the
+ * list of negatives of snapshot mode and of Hogwild chunks of 500,000 tokens or
+ * more) are sized for the worst case 2 * window * n pairs when that takes at most
+ * 1 GiB; only beyond that (wide windows on long chunks) does snapshot mode wait
+ * once per step for the pair count and grow them with 25 % head-room, and Hogwild
+ * mode draws its negatives inside the update kernel.
+ * Errors: W2V_ERR_ARG, W2V_ERR_STATE (no tables), W2V_ERR_NOMEM, W2V_ERR_CUDA
+ * (also when status bit 1 reports that a time-limited wait inside a kernel ran out).
  */
 int32_t w2v_sgns_step(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_t window,
                       uint32_t negatives, float lr, uint32_t mode, w2v_step_stats *stats);

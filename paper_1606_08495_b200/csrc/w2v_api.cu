@@ -21,7 +21,7 @@ struct w2v_handle {
     // state between w2v_shard_dots and w2v_shard_adjust
     bool shard_pending = false;
     int32_t *l_centre = nullptr, *l_context = nullptr, *l_negs = nullptr;   // pair list of a narrow shard's step
-    uint64_t l_cap_pairs = 0, l_cap_negs = 0;
+    uint64_t l_cap_pairs = 0, l_cap_context = 0, l_cap_negs = 0;
     float *inv_norm = nullptr; uint64_t inv_norm_cap = 0;                      // retrieval scratch
     float *part_cos = nullptr; long long *part_ids = nullptr; uint64_t part_cap = 0;
     uint32_t retrieval_kernel = 2;       // 0: fp32 on the CUDA cores, 1: tensor cores (3 x TF32), 2: tensor-core screen + exact fp32, 3: the screen on pairs of SMs
@@ -626,9 +626,8 @@ int32_t w2v_shard_dots(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_
         return fail(h, W2V_ERR_CAPACITY, "more targets than the arrays for the partial dot products hold");
     if (pairs > 0 && h->d / 4 <= kNarrowD4) {
         // narrow slice: write the index sets once, the three passes stream over them
-        uint64_t cap_ctx = h->l_cap_pairs;                  // centre and context lists grow together
         if ((rc = grow(h, &h->l_centre, &h->l_cap_pairs, pairs, true)) != W2V_OK) return rc;
-        if ((rc = grow(h, &h->l_context, &cap_ctx, pairs, true)) != W2V_OK) return rc;
+        if ((rc = grow(h, &h->l_context, &h->l_cap_context, pairs, true)) != W2V_OK) return rc;
         if ((rc = grow(h, &h->l_negs, &h->l_cap_negs, pairs * (uint64_t)negatives, true)) != W2V_OK) return rc;
         StepParams pl = make_params(h, window, negatives, 0.f);
         if ((rc = profile_mark(h)) != W2V_OK) return rc;
