@@ -59,10 +59,10 @@ def regroup(chunks, tokens_per_step):
     return out
 
 
-def run(cfg, cp, chunks, mode, stride=1):
+def run(cfg, cp, chunks, mode, stride=1, lr0=None):
     g = binding.W2V(cfg["vocab"], cfg["d"], SEED, row_stride=binding.aligned_row_stride(cfg["d"]))
     g.build_alias(cp.counts, cfg["subsample_t"])
-    train(gpu_step(g, cfg["window"], cfg["negatives"], mode), chunks, epochs=1, lr0=cfg["lr"], stride=stride)
+    train(gpu_step(g, cfg["window"], cfg["negatives"], mode), chunks, epochs=1, lr0=cfg["lr"] if lr0 is None else lr0, stride=stride)
     g.set_interleave(0, 1)
     loss = heldout(g, cfg, cp)
     g.close()
@@ -88,6 +88,14 @@ def test_loss_against_minibatch_size_and_staleness():
     for mode, what, loss in rows:
         print("STUDY %-9s %-26s held-out loss %.5f  (%+.2f %% of the sequential checker's)" %
               (mode, what, loss, 100.0 * (loss - want) / want))
+    # the same minibatches at half the learning rate: the size at which training blows up moves up with it
+    half = []
+    for B in (2500, 5000, 10_000):
+        stride = max(1, int(round(centres / B)))
+        loss = run(cfg, cp, chunks, binding.MODE_SNAPSHOT, stride, lr0=0.5 * cfg["lr"])
+        half.append((round(centres / stride), loss))
+        print("STUDY snapshot  %-26s held-out loss %.5f  at lr0 %.4f" % ("%d input words" % round(centres / stride), loss, 0.5 * cfg["lr"]))
+    assert np.isfinite(half[0][1]) and half[0][1] < UNTRAINED
     snap = [l for m, w, l in rows if m == "snapshot"]
     hog = [l for m, w, l in rows if m == "hogwild"]
     # the paper's minibatch sizes (50-200 input words, and 1000) train as well as one pair after another
