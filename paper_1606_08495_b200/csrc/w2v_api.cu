@@ -631,7 +631,7 @@ int32_t w2v_shard_dots(w2v_handle *h, const int32_t *tokens, uint64_t n, uint32_
         if ((rc = grow(h, &h->l_negs, &h->l_cap_negs, pairs * (uint64_t)negatives, true)) != W2V_OK) return rc;
         StepParams pl = make_params(h, window, negatives, 0.f);
         if ((rc = profile_mark(h)) != W2V_OK) return rc;
-        k = launch_emit_pairs(pl, h->l_centre, h->l_context, h->l_negs, pairs, h->sms * 8, h->stream);
+        k = launch_pair_list(pl, h->l_centre, h->l_context, h->l_negs, h->sms * 8, h->stream);
         if (k < 0) return fail(h, W2V_ERR_CUDA, "pair list launch", cudaGetLastError());
         h->launches += (uint64_t)k;
         if (h->profiling) h->prof_launches += (uint64_t)k;

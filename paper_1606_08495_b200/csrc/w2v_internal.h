@@ -123,6 +123,8 @@ int launch_emit_pairs(const StepParams &p, int32_t *centre, int32_t *context, in
                       uint64_t cap, int grid, cudaStream_t s);
 // negs[pair * negatives + k] for every pair of the chunk (needs pair_off); counts the draws
 int launch_draw_negatives(const StepParams &p, int32_t *negs, int grid, cudaStream_t s);
+// centre[pair], context[pair] and negs[pair * negatives + k] of every pair (needs pair_off); counts the draws
+int launch_pair_list(const StepParams &p, int32_t *centre, int32_t *context, int32_t *negs, int grid, cudaStream_t s);
 
 int launch_hogwild(const StepParams &p, uint32_t rows_in_flight, uint32_t blocks_per_sm, int sms,
                    cudaStream_t s);

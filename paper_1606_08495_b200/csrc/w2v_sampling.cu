@@ -389,11 +389,40 @@ int launch_pair_offsets(uint64_t n, const Scratch &sc, DevState *st, cudaStream_
     return 3;
 }
 
+// centre[pair], context[pair] for every pair of the chunk (the word ids of the pair list, without the negatives)
+__global__ void __launch_bounds__(kBlock)
+pair_words_kernel(StepParams p, int32_t *__restrict__ centre, int32_t *__restrict__ context)
+{
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    const uint32_t nk = (uint32_t)p.st->n_kept;
+    for (uint32_t q = warp; q < nk; q += nwarps) {
+        const uint32_t w = p.win[q];
+        const uint32_t left = w & 0xFFu, cnt = left + (w >> 8);
+        if (cnt == 0) continue;
+        const int32_t c = p.ctok[q];
+        const unsigned long long pair0 = p.pair_off[q];
+        for (uint32_t j = lane; j < cnt; j += 32) {
+            centre[pair0 + j] = c;
+            context[pair0 + j] = p.ctok[q - left + j + (j >= left ? 1u : 0u)];
+        }
+    }
+}
+
 int launch_draw_negatives(const StepParams &p, int32_t *negs, int grid, cudaStream_t s)
 {
     draw_negatives_kernel<<<grid, kBlock, 0, s>>>(p, negs);
     if (cudaGetLastError() != cudaSuccess) return -1;
     return 1;
+}
+
+// the whole pair list of a step for the passes that stream over it: two launches
+int launch_pair_list(const StepParams &p, int32_t *centre, int32_t *context, int32_t *negs, int grid, cudaStream_t s)
+{
+    pair_words_kernel<<<grid, kBlock, 0, s>>>(p, centre, context);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    return launch_draw_negatives(p, negs, grid, s) < 0 ? -1 : 2;
 }
 
 int launch_emit_pairs(const StepParams &p, int32_t *centre, int32_t *context, int32_t *negs,
