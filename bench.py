@@ -598,6 +598,7 @@ def run_sharded(args):
                    "parallelism": f"{S} column shards run one after another on 1 gpu",
                    "pairs_per_step": tot_pairs / K,
                    "slowest_shard_ms_per_step": max(per_shard_ms) / K,
+                   "exchange_bytes_per_shard_and_step": 4.0 * tot_pairs / K * (1 + N),
                    "pairs_per_sec_if_each_shard_had_its_own_gpu_exchange_excluded": tot_pairs / (max(per_shard_ms) * 1e-3)},
         "clocks": clocks, "gpu_launches": launches,
         "roofline": {"bound": "hbm", "kernel": "shard_dots + coefficients + shard_du + snapshot passes 2-3",

@@ -45,6 +45,25 @@ def shard_columns(d: int, shards: int):
     return out
 
 
+def conventional_bytes_per_input_word(w: float, n: float, d: int) -> float:
+    """Eq. (2): bytes a conventional parameter server moves, in each direction, per minibatch input
+    word: the input and output vectors of the word plus the output vectors of its w * n negatives,
+    d single-precision numbers each."""
+    return (2.0 + w * n) * d * 4.0
+
+
+def exchange_bytes_per_input_word(w: float, n: float, shards: int) -> float:
+    """Eq. (7): bytes of partial dot products (or, in the other direction, of coefficients) per
+    minibatch input word summed over the shards: one 4-byte number per target and shard, whatever d."""
+    return w * (n + 1.0) * shards * 4.0
+
+
+def exchange_bytes_per_step(pairs: int, negatives: int) -> int:
+    """What ONE shard sends (and receives) in a step of this library: 4 bytes per target, the
+    per-shard term of Eq. (6) with b * w = the step's positive pairs."""
+    return 4 * int(pairs) * (1 + int(negatives))
+
+
 def _targets_capacity(n_tokens: int, window: int, negatives: int) -> int:
     return max(1, int(n_tokens) * 2 * int(window) * (1 + int(negatives)))
 

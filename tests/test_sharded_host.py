@@ -13,7 +13,8 @@ import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
 
-from paper_1606_08495_b200.sharded import shard_columns
+from paper_1606_08495_b200.sharded import (conventional_bytes_per_input_word, exchange_bytes_per_input_word,
+                                           exchange_bytes_per_step, shard_columns)
 
 
 @pytest.mark.parametrize("d,shards", [(300, 1), (300, 2), (300, 8), (300, 10), (300, 75), (8, 2), (1024, 16)])
@@ -74,3 +75,28 @@ def test_two_ranks_sum_their_slices_and_reduce_the_timing(tmp_path):
     mp.spawn(_rank_main, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
     for r in range(world):
         assert open(tmp_path / f"rank{r}.txt").read().split() == ["1", "1"]
+
+
+def test_network_bytes_of_the_paper():
+    # Section 4 works Eq. (2) for w = 10, n = 10, d = 500: about 200,000 bytes per word and direction, and
+    # from it, for 10 passes over 5e10 words in a week, at least 1300 Gbit/s
+    r = conventional_bytes_per_input_word(10, 10, 500)
+    assert r == 204_000 and abs(r - 200_000) / 200_000 < 0.03
+    gbits = 10 * 5e10 * 2e5 * 8 / (7 * 24 * 60 * 60 * 1e9)
+    assert 1300 <= gbits < 1330
+    # Section 5.2: the shards' partial dot products take S in the place of d, so the ratio is about S / d
+    for S, d in [(10, 300), (15, 300), (20, 1000), (25, 1000)]:
+        ratio = exchange_bytes_per_input_word(10, 10, S) / conventional_bytes_per_input_word(10, 10, d)
+        assert abs(ratio / (S / d) - 1) < 0.1
+        assert 1 / 100 - 1e-9 <= S / d <= 1 / 15
+    # Section 6.2: at 1.6e6 input words/s with about 20 targets per word on 15 shards the scheme needs a few
+    # Gbit/s of dot products each way where a conventional server would need ~300 Gbit/s for d = 300
+    words = 1.6e6
+    conventional = words * 21 * 300 * 4 * 8 / 1e9            # 21 vectors of 300 floats per input word
+    assert 300 <= conventional <= 340
+    ours = words * 20 * 15 * 4 * 8 / 1e9
+    assert ours < 20
+    # this library's exchange: one float per target per shard and direction
+    assert exchange_bytes_per_step(4_541_742, 10) == 4 * 4_541_742 * 11 == 199_836_648
+    b, w, n, S = 1000, 6, 5, 8
+    assert exchange_bytes_per_step(b * w, n) * S == b * exchange_bytes_per_input_word(w, n, S)
