@@ -70,12 +70,13 @@ __device__ __forceinline__ unsigned long long global_ns()
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
                                           unsigned long long limit_ns = kTcWaitNs)
 {
-    const unsigned long long t0 = global_ns();
+    unsigned long long t0 = 0;                                      // the clock is read only by a wait that lasts
     for (uint32_t spin = 0; spin < (1u << 30); ++spin) {
         if (mbar_try(bar, parity)) return true;
         if ((spin & 1023u) == 1023u) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > limit_ns) break;
+            if (!t0) t0 = global_ns();
+            else if (global_ns() - t0 > limit_ns) break;
         }
     }
     *abort_flag = 1;
@@ -779,30 +780,33 @@ topk_cosine_screen_kernel(TcParams p)
                                  (uint32_t)kScABlock, afull);
                 ok = mbar_wait(afull, 0u, abort_flag);
             }
-            uint64_t g = 0;
+            // One lane issues everything, so what it executes per MMA is what bounds the block when the
+            // copies keep up: the descriptors of a tile's MMAs differ only in their address fields, which
+            // advance by a constant per k-step (the K-blocks of an operand lie side by side), so the loop
+            // body is two additions and the MMA.
+            const uint32_t n16 = (4u * p.d4 + 15u) / 16u;                  // MMAs (K = 16) per tile; k-steps of pure padding are skipped
+            constexpr uint32_t kPerStage = 2u * kScKPS;                     // MMAs per full stage
+            constexpr uint64_t kAStep = (2u * kScAChunk) >> 4, kBStep = (2u * kScBChunk) >> 4, kStageStep = (uint32_t)kStage >> 4;
+            const uint64_t adesc0 = umma_desc(smem_addr(a_op), kScAChunk, 128), bdesc0 = umma_desc(smem_addr(b_op), kScBChunk, 128);
+            uint32_t s = 0, ph = 0;
             for (uint64_t i = 0; i < n_tiles && ok; ++i) {
                 const uint32_t b = (uint32_t)(i & 1);
                 ok = mbar_wait(tempty + b, (uint32_t)(((i >> 1) & 1) ^ 1), abort_flag);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t dst = tmem_base + b * kTcN;
-                for (uint32_t st = 0; st < nst && ok; ++st, ++g) {
-                    const uint32_t s = (uint32_t)(g % kScStages);
-                    ok = mbar_wait(full + s, (uint32_t)((g / kScStages) & 1), abort_flag);
+                uint64_t qa = adesc0;
+                uint32_t left = n16, acc = 0u;
+                while (left && ok) {
+                    ok = mbar_wait(full + s, ph, abort_flag);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    for (uint32_t kb = st * kScKPS; kb < nkb && kb < (st + 1) * kScKPS; ++kb) {
-                        const uint32_t j = kb - st * kScKPS;                                 // K-block within the stage
-                        const uint32_t abase = smem_addr(a_op + (RES ? (size_t)kb * kScABlock : (size_t)s * kStage + (size_t)j * kScABlock));
-                        const uint32_t bbase = smem_addr(b_op + (size_t)s * kStage + (size_t)j * kScStageBytes);
-                        const uint32_t cols = 4u * p.d4 - kb * kScKB < (uint32_t)kScKB ? 4u * p.d4 - kb * kScKB : (uint32_t)kScKB;
-                        const uint32_t nk = (cols + 15u) / 16u;                              // MMAs of K = 16 columns with data
-                        for (uint32_t kk = 0; kk < nk; ++kk) {
-                            const uint64_t qa = umma_desc(abase + 2 * kk * kScAChunk, kScAChunk, 128);
-                            const uint64_t cb = umma_desc(bbase + 2 * kk * kScBChunk, kScBChunk, 128);
-                            umma_bf16(dst, qa, cb, idesc, (kb | kk) ? 1u : 0u);
-                        }
-                    }
+                    uint64_t cb = bdesc0 + s * kStageStep;
+                    if (!RES) qa = adesc0 + s * kStageStep;
+                    const uint32_t n = left < kPerStage ? left : kPerStage;
+                    for (uint32_t t = 0; t < n; ++t, qa += kAStep, cb += kBStep, acc = 1u) umma_bf16(dst, qa, cb, idesc, acc);
+                    left -= n;
                     umma_commit(empty + s);                       // the stage is free once these MMAs have read it
+                    if (++s == (uint32_t)kScStages) { s = 0; ph ^= 1u; }
                 }
                 if (ok) umma_commit(tfull + b);                   // the tile's accumulator is complete
             }
@@ -812,20 +816,22 @@ topk_cosine_screen_kernel(TcParams p)
         // one bulk copy per stage, issued when the MMAs that read the stage's previous contents have
         // committed; its bytes complete the stage's "full" barrier
         if (lane == 0) {
-            const uint64_t total_g = n_tiles * nst;
-            uint64_t g = 0;
-            for (; g < total_g; ++g) {
-                const uint32_t s = (uint32_t)(g % kScStages);
-                if (!mbar_wait(empty + s, (uint32_t)(((g / kScStages) & 1) ^ 1), abort_flag)) break;
-                const uint32_t kb0 = (uint32_t)(g % nst) * kScKPS;                               // first K-block of the stage
-                const uint32_t nkbs = nkb - kb0 < (uint32_t)kScKPS ? nkb - kb0 : (uint32_t)kScKPS;  // K-blocks it holds
-                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
-                             ::"r"(smem_addr(full + s)), "r"(nkbs * (uint32_t)(RES ? kScStageBytes : kScABlock + kScStageBytes)) : "memory");
-                if (!RES)
-                    bulk_to_smem(a_op + (size_t)s * kStage, p.qsplit + ((size_t)blockIdx.x * nkb + kb0) * kScABlock,
-                                 nkbs * (uint32_t)kScABlock, full + s);
-                bulk_to_smem(b_op + (size_t)s * kStage,
-                             p.ctiles + ((t_lo + g / nst) * nkb + kb0) * (size_t)kScStageBytes, nkbs * (uint32_t)kScStageBytes, full + s);
+            uint64_t g = 0;                                                   // stages issued so far
+            uint32_t s = 0, ph = 1u;
+            const unsigned char *tile = p.ctiles + t_lo * nkb * (size_t)kScStageBytes;
+            const unsigned char *qsrc = RES ? nullptr : p.qsplit + (size_t)blockIdx.x * nkb * kScABlock;
+            for (uint64_t i = 0; i < n_tiles; ++i, tile += (size_t)nkb * kScStageBytes) {
+                uint32_t kb0 = 0;
+                for (; kb0 < nkb; kb0 += kScKPS, ++g) {
+                    if (!mbar_wait(empty + s, ph, abort_flag)) break;
+                    const uint32_t nkbs = nkb - kb0 < (uint32_t)kScKPS ? nkb - kb0 : (uint32_t)kScKPS;  // K-blocks the stage holds
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                                 ::"r"(smem_addr(full + s)), "r"(nkbs * (uint32_t)(RES ? kScStageBytes : kScABlock + kScStageBytes)) : "memory");
+                    if (!RES) bulk_to_smem(a_op + (size_t)s * kStage, qsrc + (size_t)kb0 * kScABlock, nkbs * (uint32_t)kScABlock, full + s);
+                    bulk_to_smem(b_op + (size_t)s * kStage, tile + (size_t)kb0 * kScStageBytes, nkbs * (uint32_t)kScStageBytes, full + s);
+                    if (++s == (uint32_t)kScStages) { s = 0; ph ^= 1u; }
+                }
+                if (kb0 < nkb) break;                                         // a wait ran out
             }
             if (*abort_flag) {
                 // the block is giving up: let the copies still in flight land before shared memory is released
@@ -892,7 +898,7 @@ __device__ __forceinline__ void mbar_arrive_in(uint64_t *bar, uint32_t rank)
 // the time-limited wait for a barrier that another block of the cluster arrives at
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
-    const unsigned long long t0 = global_ns();
+    unsigned long long t0 = 0;
     for (uint32_t spin = 0; spin < (1u << 30); ++spin) {
         uint32_t done;
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
@@ -900,7 +906,8 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity
         if (done) return true;
         if ((spin & 1023u) == 1023u) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > kTcWaitNs) break;
+            if (!t0) t0 = global_ns();
+            else if (global_ns() - t0 > kTcWaitNs) break;
         }
     }
     *abort_flag = 1;
@@ -987,29 +994,29 @@ topk_cosine_screen_pair_kernel(TcParams p)
             if (leader) {
                 // bf16 x bf16 -> fp32, both operands K-major, M = 256 and N = 256 over the pair
                 const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcN >> 3) << 17) | ((uint32_t)((2 * kTcM) >> 4) << 24);
-                uint64_t g = 0;
+                // as in the one-block kernel: address fields advance by a constant per k-step
+                const uint32_t n16 = (4u * p.d4 + 15u) / 16u;
+                constexpr uint32_t kPerStage = 2u * kPrKPS;
+                constexpr uint64_t kAStep = (2u * kScAChunk) >> 4, kBStep = (2u * kPrBChunk) >> 4, kStageStep = (uint32_t)kPrStage >> 4;
+                const uint64_t adesc0 = umma_desc(smem_addr(a_op), kScAChunk, 128), bdesc0 = umma_desc(smem_addr(b_op), kPrBChunk, 128);
+                uint32_t s = 0, ph = 0;
                 for (uint64_t i = 0; i < n_tiles && ok; ++i) {
                     const uint32_t b = (uint32_t)(i & 1);
                     ok = mbar_wait_cluster(tempty + b, (uint32_t)(((i >> 1) & 1) ^ 1), abort_flag);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t dst = tmem_base + b * kTcN;
-                    for (uint32_t st = 0; st < nst && ok; ++st, ++g) {
-                        const uint32_t s = (uint32_t)(g % kPrStages), ph = (uint32_t)((g / kPrStages) & 1);
+                    uint64_t qa = adesc0;
+                    uint32_t left = n16, acc = 0u;
+                    while (left && ok) {
                         ok = mbar_wait(full + s, ph, abort_flag) && mbar_wait_cluster(fullF + s, ph, abort_flag);
                         if (!ok) break;
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        for (uint32_t kb = st * kPrKPS; kb < nkb && kb < (st + 1) * kPrKPS; ++kb) {
-                            const uint32_t abase = smem_addr(a_op + (size_t)kb * kScABlock);
-                            const uint32_t bbase = smem_addr(b_op + (size_t)s * kPrStage + (size_t)(kb - st * kPrKPS) * kPrKBlock);
-                            const uint32_t cols = 4u * p.d4 - kb * kScKB < (uint32_t)kScKB ? 4u * p.d4 - kb * kScKB : (uint32_t)kScKB;
-                            const uint32_t nk = (cols + 15u) / 16u;
-                            for (uint32_t kk = 0; kk < nk; ++kk) {
-                                const uint64_t qa = umma_desc(abase + 2 * kk * kScAChunk, kScAChunk, 128);
-                                const uint64_t cb = umma_desc(bbase + 2 * kk * kPrBChunk, kPrBChunk, 128);
-                                umma_bf16_pair(dst, qa, cb, idesc, (kb | kk) ? 1u : 0u);
-                            }
-                        }
+                        uint64_t cb = bdesc0 + s * kStageStep;
+                        const uint32_t n = left < kPerStage ? left : kPerStage;
+                        for (uint32_t t = 0; t < n; ++t, qa += kAStep, cb += kBStep, acc = 1u) umma_bf16_pair(dst, qa, cb, idesc, acc);
+                        left -= n;
                         umma_commit_pair(empty + s);
+                        if (++s == (uint32_t)kPrStages) { s = 0; ph ^= 1u; }
                     }
                     if (ok) umma_commit_pair(tfull + b);
                 }
@@ -1018,17 +1025,21 @@ topk_cosine_screen_pair_kernel(TcParams p)
     } else if (warp == 5) {
         // producer: the own half of every stage
         if (lane == 0) {
-            uint64_t g = 0;
-            for (; g < total_g; ++g) {
-                const uint32_t s = (uint32_t)(g % kPrStages), ph = (uint32_t)(((g / kPrStages) & 1) ^ 1);
-                if (!(leader ? mbar_wait(empty + s, ph, abort_flag) : mbar_wait_cluster(empty + s, ph, abort_flag))) break;
-                const uint32_t kb0 = (uint32_t)(g % nst) * kPrKPS;
-                const uint32_t nkbs = nkb - kb0 < (uint32_t)kPrKPS ? nkb - kb0 : (uint32_t)kPrKPS;
-                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
-                             ::"r"(smem_addr(full + s)), "r"(nkbs * (uint32_t)kPrKBlock) : "memory");
-                // half tile number 2 T + rank of the packed copy (tiles of 128 rows)
-                bulk_to_smem(b_op + (size_t)s * kPrStage,
-                             p.ctiles + ((2 * (t_lo + g / nst) + rank) * nkb + kb0) * (size_t)kPrKBlock, nkbs * (uint32_t)kPrKBlock, full + s);
+            uint64_t g = 0;                                                   // stages issued so far
+            uint32_t s = 0, ph = 1u;
+            // half tile number 2 T + rank of the packed copy (tiles of 128 rows)
+            const unsigned char *tile = p.ctiles + (2 * t_lo + rank) * nkb * (size_t)kPrKBlock;
+            for (uint64_t i = 0; i < n_tiles; ++i, tile += 2 * (size_t)nkb * kPrKBlock) {
+                uint32_t kb0 = 0;
+                for (; kb0 < nkb; kb0 += kPrKPS, ++g) {
+                    if (!(leader ? mbar_wait(empty + s, ph, abort_flag) : mbar_wait_cluster(empty + s, ph, abort_flag))) break;
+                    const uint32_t nkbs = nkb - kb0 < (uint32_t)kPrKPS ? nkb - kb0 : (uint32_t)kPrKPS;
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                                 ::"r"(smem_addr(full + s)), "r"(nkbs * (uint32_t)kPrKBlock) : "memory");
+                    bulk_to_smem(b_op + (size_t)s * kPrStage, tile + (size_t)kb0 * kPrKBlock, nkbs * (uint32_t)kPrKBlock, full + s);
+                    if (++s == (uint32_t)kPrStages) { s = 0; ph ^= 1u; }
+                }
+                if (kb0 < nkb) break;                                         // a wait ran out
             }
             if (*abort_flag) {
                 for (uint64_t j = g > (uint64_t)kPrStages ? g - kPrStages : 0; j < g; ++j)
