@@ -617,7 +617,7 @@ __device__ __forceinline__ void screen_epilogue(const TcParams &p, const long lo
             if (!owners) break;
             bool on[kExact];
             uint32_t src[kExact], hv[kExact];
-            float th[kExact], fl[kExact], qi[kExact], dot[kExact], e0[kExact], e1[kExact];
+            float th[kExact], fl[kExact], qi[kExact], dot[kExact], e0[kExact], e1[kExact], cinv[kExact];
             long long i0[kExact], i1[kExact], qr[kExact];
             uint64_t cnd[kExact];
 #pragma unroll
@@ -633,8 +633,9 @@ __device__ __forceinline__ void screen_epilogue(const TcParams &p, const long lo
                 fl[e] = __shfl_sync(kFullMask, flo, src[e]);
                 qi[e] = __shfl_sync(kFullMask, qinv, src[e]);
                 if (on[e] && lane == src[e]) maybe &= maybe - 1u;
-                e0[e] = 0.f; e1[e] = 0.f; i0[e] = -1; i1[e] = -1; dot[e] = 0.f;
+                e0[e] = 0.f; e1[e] = 0.f; i0[e] = -1; i1[e] = -1; dot[e] = 0.f; cinv[e] = 0.f;
                 if (on[e]) {
+                    cinv[e] = __ldg(p.inv_norm + cnd[e]);                   // fetched with the rows, not after the sum
                     const size_t lb = ((size_t)list * p.m + (q0 + warp * 32u + src[e])) * p.K;
                     if (lane < hv[e]) { e0[e] = __ldcg(p.part_cos + lb + lane); i0[e] = __ldcg(p.part_ids + lb + lane); }
                     if (lane + 32u < hv[e]) { e1[e] = __ldcg(p.part_cos + lb + lane + 32u); i1[e] = __ldcg(p.part_ids + lb + lane + 32u); }
@@ -659,7 +660,7 @@ __device__ __forceinline__ void screen_epilogue(const TcParams &p, const long lo
 #pragma unroll
             for (int e = 0; e < kExact; ++e) {
                 if (!on[e]) continue;                                                   // same for every lane
-                const float cs = dot[e] * qi[e] * __ldg(p.inv_norm + cnd[e]);
+                const float cs = dot[e] * qi[e] * cinv[e];
                 const long long cid = (long long)(p.cand_lo + cnd[e]);
                 if (!(cs > p.tau) || cid == qr[e] || (hv[e] == p.K && cs < th[e]) || cs < fl[e]) continue;
                 const size_t lb = ((size_t)list * p.m + (q0 + warp * 32u + src[e])) * p.K;
