@@ -739,7 +739,6 @@ topk_cosine_screen_kernel(TcParams p)
     const uint64_t tiles = (nc + kTcN - 1) / kTcN;
     const uint64_t t_lo = tiles * blockIdx.y / p.splits, t_hi = tiles * (blockIdx.y + 1) / p.splits;
     const uint32_t nkb = (4u * p.d4 + kScKB - 1) / kScKB;
-    const uint32_t nst = (nkb + kScKPS - 1) / kScKPS;                       // stages per tile
     const uint64_t n_tiles = t_hi - t_lo;
 
     if (tid == 0) {
