@@ -767,7 +767,11 @@ int32_t w2v_topk_cosine(w2v_handle *h, uint32_t which, const int64_t *queries, u
     // the screening kernel takes the candidates in chunks, each with its own set of partial lists
     const uint64_t chunk = screen ? topk_screen_chunk(nc, h->d) : nc;
     const uint64_t chunks = chunk ? (nc + chunk - 1) / chunk : 0;
-    const uint64_t splits = tc ? topk_splits(m, chunk, h->sms, 128, 256) : topk_splits(m, nc, h->sms);
+    // Every split builds a list of its own per query.  With a threshold that few candidates pass that costs
+    // nothing; without one (tau <= -1: plain top-K) each list takes some K ln(n / K) exact cosines to fill, so
+    // the screening kernel then settles for fewer, longer splits (a last wave 85 % full instead of 95 %).
+    const uint64_t splits = tc ? topk_splits(m, chunk, h->sms, 128, 256, screen && tau <= -1.0f ? 0.85 : 0.95)
+                               : topk_splits(m, nc, h->sms);
     const uint64_t lists = screen ? chunks * splits : splits;
     const uint64_t need = (splits > 1 || tc) ? lists * m * K : 0;
     if (screen && m > h->floor_cap) {

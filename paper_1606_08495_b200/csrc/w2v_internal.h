@@ -163,7 +163,7 @@ int launch_probe_bulk_ring(const unsigned char *src, unsigned long long span, ui
                            uint32_t copies, uint32_t producers, int *error, int sms, cudaStream_t s);
 
 // ---- cosine retrieval (w2v_topk.cu) ----
-uint32_t topk_splits(uint64_t m, uint64_t n_candidates, int sms, uint32_t block_queries = 0, uint32_t tile_rows = 0);
+uint32_t topk_splits(uint64_t m, uint64_t n_candidates, int sms, uint32_t block_queries = 0, uint32_t tile_rows = 0, double min_fill = 0.95);
 int launch_topk_merge(const float *part_cos, const long long *part_ids, uint64_t m, uint32_t K, uint32_t splits,
                       float *out_cos, long long *out_ids, int sms, cudaStream_t s);
 // tensor-core variant (w2v_topk_tc.cu): partial lists only, 128 queries per block, tiles of 256 candidates

@@ -311,9 +311,9 @@ size_t topk_smem_bytes(uint32_t d, uint32_t K, int BQ)
 }
 
 // How many ways to split the candidates so that the grid fills whole waves of one block per SM:
-// the smallest split count (at most 64, at most one per tile) whose last wave is at least 95 % full,
-// else the fullest one.
-uint32_t topk_splits(uint64_t m, uint64_t n_candidates, int sms, uint32_t block_queries, uint32_t tile_rows)
+// the smallest split count (at most 64, at most one per tile) whose last wave is at least `min_fill`
+// full (95 % unless given), else the fullest one.
+uint32_t topk_splits(uint64_t m, uint64_t n_candidates, int sms, uint32_t block_queries, uint32_t tile_rows, double min_fill)
 {
     if (block_queries == 0) { block_queries = 64; tile_rows = kTopkBC; }
     const uint64_t qblocks = (m + block_queries - 1) / block_queries, tiles = (n_candidates + tile_rows - 1) / tile_rows;
@@ -324,7 +324,7 @@ uint32_t topk_splits(uint64_t m, uint64_t n_candidates, int sms, uint32_t block_
         const uint64_t blocks = qblocks * sp, waves = (blocks + sms - 1) / sms;
         const double fill = (double)blocks / (double)(waves * sms);
         if (fill > best_fill + 1e-9) { best_fill = fill; best = (uint32_t)sp; }
-        if (fill >= 0.95) return (uint32_t)sp;
+        if (fill >= min_fill) return (uint32_t)sp;
     }
     return best;
 }
