@@ -769,8 +769,14 @@ def run_probe(args):
         model.sync()
         ring[f"{stage}B_x{stages}_stages_{producers}_producer"] = {"ms": best, "GBps_per_sm": done / (best * 1e-3) / 1e9,
                                                                    "ns_per_stage": best * 1e6 / (done / stage)}
+    # producer lanes, ring and MMA issuer coupled, without an epilogue: SM cycles per 19-MMA tile (2432 at the pipe's rate)
+    feed = {}
+    tiles = int(min(3900, cfg["vocab"] * row_stride * 4 // 3 // 163840))
+    for kps, stages, span in ((3, 3, 0), (3, 3, 1), (2, 4, 0), (2, 4, 1), (4, 2, 1), (1, 9, 0)):
+        cyc, waited = binding.w2v_probe_mma_ring(model.h, kps, stages, tiles, span)
+        feed[f"{kps}_kblocks_x{stages}_stages_{'spanning_tiles' if span else 'per_tile'}"] = {"cycles_per_tile": cyc, "of_them_waiting_for_data": waited}
     line = {"metric": "random_row_traffic", "unit": "GB/s of row bytes (read + written)", "n_gpus": 1,
-            "bulk_copy_ring": ring,
+            "bulk_copy_ring": ring, "mma_ring_cycles_per_tile": feed,
             "config": {"workload": name + " (memory-system probe)", "vocab": cfg["vocab"], "d": d,
                        "row_stride_floats": row_stride, "rows_per_launch": rows,
                        "table_GB": cfg["vocab"] * row_stride * 4 / 1e9},

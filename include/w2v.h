@@ -457,6 +457,25 @@ int32_t w2v_probe_bulk_ring(w2v_handle *h, uint32_t stage_bytes, uint32_t stages
                             uint64_t bytes_per_sm, double *ms, uint64_t *bytes_done);
 
 /*
+ * Third measuring aid (no counterpart in the paper): what the feed of the retrieval screen can reach
+ * without its epilogue.  One block per SM holds an 80 KB query operand in shared memory; two producer
+ * lanes fill a ring of `stages` slots of `kblocks_per_stage` K-blocks (16 KB each, ten per tile of 256
+ * candidates) with one bulk copy per slot; one lane issues each tile's 19 bf16 MMAs (128 x 256 x 16) from
+ * the slots and commits the slot's release.  Groups of 64 blocks read the same stream of bytes of V
+ * (interpreted as bf16: only the timing matters), as the blocks of one candidate split do.
+ *   kblocks_per_stage * stages  at most 9 (144 KB of ring);  stages at least 2.
+ *   tiles        tiles per block; three streams of tiles * 160 KB must fit into V.
+ *   span_tiles   non-zero: a slot holds the next K-blocks whichever tile they belong to; zero: slots do
+ *                not span tiles (the last slot of a tile is short), as in the committed kernel.
+ *   cycles_per_tile, wait_cycles_per_tile  host; SM cycles per tile of block 0's MMA lane, and the part of
+ *                them it spent waiting for data.  The tensor pipe alone needs 19 x 128 = 2432.
+ * Reads V only.  Synchronises the stream.  All waits are bounded; a block that gives up makes
+ * the next w2v_sync return W2V_ERR_CUDA.
+ */
+int32_t w2v_probe_mma_ring(w2v_handle *h, uint32_t kblocks_per_stage, uint32_t stages, uint32_t tiles, uint32_t span_tiles,
+                           double *cycles_per_tile, double *wait_cycles_per_tile);
+
+/*
  * Launch shape of the update kernels: rows in flight per warp (1..8; 0 = default)
  * and resident thread blocks per SM (0 = as many as fit).  Results do not depend
  * on it in snapshot mode.

@@ -28,7 +28,7 @@ EXPORTS = (
     "w2v_set_step", "w2v_get_step", "w2v_get_table_ptrs", "w2v_sync", "w2v_profile_enable",
     "w2v_profile_read", "w2v_get_launch_count", "w2v_set_tuning", "w2v_last_error",
     "w2v_sample_pairs_noalloc", "w2v_peer_barrier", "w2v_probe_rows",
-    "w2v_selftest_bounded_wait", "w2v_probe_bulk_ring",
+    "w2v_selftest_bounded_wait", "w2v_probe_bulk_ring", "w2v_probe_mma_ring",
 )
 
 
@@ -77,6 +77,7 @@ def load():
         "w2v_probe_rows": [vp, u32, u64, u64, C.POINTER(C.c_double), C.POINTER(u64)],
         "w2v_selftest_bounded_wait": [vp, u32],
         "w2v_probe_bulk_ring": [vp, u32, u32, u32, u64, C.POINTER(C.c_double), C.POINTER(u64)],
+        "w2v_probe_mma_ring": [vp, u32, u32, u32, u32, C.POINTER(C.c_double), C.POINTER(C.c_double)],
         "w2v_destroy": [vp],
         "w2v_build_alias": [vp, vp, C.c_double],
         "w2v_get_tables": [vp, vp, vp, vp],
@@ -191,6 +192,14 @@ def w2v_probe_bulk_ring(h, stage_bytes, stages, producers, bytes_per_sm):
     _check(h, load().w2v_probe_bulk_ring(h, int(stage_bytes), int(stages), int(producers), int(bytes_per_sm),
                                          C.byref(ms), C.byref(done)))
     return ms.value, int(done.value)
+
+
+def w2v_probe_mma_ring(h, kblocks_per_stage, stages, tiles, span_tiles):
+    """(SM cycles per tile, cycles of them spent waiting for data) of the producer / ring / MMA probe."""
+    cyc, waited = C.c_double(0.0), C.c_double(0.0)
+    _check(h, load().w2v_probe_mma_ring(h, int(kblocks_per_stage), int(stages), int(tiles), int(bool(span_tiles)),
+                                        C.byref(cyc), C.byref(waited)))
+    return cyc.value, waited.value
 
 
 def w2v_selftest_bounded_wait(h, timeout_ms):

@@ -902,6 +902,34 @@ int32_t w2v_probe_bulk_ring(w2v_handle *h, uint32_t stage_bytes, uint32_t stages
     return W2V_OK;
 }
 
+int32_t w2v_probe_mma_ring(w2v_handle *h, uint32_t kblocks_per_stage, uint32_t stages, uint32_t tiles, uint32_t span_tiles,
+                           double *cycles_per_tile, double *wait_cycles_per_tile)
+{
+    if (!h) return W2V_ERR_ARG;
+    if (!cycles_per_tile || !wait_cycles_per_tile) return fail(h, W2V_ERR_ARG, "an output pointer is NULL");
+    if (kblocks_per_stage < 1 || stages < 2 || (uint64_t)kblocks_per_stage * stages > 9)
+        return fail(h, W2V_ERR_ARG, "need at least 2 stages and at most 9 K-blocks (144 KB) in the ring");
+    if (tiles < 1 || tiles > (1u << 20)) return fail(h, W2V_ERR_ARG, "tiles must be in 1..2^20");
+    // three streams (one per group of 64 blocks) of tiles x 160 KB each must fit into the output table
+    const uint64_t table_bytes = (uint64_t)h->vocab * h->ld * sizeof(float);
+    const uint64_t stream = (uint64_t)tiles * 10u * 16384u;
+    const uint64_t groups = ((uint64_t)h->sms + 63) / 64;
+    if (stream * groups > table_bytes || stream < 81920) return fail(h, W2V_ERR_ARG, "the table is too small for this many tiles");
+    DeviceGuard g(h->device);
+    int32_t rc;
+    if ((rc = ensure_error_word(h)) != W2V_OK) return rc;
+    const int k = launch_probe_mma_ring(reinterpret_cast<const unsigned char *>(h->V), stream, kblocks_per_stage, stages, tiles,
+                                        span_tiles ? 1u : 0u, h->tc_error, h->sms, h->stream);
+    if (k < 0) return fail(h, W2V_ERR_CUDA, "probe launch", cudaGetLastError());
+    h->launches += (uint64_t)k;
+    W2V_CUDA(h, cudaStreamSynchronize(h->stream));
+    long long cyc = 0, waited = 0;
+    if (read_probe_mma_ring(&cyc, &waited) != 0) return fail(h, W2V_ERR_CUDA, "probe read-back", cudaGetLastError());
+    *cycles_per_tile = (double)cyc / tiles;
+    *wait_cycles_per_tile = (double)waited / tiles;
+    return W2V_OK;
+}
+
 int32_t w2v_set_step(w2v_handle *h, uint64_t step_id)
 {
     if (!h) return W2V_ERR_ARG;

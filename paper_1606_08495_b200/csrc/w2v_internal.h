@@ -159,6 +159,9 @@ int launch_probe_rows(float *V, const uint2 *alias, uint32_t vocab, uint32_t d4,
                       unsigned long long *rows_done);
 
 // one block per SM pulls `copies` bulk copies of stage_bytes from src[0, span) through a ring of `stages` slots
+int launch_probe_mma_ring(const unsigned char *src, unsigned long long stream_stride, uint32_t kps, uint32_t stages, uint32_t tiles,
+                          uint32_t span_tiles, int *error, int sms, cudaStream_t s);
+int read_probe_mma_ring(long long *cycles, long long *waited);
 int launch_probe_bulk_ring(const unsigned char *src, unsigned long long span, uint32_t stage_bytes, uint32_t stages,
                            uint32_t copies, uint32_t producers, int *error, int sms, cudaStream_t s);
 

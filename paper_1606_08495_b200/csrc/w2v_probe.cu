@@ -154,6 +154,130 @@ probe_bulk_ring_kernel(const unsigned char *src, unsigned long long span, uint32
     if (threadIdx.x == 0 && abort_word) atomicExch(error, 4);
 }
 
+// ---- producer, ring and MMA issuer coupled, without an epilogue ------------------------------------
+// What the retrieval screen's feed can reach at best: one block per SM with an 80 KB query operand in
+// shared memory, a ring of `stages` slots of `kps` K-blocks (16 KB each, 10 per 256-candidate tile), two
+// producer lanes issuing one bulk copy per slot, and one lane issuing the tile's 19 bf16 MMAs
+// (128 x 256 x 16) from the slots and committing each slot's "empty" barrier.  Nobody reads the two
+// accumulators.  span_tiles = 1: a slot holds the next kps K-blocks whichever tile they belong to;
+// 0: slots do not span tiles (the tile's last slot is short).  Groups of 64 blocks read the same stream,
+// as the blocks of one candidate split do.  The operands are whatever bytes the table holds, read as
+// bf16: only the timing is of interest.  Waits are bounded; a block that gives up raises *error.
+constexpr int kRingA = 10 * 4 * 128 * 16;               // the query operand: 10 K-blocks x 4 chunks x 128 rows x 16 B
+constexpr int kRingKB = 4 * 256 * 16;                   // one K-block of a candidate tile
+__device__ long long g_probe_cycles[2];                 // block 0: cycles of the MMA lane's loop, cycles it waited for data
+
+__device__ __forceinline__ uint64_t probe_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo)
+{
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+__device__ __forceinline__ void probe_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}\n"
+                 ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0), "r"(0), "r"(0), "r"(0) : "memory");
+}
+__device__ __forceinline__ void probe_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(probe_saddr(bar)) : "memory");
+}
+
+__global__ void __launch_bounds__(128, 1)
+probe_mma_ring_kernel(const unsigned char *src, unsigned long long stream_stride, uint32_t kps, uint32_t stages, uint32_t tiles,
+                      uint32_t span_tiles, int *error)
+{
+    extern __shared__ __align__(128) unsigned char probe_smem[];
+    unsigned char *As = probe_smem, *Bs = probe_smem + kRingA;
+    const uint32_t stage_bytes = kps * (uint32_t)kRingKB;
+    uint64_t *full = reinterpret_cast<uint64_t *>(Bs + (size_t)stages * stage_bytes), *empty = full + stages, *done = empty + stages;
+    uint32_t *slot = reinterpret_cast<uint32_t *>(done + 1);
+    __shared__ int abort_word;
+    volatile int *abort_flag = &abort_word;
+    const uint32_t tid = threadIdx.x, warp = tid >> 5;
+    const unsigned char *stream = src + (unsigned long long)(blockIdx.x / 64u) * stream_stride;
+    for (uint32_t i = tid; i < (uint32_t)kRingA / 16u; i += 128) reinterpret_cast<uint4 *>(As)[i] = reinterpret_cast<const uint4 *>(stream)[i];
+    if (tid == 0) {
+        abort_word = 0;
+        for (uint32_t i = 0; i < 2 * stages + 1; ++i)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(probe_saddr(full + i)), "r"(1));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(probe_saddr(slot)), "r"(512));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");         // the operand was written by ordinary stores
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tm = *slot;
+    const uint32_t nkb = 10, total_kb = tiles * nkb;
+    const uint32_t spt = (nkb + kps - 1) / kps;                          // slots per tile when slots do not span tiles
+    const uint32_t total_g = span_tiles ? (total_kb + kps - 1) / kps : tiles * spt;
+    if (tid == 0) {
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        const uint64_t a0 = probe_desc(probe_saddr(As), 128 * 16, 128), b0 = probe_desc(probe_saddr(Bs), 256 * 16, 128);
+        constexpr uint64_t aS = (2 * 128 * 16) >> 4, bS = (2 * 256 * 16) >> 4;
+        long long waited = 0;
+        const long long t0 = clock64();
+        uint32_t s = 0, ph = 0, kb = 0, tile = 0;
+        bool ok = true;
+        for (uint32_t g = 0; g < total_g; ++g) {
+            const long long w0 = clock64();
+            ok = probe_wait(full + s, ph, abort_flag);
+            if (!ok) break;
+            waited += clock64() - w0;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t cnt = span_tiles ? (total_kb - g * kps < kps ? total_kb - g * kps : kps) : (nkb - kb < kps ? nkb - kb : kps);
+            uint64_t cb = b0 + (uint64_t)s * (stage_bytes >> 4);
+            for (uint32_t j = 0; j < cnt; ++j) {
+                const uint32_t d = tm + (tile & 1u) * 256u;
+                probe_mma(d, a0 + kb * 2 * aS, cb, idesc, kb ? 1u : 0u);
+                if (kb + 1 < nkb) probe_mma(d, a0 + kb * 2 * aS + aS, cb + bS, idesc, 1u);     // the tile's last K-block: one k-step of data
+                cb += 2 * bS;
+                if (++kb == nkb) { kb = 0; ++tile; }
+            }
+            probe_commit(empty + s);
+            if (++s == stages) { s = 0; ph ^= 1u; }
+        }
+        const long long t1 = clock64();
+        probe_commit(done);                                               // every MMA has completed before tensor memory is released
+        if (ok) probe_wait(done, 0u, abort_flag);
+        if (blockIdx.x == 0) { g_probe_cycles[0] = t1 - t0; g_probe_cycles[1] = waited; }
+    } else if (tid == 32 || tid == 64) {
+        // Stages alternate between the two lanes.  With two or more slots a lane that has passed its wait for
+        // slot use u - 1 has thereby seen every earlier release of that slot, so the parity it waits on next
+        // cannot be mistaken for an older phase.
+        const uint32_t w = tid == 32 ? 0u : 1u;
+        uint32_t g = w;
+        for (; g < total_g; g += 2) {
+            const uint32_t s = g % stages;
+            if (!probe_wait(empty + s, ((g / stages) & 1u) ^ 1u, abort_flag)) break;
+            uint32_t kb_first, cnt;
+            if (span_tiles) { kb_first = g * kps; cnt = total_kb - kb_first < kps ? total_kb - kb_first : kps; }
+            else { const uint32_t t = g / spt, st = g - t * spt; kb_first = t * nkb + st * kps; cnt = nkb - st * kps < kps ? nkb - st * kps : kps; }
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(probe_saddr(full + s)), "r"(cnt * (uint32_t)kRingKB) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(probe_saddr(Bs + (size_t)s * stage_bytes)), "l"(stream + (unsigned long long)kb_first * kRingKB),
+                           "r"(cnt * (uint32_t)kRingKB), "r"(probe_saddr(full + s)) : "memory");
+        }
+        // this lane's copies still in flight land before shared memory goes away
+        for (uint32_t back = 2; back <= stages + 1u && back <= g; back += 2) {
+            const uint32_t j = g - back;
+            for (uint32_t spin = 0; spin < (1u << 20); ++spin)
+                if (probe_try(full + j % stages, (j / stages) & 1u)) break;
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (tid == 0 && abort_word) atomicExch(error, 4);
+    if (warp == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(512));
+    }
+}
+
 }  // namespace
 
 int launch_probe_bulk_ring(const unsigned char *src, unsigned long long span, uint32_t stage_bytes, uint32_t stages,
@@ -163,6 +287,24 @@ int launch_probe_bulk_ring(const unsigned char *src, unsigned long long span, ui
     if (cudaFuncSetAttribute(probe_bulk_ring_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess) return -1;
     probe_bulk_ring_kernel<<<sms, 256, sm, s>>>(src, span, stage_bytes, stages, copies, producers, error);
     return cudaGetLastError() != cudaSuccess ? -1 : 1;
+}
+
+int launch_probe_mma_ring(const unsigned char *src, unsigned long long stream_stride, uint32_t kps, uint32_t stages, uint32_t tiles,
+                          uint32_t span_tiles, int *error, int sms, cudaStream_t s)
+{
+    const size_t sm = (size_t)kRingA + (size_t)stages * kps * kRingKB + 16 * (size_t)stages + 64;
+    if (cudaFuncSetAttribute(probe_mma_ring_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess) return -1;
+    probe_mma_ring_kernel<<<sms, 128, sm, s>>>(src, stream_stride, kps, stages, tiles, span_tiles, error);
+    return cudaGetLastError() != cudaSuccess ? -1 : 1;
+}
+
+// cycles of block 0's MMA lane (whole loop, and the part spent waiting for data); call after the stream has been synchronised
+int read_probe_mma_ring(long long *cycles, long long *waited)
+{
+    long long v[2];
+    if (cudaMemcpyFromSymbol(v, g_probe_cycles, sizeof v) != cudaSuccess) return -1;
+    *cycles = v[0]; *waited = v[1];
+    return 0;
 }
 
 int launch_probe_rows(float *V, const uint2 *alias, uint32_t vocab, uint32_t d4, uint32_t ld4, uint32_t span,

@@ -497,8 +497,17 @@ def test_memory_probe_leaves_the_table_as_it_was():
     for stage, stages, producers in ((4096, 4, 1), (16384, 3, 2), (1024, 64, 4)):
         ms, done = binding.w2v_probe_bulk_ring(gpu.h, stage, stages, producers, 1 << 20)
         assert ms > 0 and done == (1 << 20) // stage * stage
+    # and so does the producer / ring / MMA pipeline (two streams of 5 tiles fit this table; the tensor
+    # pipe alone needs 19 x 128 cycles per tile, so no configuration can be faster than that)
+    for kps, stages, span in ((3, 3, 0), (3, 3, 1), (2, 4, 1), (1, 9, 0), (4, 2, 1)):
+        cyc, waited = binding.w2v_probe_mma_ring(gpu.h, kps, stages, 5, span)
+        assert cyc >= 19 * 128 * 0.9 and 0 <= waited <= cyc
     gpu.sync()
     assert np.array_equal(gpu.read_rows(1, ids), Vv)
+    for args in ((3, 1, 5, 0), (5, 2, 5, 0), (0, 3, 5, 0), (3, 3, 0, 0), (3, 3, 100, 0)):       # one stage, ring too large, ..., table too small
+        with pytest.raises(binding.W2VError) as e:
+            binding.w2v_probe_mma_ring(gpu.h, *args)
+        assert e.value.code == binding.W2V_ERR_ARG
     for args in ((24, 4, 1, 1 << 20), (4096, 0, 1, 1 << 20), (65536, 4, 1, 1 << 20), (4096, 4, 5, 1 << 20), (4096, 4, 1, 100)):
         with pytest.raises(binding.W2VError) as e:
             binding.w2v_probe_bulk_ring(gpu.h, *args)
