@@ -499,6 +499,68 @@ topk_pack_candidates_kernel(const float *__restrict__ table, float *__restrict__
 }
 
 // fp32 dot product of two table rows by the whole warp (every lane gets the sum)
+// The same packed copy for rows of at most 320 columns, staged through shared memory: sixteen warps read
+// the tile's rows with coalesced 16-byte loads (four rows per warp in flight), reduce the norm with
+// shuffles and write the scaled bf16 values into a shared-memory image of the tile (chunk stride padded
+// by 16 bytes against bank conflicts); the image then goes out as one contiguous run.  Every row is read
+// once and every output byte written once, in whole lines (the one-thread-per-row kernel above moves
+// 1.5 times the bytes).
+constexpr int kPackThreads = 512;
+constexpr uint32_t kPackMaxF = 96;                                // float4 slots per row a lane can hold (3 x 32)
+template <int NT>
+__global__ void __launch_bounds__(kPackThreads)
+topk_pack_candidates_smem_kernel(const float *__restrict__ table, float *__restrict__ inv_norm, uint32_t d4, uint32_t ld4,
+                                 uint64_t cand_lo, uint64_t nc, uint64_t tiles, uint32_t nkb, unsigned char *__restrict__ out)
+{
+    extern __shared__ __align__(16) unsigned char pack_stage[];
+    constexpr uint32_t kChunk = NT * 16, kPad = kChunk + 16;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t nf = nkb * (kScKB / 4);                         // float4 slots per row of the packed copy (zeros from d4 on)
+    for (uint64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+        for (uint32_t r0 = warp * 4; r0 < (uint32_t)NT; r0 += (kPackThreads / 32) * 4) {
+            float4 x[4][3];
+            bool valid[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const uint64_t c = tile * NT + r0 + t;
+                valid[t] = c < nc;
+                const float4 *row = reinterpret_cast<const float4 *>(table) + (size_t)(cand_lo + (valid[t] ? c : 0)) * ld4;
+#pragma unroll
+                for (int k = 0; k < 3; ++k) {
+                    const uint32_t f = lane + 32u * k;
+                    x[t][k] = valid[t] && f < d4 ? __ldg(row + f) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                float q = 0.f;
+#pragma unroll
+                for (int k = 0; k < 3; ++k) {
+                    q = fmaf(x[t][k].x, x[t][k].x, q); q = fmaf(x[t][k].y, x[t][k].y, q);
+                    q = fmaf(x[t][k].z, x[t][k].z, q); q = fmaf(x[t][k].w, x[t][k].w, q);
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(kFullMask, q, o);
+                const float ic = q > 0.f ? 1.0f / sqrtf(q) : 0.f;   // unit rows: an accumulator column times 1/|query| is a cosine
+                if (lane == 0 && valid[t]) inv_norm[tile * NT + r0 + t] = ic;
+#pragma unroll
+                for (int k = 0; k < 3; ++k) {
+                    const uint32_t f = lane + 32u * k;
+                    if (f < nf)
+                        *reinterpret_cast<uint2 *>(pack_stage + (size_t)(f >> 1) * kPad + (r0 + t) * 16u + (f & 1u) * 8u) =
+                            make_uint2(bf16x2(x[t][k].x * ic, x[t][k].y * ic), bf16x2(x[t][k].z * ic, x[t][k].w * ic));
+                }
+            }
+        }
+        __syncthreads();
+        uint4 *dst = reinterpret_cast<uint4 *>(out + tile * nkb * (size_t)(kScCh * kChunk));
+        const uint32_t total = nkb * kScCh * NT;
+        for (uint32_t i = threadIdx.x; i < total; i += kPackThreads)
+            dst[i] = *reinterpret_cast<const uint4 *>(pack_stage + (size_t)(i / NT) * kPad + (i % NT) * 16u);
+        __syncthreads();
+    }
+}
+
 __device__ __forceinline__ float warp_row_dot(const float4 *__restrict__ T4, size_t a, size_t b, uint32_t d4, uint32_t ld4,
                                               uint32_t lane)
 {
@@ -1205,7 +1267,15 @@ int launch_topk_tc(const float *table, uint32_t d, uint32_t ld, uint64_t vocab, 
     for (uint64_t c0 = 0; c0 < nc; c0 += chunk, ++list) {
         const uint64_t n = nc - c0 < chunk ? nc - c0 : chunk;
         const uint64_t tiles = (n + kTcN - 1) / kTcN;
-        if (pair)
+        if (nkb * (kScKB / 4) <= kPackMaxF && nkb <= (uint32_t)kScMaxKB) {               // rows of at most 320 columns: through shared memory
+            const size_t psm = (size_t)nkb * kScCh * ((pair ? kPrHalf : kTcN) * 16 + 16);
+            const void *pk = pair ? (const void *)topk_pack_candidates_smem_kernel<kPrHalf> : (const void *)topk_pack_candidates_smem_kernel<kTcN>;
+            if (cudaFuncSetAttribute(pk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm) != cudaSuccess) return -1;
+            if (pair)
+                topk_pack_candidates_smem_kernel<kPrHalf><<<sms * 2, kPackThreads, psm, s>>>(table, inv_norm + c0, d / 4, ld / 4, cand_lo + c0, n, 2 * tiles, nkb, ctiles);
+            else
+                topk_pack_candidates_smem_kernel<kTcN><<<sms, kPackThreads, psm, s>>>(table, inv_norm + c0, d / 4, ld / 4, cand_lo + c0, n, tiles, nkb, ctiles);
+        } else if (pair)
             topk_pack_candidates_kernel<kPrHalf><<<sms * 32, kPrHalf, 0, s>>>(table, inv_norm + c0, d / 4, ld / 4, cand_lo + c0, n, 2 * tiles, nkb, ctiles);
         else
             topk_pack_candidates_kernel<kTcN><<<sms * 16, kTcN, 0, s>>>(table, inv_norm + c0, d / 4, ld / 4, cand_lo + c0, n, tiles, nkb, ctiles);
