@@ -410,7 +410,8 @@ topk_cosine_tc_kernel(TcParams p)
 // a ring of bulk copies alone, without MMAs, moves 50-66 GB/s per SM with 16 KB stages at any depth,
 // twice that with 32 KB and three times with 48 KB stages): with 16 KB stages that hand-over rate, not
 // bytes or MMAs, bounded the kernel (19.0 -> 16.6 ms for 8192 queries x 3 M candidates; 32 KB x 4 and
-// 64 KB x 2 measure the same).
+// 64 KB x 2 measure the same).  The next bound was what the MMA lane executes per MMA (16.6 -> 13.6 ms,
+// see its loop), and every wait in that lane still costs tensor-pipe time.
 constexpr float kScreenEps = 8.5e-3f;
 constexpr int kScKB = 32;                                        // columns per stage
 constexpr int kScCh = kScKB / 8;                                 // 16-byte chunks (8 bf16) per row and stage
